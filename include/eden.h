@@ -1,0 +1,185 @@
+/*
+ * eden.h -- C ABI of the EDEN hot path on one NVIDIA B200 (sm_100a).
+ *
+ * EDEN (arXiv 2108.08842) estimates the mean of n client vectors x_c in R^d from one
+ * short message per client.  This library implements the sender's compress step and
+ * the receiver's decompress-and-average step (the paper's Figure 1) as CUDA kernels.
+ *
+ * Conventions shared by every entry point
+ *   - "dev" pointers are CUDA device pointers on the context's device, "host" pointers
+ *     are ordinary host memory.  The caller owns every buffer it passes in; the library
+ *     owns nothing but the context object and never frees or reallocates caller memory.
+ *   - Work is enqueued on the context's stream and is asynchronous unless stated.
+ *     Host arrays (bits, seeds, pointer tables) are consumed before the call returns.
+ *   - Every function returns EDEN_OK (0) or a negative EDEN_ERR_* code.  Nothing
+ *     throws or aborts across this boundary.  Data-dependent conditions (a zero or
+ *     non-finite vector, a client with no packet) are reported through the device
+ *     status word, read with eden_status().
+ *   - bits (the per-client budget b) and seed (the randomness a sender shares with the
+ *     receiver, Section 2.1) are side information both sides agree on (Section 4.1:
+ *     "b does need to be sent or otherwise agreed upon"); they are arguments on both
+ *     sides and are not stored in the message.  Seeds must differ between clients and
+ *     between rounds; that is the caller's duty.
+ *   - Supported budgets: 0 < b <= 1 (one-bit codes; b < 1 adds the shared-seed
+ *     sparsification of Section 4.1) and the integers 2..8 (Section 3).  Other values
+ *     return EDEN_ERR_UNSUPPORTED_BITS.
+ *   - Rotation (Section 5): R = (1/sqrt D) H_D Diag(s), H_D the Sylvester-ordered
+ *     Walsh-Hadamard matrix, D = 2^ceil(log2 d') with d' = d for b >= 1 and d' = the
+ *     kept count k for b < 1; shorter vectors are zero-padded, all D coordinates are
+ *     coded and the estimate is truncated back.  Signs s come from Philox4x32-10,
+ *     key = seed, counter = (t, 0, stream, 0): stream 0 call t gives the 128 sign bits
+ *     of coordinates 128t..128t+127 (word (i/32)%4, bit i%32, 1 = minus); stream 1
+ *     call t gives the 32-bit mask keys of input coordinates 4t..4t+3.
+ *   - Message layout: coordinates in groups of 32; 32-bit word g*W + j holds bit j of
+ *     the codes of coordinates 32g..32g+31 (bit l = coordinate 32g + l), W the code
+ *     width.  A code is the rank of its quantisation value in ascending order.  A
+ *     packet is 1024 consecutive rotated coordinates = 128*W bytes.  The scale S
+ *     travels beside the codes as one fp32.
+ */
+#ifndef EDEN_H_
+#define EDEN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define EDEN_OK                    0
+#define EDEN_ERR_INVALID_ARG      -1
+#define EDEN_ERR_UNSUPPORTED_BITS -2
+#define EDEN_ERR_CUDA             -3
+#define EDEN_ERR_WORKSPACE        -4   /* workspace too small for this call */
+#define EDEN_ERR_TOO_LARGE        -5   /* d beyond EDEN_MAX_DIM */
+
+/* bits of the device status word (eden_status) */
+#define EDEN_STATUS_ZERO_VECTOR  0x1u  /* some client had ||x|| = 0: scale 0, codes 0   */
+#define EDEN_STATUS_NONFINITE    0x2u  /* some client's norm was inf/nan: its output is unspecified */
+#define EDEN_STATUS_NO_DATA      0x4u  /* some client had no packet received: it was skipped */
+
+#define EDEN_PACKET_COORDS 1024u
+#define EDEN_MAX_DIM       (1ull << 30)
+
+typedef struct eden_ctx eden_ctx;
+
+/* Per-client figures of the most recent eden_encode / eden_mean / eden_decode_accumulate
+ * call (eden_client_stats). */
+typedef struct eden_client_stat {
+    double norm2;      /* encode: ||y||^2 of the (sparsified) vector that was rotated      */
+    double dot;        /* encode: sum_i h_i Q(z_i) with h = H_D Diag(s) y (unnormalised)    */
+    double received;   /* decode: fraction p of rotated coordinates that arrived           */
+    uint32_t flags;    /* EDEN_STATUS_* bits that apply to this client                     */
+    uint32_t reserved;
+} eden_client_stat;
+
+/* ---- size rules: pure host functions of (d, bits); no GPU work ------------------- */
+
+/* k = d for bits >= 1, else floor(d*bits + 0.5) clamped to [1, d] (Section 4.1: the
+ * mask has exactly d*p ones). */
+uint64_t eden_kept_count(uint64_t d, double bits);
+/* D = smallest power of two >= (bits >= 1 ? d : k)  (Section 5; zero padding). */
+uint64_t eden_rot_dim(uint64_t d, double bits);
+/* W = 1 for bits <= 1, else (int)bits; 0 if the budget is unsupported (Section 3). */
+uint32_t eden_code_width(double bits);
+/* bytes of one client's packed codes: D*W/8 rounded up to a multiple of 16
+ * (Section 2.2.1: ceil(log2 |I|) * d bits). */
+uint64_t eden_code_bytes(uint64_t d, double bits);
+/* ceil(D / 1024): packets of one client's message (Section 4.2). */
+uint64_t eden_num_packets(uint64_t d, double bits);
+/* 32-bit words of a received-packet bitmap: ceil(packets / 32). */
+uint64_t eden_recv_mask_words(uint64_t d, double bits);
+/* Bytes of device workspace that lets eden_encode / eden_mean process n_batch clients
+ * of dimension up to d_max per launch group (any budgets).  A smaller workspace is
+ * accepted as long as it holds one client: calls then run in several groups. */
+uint64_t eden_workspace_bytes(uint64_t d_max, uint32_t n_batch);
+
+/* The quantiser the library uses for code width W (1..8): 2^W values in ascending
+ * order and the 2^W - 1 interval boundaries between them, rounded to fp32
+ * (Section 3: Lloyd-Max for N(0,1), centre-of-mass values).  Host arrays, host only. */
+int eden_table(uint32_t W, float* centroids, float* boundaries);
+
+/* ---- context ---------------------------------------------------------------------- */
+
+/* Creates a context bound to a device, a stream (cudaStream_t passed as void*, NULL =
+ * the default stream) and a caller-allocated device workspace (256-byte aligned).  The
+ * context keeps pointers into the workspace; the caller must keep it alive and must
+ * not use it while a call is in flight.  Uploads the quantiser tables (synchronous). */
+int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
+                void* workspace_dev, uint64_t workspace_bytes);
+int eden_destroy(eden_ctx* ctx);
+
+/* ---- sender: Sections 2.2.1, 2.3, 4.1 --------------------------------------------- */
+
+/* Compresses n independent clients.
+ *   x      dev, fp32, n rows, row c starts at x + c*ld_x, ld_x >= d; read only.
+ *   bits   host, n budgets.          seeds  host, n shared seeds.
+ *   codes  host array of n dev pointers, each to eden_code_bytes(d, bits[c]) bytes,
+ *          16-byte aligned; overwritten with the packed codes Q(eta_x R(x)).
+ *   scales dev, fp32[n]; scales[c] = S_c = ||x_c||^2 / <R(x_c), Q(eta R(x_c))>
+ *          (for b < 1: the scale of the sparsified, 1/p-rescaled vector).
+ * A zero vector gives scale 0 and all-zero codes (status ZERO_VECTOR). */
+int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                const double* bits, const uint64_t* seeds,
+                uint8_t* const* codes, float* scales);
+
+/* ---- receiver: Sections 2.2.2, 4.1, 4.2 ------------------------------------------- */
+
+/* acc[i] += sum_c x_hat_c[i] over the n given clients, x_hat_c = (S_c/p_c) R_c^-1(Q_c)
+ * scattered back through the client's sparsification mask when b < 1.
+ *   codes      host array of n dev pointers (layout above); scales dev fp32[n].
+ *   recv_masks host array of n dev pointers or NULL; entry c (NULL = nothing lost)
+ *              points to eden_recv_mask_words() words, bit i of word i/32 = packet i
+ *              arrived.  Lost coordinates count as 0 and p_c = received/D (Section 4.2).
+ *   acc        dev fp32[d], read and written.
+ *   n_used     host, optional: set to n; clients with no packet received are skipped
+ *              and flagged (status NO_DATA) but still counted, because the mean of
+ *              Section 2.2.2 is over all n senders.
+ * No per-client estimate is stored for b >= 1; clients with b < 1 use the workspace. */
+int eden_decode_accumulate(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                           const double* bits, const uint64_t* seeds,
+                           const uint32_t* const* recv_masks,
+                           uint64_t d, uint32_t n, float* acc, uint32_t* n_used);
+
+/* mean[i] = (1/n) sum_c x_hat_c[i]; same inputs; mean (dev fp32[d]) is overwritten. */
+int eden_mean(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+              const double* bits, const uint64_t* seeds,
+              const uint32_t* const* recv_masks,
+              uint64_t d, uint32_t n, float* mean);
+
+/* The sparsification mask of Section 4.1 for (seed, d, bits < 1) as a bitmap:
+ * mask_bits dev, ceil(d/32) words, bit i of word i/32 = coordinate i is kept. */
+int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bits,
+                             uint32_t* mask_bits);
+
+/* ---- the same two steps on host memory (copies included) --------------------------- */
+
+/* x, codes (array of n host pointers), scales are HOST buffers (pinned memory makes the
+ * copies asynchronous).  Copies x to the device, encodes, copies codes and scales back
+ * and synchronises the stream.  Needs eden_host_workspace_bytes() of workspace. */
+int eden_encode_host(eden_ctx* ctx, const float* x_host, uint64_t ld_x, uint64_t d, uint32_t n,
+                     const double* bits, const uint64_t* seeds,
+                     uint8_t* const* codes_host, float* scales_host);
+/* codes, scales, recv_masks (entries may be NULL), mean are HOST buffers. */
+int eden_mean_host(eden_ctx* ctx, const uint8_t* const* codes_host, const float* scales_host,
+                   const double* bits, const uint64_t* seeds,
+                   const uint32_t* const* recv_masks_host,
+                   uint64_t d, uint32_t n, float* mean_host);
+/* workspace for the two calls above: staging for n vectors, their codes and the mean
+ * on top of eden_workspace_bytes(d, n). */
+uint64_t eden_host_workspace_bytes(uint64_t d, uint32_t n);
+
+/* ---- status ----------------------------------------------------------------------- */
+
+/* Synchronises the stream and returns the OR of EDEN_STATUS_* bits raised since the
+ * last eden_status call (then clears them). */
+int eden_status(eden_ctx* ctx, uint32_t* device_status_word);
+/* Synchronises and copies the per-client figures of the most recent call (host array, n). */
+int eden_client_stats(eden_ctx* ctx, uint32_t n, eden_client_stat* out);
+/* Number of kernels the library has launched on this context so far. */
+uint64_t eden_launch_count(const eden_ctx* ctx);
+const char* eden_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EDEN_H_ */

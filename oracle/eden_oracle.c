@@ -310,7 +310,7 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
     uint64_t k = eden_oracle_kept_count(d, bits);
     uint64_t D = eden_oracle_rot_dim(d, bits);
     uint32_t W = eden_oracle_code_width(bits);
-    uint64_t n_words = (D * W + 31u) / 32u;
+    uint64_t n_words = ((D + 31u) / 32u) * W; /* W words per group of 32 coordinates */
 
     double *y = (double *)calloc(D, sizeof(double));
     if (!y) return -1;

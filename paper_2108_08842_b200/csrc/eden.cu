@@ -1,0 +1,728 @@
+// C ABI of the EDEN hot path (declared in include/eden.h): argument checks, the pass
+// plan, workspace carving and kernel launches.  All arithmetic runs in the kernels.
+#include "../../include/eden.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "eden_device.cuh"
+#include "kernels_generic.cuh"
+#include "kernels_select.cuh"
+#include "lloyd_max.h"
+
+using namespace eden;
+
+// ------------------------------------------------------------------------------------
+// size rules
+// ------------------------------------------------------------------------------------
+static int ceil_log2(uint64_t v)
+{
+    int l = 0;
+    while ((1ull << l) < v) ++l;
+    return l;
+}
+
+extern "C" uint64_t eden_kept_count(uint64_t d, double bits)
+{
+    if (bits >= 1.0) return d;
+    uint64_t k = (uint64_t)std::floor((double)d * bits + 0.5);
+    if (k < 1) k = 1;
+    if (k > d) k = d;
+    return k;
+}
+
+extern "C" uint64_t eden_rot_dim(uint64_t d, double bits)
+{
+    return 1ull << ceil_log2(eden_kept_count(d, bits));
+}
+
+extern "C" uint32_t eden_code_width(double bits)
+{
+    if (!(bits > 0.0)) return 0;
+    if (bits <= 1.0) return 1;
+    if (bits > 8.0 || bits != std::floor(bits)) return 0;
+    return (uint32_t)bits;
+}
+
+extern "C" uint64_t eden_code_bytes(uint64_t d, double bits)
+{
+    const uint64_t D = eden_rot_dim(d, bits);
+    const uint64_t bytes = ((D + 31) / 32) * eden_code_width(bits) * 4;
+    return (bytes + 15) / 16 * 16;
+}
+
+extern "C" uint64_t eden_num_packets(uint64_t d, double bits)
+{
+    return (eden_rot_dim(d, bits) + EDEN_PACKET_COORDS - 1) / EDEN_PACKET_COORDS;
+}
+
+extern "C" uint64_t eden_recv_mask_words(uint64_t d, double bits)
+{
+    return (eden_num_packets(d, bits) + 31) / 32;
+}
+
+// ------------------------------------------------------------------------------------
+// quantiser tables (host copy, built once per process)
+// ------------------------------------------------------------------------------------
+namespace {
+
+struct Tables {
+    float pos_boundary[256];
+    float pos_value[256];
+    std::vector<float> centroids[9], boundaries[9];
+};
+
+const Tables& tables()
+{
+    static Tables t;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        std::memset(t.pos_boundary, 0, sizeof(t.pos_boundary));
+        std::memset(t.pos_value, 0, sizeof(t.pos_value));
+        for (int W = 1; W <= 8; ++W) {
+            std::vector<double> c, b;
+            lloyd_max_table(W, c, b);
+            t.centroids[W].assign(c.begin(), c.end());
+            t.boundaries[W].assign(b.begin(), b.end());
+            const int half = 1 << (W - 1), off = half - 1;
+            for (int j = 0; j < half; ++j) t.pos_value[off + j] = (float)c[half + j];
+            for (int j = 0; j + 1 < half; ++j) t.pos_boundary[off + j] = (float)b[half + j];
+        }
+    });
+    return t;
+}
+
+uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+constexpr uint64_t kHistBytes = 2ull * 65536 * sizeof(uint32_t);
+
+// fixed part of the workspace: status word, mask-selection scratch
+struct FixedLayout {
+    uint64_t status, sel, hist, chunks, end;
+};
+
+FixedLayout fixed_layout(uint64_t d_max)
+{
+    FixedLayout f;
+    f.status = 0;
+    f.sel = 256;
+    f.hist = 512;
+    f.chunks = f.hist + kHistBytes;
+    const uint64_t n_chunks = (d_max + kSelChunk - 1) / kSelChunk;
+    f.end = align_up(f.chunks + n_chunks * sizeof(unsigned long long), 256);
+    return f;
+}
+
+uint64_t per_client_bytes() { return align_up(sizeof(ClientDesc), 16) + align_up(sizeof(ClientState), 16); }
+
+}  // namespace
+
+extern "C" uint64_t eden_workspace_bytes(uint64_t d_max, uint32_t n_batch)
+{
+    if (n_batch == 0) n_batch = 1;
+    const uint64_t D = 1ull << ceil_log2(d_max ? d_max : 1);
+    return fixed_layout(d_max).end + align_up(per_client_bytes() * n_batch, 256) + 1024 +
+           (uint64_t)n_batch * D * sizeof(float);
+}
+
+extern "C" int eden_table(uint32_t W, float* centroids, float* boundaries)
+{
+    if (W < 1 || W > 8 || !centroids || !boundaries) return EDEN_ERR_INVALID_ARG;
+    const Tables& t = tables();
+    std::copy(t.centroids[W].begin(), t.centroids[W].end(), centroids);
+    std::copy(t.boundaries[W].begin(), t.boundaries[W].end(), boundaries);
+    return EDEN_OK;
+}
+
+extern "C" const char* eden_strerror(int code)
+{
+    switch (code) {
+        case EDEN_OK: return "ok";
+        case EDEN_ERR_INVALID_ARG: return "invalid argument";
+        case EDEN_ERR_UNSUPPORTED_BITS: return "unsupported bit budget (use 0 < b <= 1 or an integer 2..8)";
+        case EDEN_ERR_CUDA: return "CUDA error";
+        case EDEN_ERR_WORKSPACE: return "workspace too small";
+        case EDEN_ERR_TOO_LARGE: return "dimension too large";
+        default: return "unknown error";
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// context
+// ------------------------------------------------------------------------------------
+struct eden_ctx {
+    int device;
+    cudaStream_t stream;
+    char* ws;
+    uint64_t ws_bytes;
+    uint64_t launches;
+    std::vector<uint32_t> order;     // processing order of the last call: order[j] = client
+    uint64_t states_off;             // where the last call put its ClientState array
+};
+
+#define CUDA_OK(expr)                                 \
+    do {                                              \
+        if ((expr) != cudaSuccess) return EDEN_ERR_CUDA; \
+    } while (0)
+
+#define LAUNCH(ctx, kernel, grid, block, smem, ...)                          \
+    do {                                                                     \
+        kernel<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);           \
+        ++(ctx)->launches;                                                   \
+        if (cudaGetLastError() != cudaSuccess) return EDEN_ERR_CUDA;         \
+    } while (0)
+
+extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
+                           void* workspace_dev, uint64_t workspace_bytes)
+{
+    if (!out || !workspace_dev || ((uintptr_t)workspace_dev & 255u)) return EDEN_ERR_INVALID_ARG;
+    if (workspace_bytes < fixed_layout(1).end) return EDEN_ERR_WORKSPACE;
+    CUDA_OK(cudaSetDevice(cuda_device));
+    eden_ctx* ctx = new (std::nothrow) eden_ctx();
+    if (!ctx) return EDEN_ERR_INVALID_ARG;
+    ctx->device = cuda_device;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->ws = (char*)workspace_dev;
+    ctx->ws_bytes = workspace_bytes;
+    ctx->launches = 0;
+    ctx->states_off = 0;
+    const Tables& t = tables();
+    if (cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_pos_value, t.pos_value, sizeof(t.pos_value)) != cudaSuccess ||
+        cudaMemsetAsync(ctx->ws, 0, 256, ctx->stream) != cudaSuccess ||
+        cudaStreamSynchronize(ctx->stream) != cudaSuccess) {
+        delete ctx;
+        return EDEN_ERR_CUDA;
+    }
+    *out = ctx;
+    return EDEN_OK;
+}
+
+extern "C" int eden_destroy(eden_ctx* ctx)
+{
+    if (!ctx) return EDEN_ERR_INVALID_ARG;
+    delete ctx;
+    return EDEN_OK;
+}
+
+extern "C" uint64_t eden_launch_count(const eden_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int eden_status(eden_ctx* ctx, uint32_t* word)
+{
+    if (!ctx || !word) return EDEN_ERR_INVALID_ARG;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    CUDA_OK(cudaMemcpyAsync(word, ctx->ws, sizeof(uint32_t), cudaMemcpyDeviceToHost, ctx->stream));
+    CUDA_OK(cudaMemsetAsync(ctx->ws, 0, sizeof(uint32_t), ctx->stream));
+    CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    return EDEN_OK;
+}
+
+extern "C" int eden_client_stats(eden_ctx* ctx, uint32_t n, eden_client_stat* out)
+{
+    if (!ctx || !out || n != ctx->order.size()) return EDEN_ERR_INVALID_ARG;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    std::vector<ClientState> st(n);
+    CUDA_OK(cudaMemcpyAsync(st.data(), ctx->ws + ctx->states_off, n * sizeof(ClientState),
+                            cudaMemcpyDeviceToHost, ctx->stream));
+    CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    for (uint32_t j = 0; j < n; ++j) {
+        eden_client_stat& o = out[ctx->order[j]];
+        o.norm2 = st[j].norm2;
+        o.dot = st[j].dot;
+        o.received = st[j].received;
+        o.flags = st[j].flags;
+        o.reserved = 0;
+    }
+    return EDEN_OK;
+}
+
+// ------------------------------------------------------------------------------------
+// planning
+// ------------------------------------------------------------------------------------
+namespace {
+
+struct ClientPlan {
+    uint32_t index;      // position in the caller's arrays
+    uint64_t k, D;
+    int L, W;
+    bool subbit;
+    bool needs_work;
+};
+
+// A set of clients of one rotation dimension launched together.
+struct Group {
+    std::vector<uint32_t> members;   // indices into the plan array
+    int L;
+    bool subbit;
+};
+
+struct CallLayout {
+    uint64_t descs_off, states_off, work_off, work_bytes;
+};
+
+int plan_clients(uint64_t d, uint32_t n, const double* bits, std::vector<ClientPlan>& plan)
+{
+    if (d == 0 || n == 0 || !bits) return EDEN_ERR_INVALID_ARG;
+    if (d > EDEN_MAX_DIM) return EDEN_ERR_TOO_LARGE;
+    plan.resize(n);
+    for (uint32_t c = 0; c < n; ++c) {
+        const uint32_t W = eden_code_width(bits[c]);
+        if (W == 0) return EDEN_ERR_UNSUPPORTED_BITS;
+        ClientPlan& p = plan[c];
+        p.index = c;
+        p.k = eden_kept_count(d, bits[c]);
+        p.D = eden_rot_dim(d, bits[c]);
+        p.L = ceil_log2(p.D);
+        p.W = (int)W;
+        p.subbit = bits[c] < 1.0;
+        p.needs_work = p.subbit || p.L > kGenericTileLog;
+    }
+    return EDEN_OK;
+}
+
+int carve(const eden_ctx* ctx, uint64_t d, uint32_t n, CallLayout& lay)
+{
+    const FixedLayout f = fixed_layout(d);
+    lay.descs_off = f.end;
+    lay.states_off = lay.descs_off + align_up(sizeof(ClientDesc) * (uint64_t)n, 256);
+    lay.work_off = lay.states_off + align_up(sizeof(ClientState) * (uint64_t)n, 256);
+    if (lay.work_off > ctx->ws_bytes) return EDEN_ERR_WORKSPACE;
+    lay.work_bytes = ctx->ws_bytes - lay.work_off;
+    return EDEN_OK;
+}
+
+// Groups: clients with b >= 1 by rotation dimension, split so that each group's work
+// buffers fit; every client with b < 1 alone (the mask scratch is shared).
+int make_groups(const std::vector<ClientPlan>& plan, uint64_t work_bytes, std::vector<Group>& groups)
+{
+    std::vector<uint32_t> idx;
+    for (uint32_t c = 0; c < plan.size(); ++c)
+        if (!plan[c].subbit) idx.push_back(c);
+    std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) { return plan[a].L > plan[b].L; });
+    size_t i = 0;
+    while (i < idx.size()) {
+        Group g;
+        g.L = plan[idx[i]].L;
+        g.subbit = false;
+        const uint64_t need = plan[idx[i]].needs_work ? plan[idx[i]].D * sizeof(float) : 0;
+        if (need > work_bytes) return EDEN_ERR_WORKSPACE;
+        uint64_t used = 0;
+        while (i < idx.size() && plan[idx[i]].L == g.L && used + need <= work_bytes &&
+               g.members.size() < 32768) {
+            g.members.push_back(idx[i]);
+            used += need;
+            ++i;
+        }
+        groups.push_back(g);
+    }
+    for (uint32_t c = 0; c < plan.size(); ++c) {
+        if (!plan[c].subbit) continue;
+        if (plan[c].D * sizeof(float) > work_bytes) return EDEN_ERR_WORKSPACE;
+        Group g;
+        g.L = plan[c].L;
+        g.subbit = true;
+        g.members.push_back(c);
+        groups.push_back(g);
+    }
+    return EDEN_OK;
+}
+
+// Column passes over the bits above the row pass, top range first.
+struct BitRange { int lo, lr; };
+
+void column_ranges(int L, int lc, int max_lr, std::vector<BitRange>& out)
+{
+    const int rem = L - lc;
+    if (rem <= 0) return;
+    const int passes = (rem + max_lr - 1) / max_lr;
+    int hi = L;
+    for (int p = 0; p < passes; ++p) {
+        const int lr = (hi - lc + (passes - p) - 1) / (passes - p);
+        out.push_back({hi - lr, lr});
+        hi -= lr;
+    }
+}
+
+PassGeom column_geom(const BitRange& r)
+{
+    PassGeom g;
+    g.lr = r.lr;
+    g.lo = r.lo;
+    g.lw = std::min(r.lo, kGenericTileLog - r.lr);
+    g.lt = g.lw + g.lr;
+    return g;
+}
+
+PassGeom row_geom(int lc) { return PassGeom{lc, lc, lc, 0}; }
+
+// Exact-size mask selection for one client (Section 4.1): fills the MaskSelect and the
+// scanned chunk offsets in the fixed scratch.
+int run_selection(eden_ctx* ctx, const FixedLayout& f, uint64_t seed, uint64_t d, uint64_t k)
+{
+    MaskSelect* sel = (MaskSelect*)(ctx->ws + f.sel);
+    uint32_t* hist = (uint32_t*)(ctx->ws + f.hist);
+    unsigned long long* chunks = (unsigned long long*)(ctx->ws + f.chunks);
+    const uint64_t calls = (d + 3) / 4;
+    const unsigned grid = (unsigned)((calls + kSelThreads - 1) / kSelThreads);
+    CUDA_OK(cudaMemsetAsync(hist, 0, kHistBytes, ctx->stream));
+    LAUNCH(ctx, k_sel_hist, grid, kSelThreads, 0, seed, d, 0, sel, hist);
+    LAUNCH(ctx, k_sel_find, 1, 1024, 0, hist, k, 0, sel);
+    LAUNCH(ctx, k_sel_hist, grid, kSelThreads, 0, seed, d, 1, sel, hist + 65536);
+    LAUNCH(ctx, k_sel_find, 1, 1024, 0, hist + 65536, k, 1, sel);
+    LAUNCH(ctx, k_sel_chunk_count, grid, kSelThreads, 0, seed, d, sel, chunks);
+    LAUNCH(ctx, k_sel_chunk_scan, 1, 1024, 0, chunks, (uint64_t)grid);
+    return EDEN_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------
+// sender
+// ------------------------------------------------------------------------------------
+extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                           const double* bits, const uint64_t* seeds,
+                           uint8_t* const* codes, float* scales)
+{
+    if (!ctx || !x || !seeds || !codes || !scales || ld_x < d) return EDEN_ERR_INVALID_ARG;
+    std::vector<ClientPlan> plan;
+    int rc = plan_clients(d, n, bits, plan);
+    if (rc) return rc;
+    for (uint32_t c = 0; c < n; ++c)
+        if (!codes[c] || ((uintptr_t)codes[c] & 15u)) return EDEN_ERR_INVALID_ARG;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    CallLayout lay;
+    rc = carve(ctx, d, n, lay);
+    if (rc) return rc;
+    std::vector<Group> groups;
+    rc = make_groups(plan, lay.work_bytes, groups);
+    if (rc) return rc;
+    const FixedLayout f = fixed_layout(d);
+
+    // descriptors in processing order
+    std::vector<ClientDesc> descs;
+    descs.reserve(n);
+    ctx->order.clear();
+    std::vector<uint32_t> group_start;
+    for (const Group& g : groups) {
+        group_start.push_back((uint32_t)descs.size());
+        uint64_t off = 0;
+        for (uint32_t m : g.members) {
+            const ClientPlan& p = plan[m];
+            ClientDesc cd;
+            std::memset(&cd, 0, sizeof(cd));
+            cd.work = p.needs_work ? (float*)(ctx->ws + lay.work_off + off) : nullptr;
+            if (p.needs_work) off += p.D * sizeof(float);
+            cd.src = p.subbit ? cd.work : x + (uint64_t)p.index * ld_x;
+            cd.codes = (uint32_t*)codes[p.index];
+            cd.recv = nullptr;
+            cd.seed = seeds[p.index];
+            cd.valid = p.k;
+            cd.d = d;
+            cd.W = (uint32_t)p.W;
+            cd.L = (uint32_t)p.L;
+            cd.subbit = p.subbit;
+            cd.index = p.index;
+            cd.extra_scale = p.subbit ? (double)d / (double)p.k : 1.0;
+            cd.mean_scale = 1.0;
+            descs.push_back(cd);
+            ctx->order.push_back(p.index);
+        }
+    }
+    ClientDesc* d_descs = (ClientDesc*)(ctx->ws + lay.descs_off);
+    ClientState* d_states = (ClientState*)(ctx->ws + lay.states_off);
+    uint32_t* d_status = (uint32_t*)(ctx->ws + f.status);
+    ctx->states_off = lay.states_off;
+    CUDA_OK(cudaMemcpyAsync(d_descs, descs.data(), sizeof(ClientDesc) * n, cudaMemcpyHostToDevice, ctx->stream));
+    CUDA_OK(cudaMemsetAsync(d_states, 0, sizeof(ClientState) * n, ctx->stream));
+
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
+        if (g.subbit) {
+            const ClientPlan& p = plan[g.members[0]];
+            rc = run_selection(ctx, f, seeds[p.index], d, p.k);
+            if (rc) return rc;
+            const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
+            LAUNCH(ctx, k_sel_apply<SEL_COMPACT>, grid, kSelThreads, 0, seeds[p.index], d,
+                   (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
+                   x + (uint64_t)p.index * ld_x, descs[first].work, (uint32_t*)nullptr);
+        }
+        if (g.L <= kGenericTileLog) {
+            const PassGeom rg = row_geom(g.L);
+            LAUNCH(ctx, k_enc_last<true>, dim3(1, gn), kGenericThreads, sizeof(float) << g.L,
+                   d_descs + first, d_states + first, rg);
+        } else {
+            const int lc = kGenericTileLog;
+            std::vector<BitRange> cols;
+            column_ranges(g.L, lc, 8, cols);
+            for (size_t pi = 0; pi < cols.size(); ++pi) {
+                const PassGeom cg = column_geom(cols[pi]);
+                const unsigned tiles = (unsigned)((1ull << g.L) >> cg.lt);
+                if (pi == 0)
+                    LAUNCH(ctx, k_enc_first, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
+                           d_descs + first, d_states + first, cg);
+                else
+                    LAUNCH(ctx, k_mid, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
+                           d_descs + first, cg);
+            }
+            const PassGeom rg = row_geom(lc);
+            LAUNCH(ctx, k_enc_last<false>, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
+                   sizeof(float) << lc, d_descs + first, d_states + first, rg);
+        }
+    }
+    LAUNCH(ctx, k_enc_scale, (n + 127) / 128, 128, 0, d_descs, d_states, scales, n, d_status);
+    return EDEN_OK;
+}
+
+// ------------------------------------------------------------------------------------
+// receiver
+// ------------------------------------------------------------------------------------
+static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                         const double* bits, const uint64_t* seeds,
+                         const uint32_t* const* recv_masks, uint64_t d, uint32_t n,
+                         float* out, bool mean)
+{
+    if (!ctx || !codes || !scales || !seeds || !out) return EDEN_ERR_INVALID_ARG;
+    std::vector<ClientPlan> plan;
+    int rc = plan_clients(d, n, bits, plan);
+    if (rc) return rc;
+    for (uint32_t c = 0; c < n; ++c)
+        if (!codes[c] || ((uintptr_t)codes[c] & 3u)) return EDEN_ERR_INVALID_ARG;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    CallLayout lay;
+    rc = carve(ctx, d, n, lay);
+    if (rc) return rc;
+    std::vector<Group> groups;
+    rc = make_groups(plan, lay.work_bytes, groups);
+    if (rc) return rc;
+    const FixedLayout f = fixed_layout(d);
+
+    std::vector<ClientDesc> descs;
+    descs.reserve(n);
+    ctx->order.clear();
+    std::vector<uint32_t> group_start;
+    for (const Group& g : groups) {
+        group_start.push_back((uint32_t)descs.size());
+        uint64_t off = 0;
+        for (uint32_t m : g.members) {
+            const ClientPlan& p = plan[m];
+            ClientDesc cd;
+            std::memset(&cd, 0, sizeof(cd));
+            cd.work = p.needs_work ? (float*)(ctx->ws + lay.work_off + off) : nullptr;
+            if (p.needs_work) off += p.D * sizeof(float);
+            cd.src = nullptr;
+            cd.codes = (uint32_t*)codes[p.index];
+            cd.recv = recv_masks ? recv_masks[p.index] : nullptr;
+            cd.seed = seeds[p.index];
+            cd.valid = p.k;
+            cd.d = d;
+            cd.W = (uint32_t)p.W;
+            cd.L = (uint32_t)p.L;
+            cd.subbit = p.subbit;
+            cd.index = p.index;
+            cd.extra_scale = 1.0;
+            cd.mean_scale = mean ? 1.0 / (double)n : 1.0;
+            descs.push_back(cd);
+            ctx->order.push_back(p.index);
+        }
+    }
+    ClientDesc* d_descs = (ClientDesc*)(ctx->ws + lay.descs_off);
+    ClientState* d_states = (ClientState*)(ctx->ws + lay.states_off);
+    uint32_t* d_status = (uint32_t*)(ctx->ws + f.status);
+    ctx->states_off = lay.states_off;
+    CUDA_OK(cudaMemcpyAsync(d_descs, descs.data(), sizeof(ClientDesc) * n, cudaMemcpyHostToDevice, ctx->stream));
+    CUDA_OK(cudaMemsetAsync(d_states, 0, sizeof(ClientState) * n, ctx->stream));
+    LAUNCH(ctx, k_dec_prep, n, 256, 0, d_descs, d_states, scales, d_status);
+
+    // the first group with b >= 1 covers every output coordinate, so for the mean it may
+    // overwrite; everything after it accumulates
+    bool written = !mean;
+    if (mean && (groups.empty() || groups[0].subbit)) {
+        CUDA_OK(cudaMemsetAsync(out, 0, d * sizeof(float), ctx->stream));
+        written = true;
+    }
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+        const Group& g = groups[gi];
+        const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
+        int mode = g.subbit ? OUT_YHAT : (written ? OUT_ACC : OUT_WRITE);
+        if (g.subbit) {
+            const ClientPlan& p = plan[g.members[0]];
+            rc = run_selection(ctx, f, seeds[p.index], d, p.k);
+            if (rc) return rc;
+        }
+        if (g.L <= kGenericTileLog) {
+            const PassGeom rg = row_geom(g.L);
+            LAUNCH(ctx, k_dec_last<true>, dim3(1), kGenericThreads, sizeof(float) << g.L,
+                   d_descs + first, d_states + first, gn, rg, out, d, mode);
+        } else {
+            const int lc = kGenericTileLog;
+            LAUNCH(ctx, k_dec_first, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
+                   sizeof(float) << lc, d_descs + first, row_geom(lc));
+            std::vector<BitRange> cols;
+            column_ranges(g.L, lc, 8, cols);
+            for (size_t pi = 0; pi < cols.size(); ++pi) {
+                const PassGeom cg = column_geom(cols[pi]);
+                const unsigned tiles = (unsigned)((1ull << g.L) >> cg.lt);
+                if (pi + 1 < cols.size())
+                    LAUNCH(ctx, k_mid, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
+                           d_descs + first, cg);
+                else
+                    LAUNCH(ctx, k_dec_last<false>, dim3(tiles), kGenericThreads, sizeof(float) << cg.lt,
+                           d_descs + first, d_states + first, gn, cg, out, d, mode);
+            }
+        }
+        if (g.subbit) {
+            const ClientPlan& p = plan[g.members[0]];
+            const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
+            LAUNCH(ctx, k_sel_apply<SEL_SCATTER_ACC>, grid, kSelThreads, 0, seeds[p.index], d,
+                   (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
+                   (const float*)descs[first].work, out, (uint32_t*)nullptr);
+        } else {
+            written = true;
+        }
+    }
+    return EDEN_OK;
+}
+
+extern "C" int eden_decode_accumulate(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                                      const double* bits, const uint64_t* seeds,
+                                      const uint32_t* const* recv_masks,
+                                      uint64_t d, uint32_t n, float* acc, uint32_t* n_used)
+{
+    const int rc = decode_common(ctx, codes, scales, bits, seeds, recv_masks, d, n, acc, false);
+    if (rc == EDEN_OK && n_used) *n_used = n;
+    return rc;
+}
+
+extern "C" int eden_mean(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                         const double* bits, const uint64_t* seeds,
+                         const uint32_t* const* recv_masks,
+                         uint64_t d, uint32_t n, float* mean)
+{
+    return decode_common(ctx, codes, scales, bits, seeds, recv_masks, d, n, mean, true);
+}
+
+extern "C" int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bits,
+                                        uint32_t* mask_bits)
+{
+    if (!ctx || !mask_bits || d == 0 || !(bits > 0.0) || !(bits < 1.0)) return EDEN_ERR_INVALID_ARG;
+    if (d > EDEN_MAX_DIM) return EDEN_ERR_TOO_LARGE;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    const FixedLayout f = fixed_layout(d);
+    if (f.end > ctx->ws_bytes) return EDEN_ERR_WORKSPACE;
+    const int rc = run_selection(ctx, f, seed, d, eden_kept_count(d, bits));
+    if (rc) return rc;
+    const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
+    LAUNCH(ctx, k_sel_apply<SEL_MASK_BITS>, grid, kSelThreads, 0, seed, d,
+           (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
+           (const float*)nullptr, (float*)nullptr, mask_bits);
+    return EDEN_OK;
+}
+
+// ------------------------------------------------------------------------------------
+// host-buffer variants: stage through the tail of the workspace
+// ------------------------------------------------------------------------------------
+extern "C" uint64_t eden_host_workspace_bytes(uint64_t d, uint32_t n)
+{
+    const uint64_t D = 1ull << ceil_log2(d ? d : 1);
+    // vectors, codes at 8 bits, scales, masks, mean
+    const uint64_t staging = (uint64_t)n * align_up(d * sizeof(float), 256) +
+                             (uint64_t)n * align_up(D, 256) + align_up(n * sizeof(float), 256) +
+                             (uint64_t)n * align_up(((D + 1023) / 1024 + 31) / 32 * 4, 256) +
+                             align_up(d * sizeof(float), 256) + 4096;
+    return eden_workspace_bytes(d, n) + staging;
+}
+
+namespace {
+struct Staging {
+    char* base;
+    uint64_t left;
+    void* take(uint64_t bytes)
+    {
+        bytes = align_up(bytes, 256);
+        if (bytes > left) return nullptr;
+        left -= bytes;
+        return base + left;   // carve downwards from the end of the workspace
+    }
+};
+}  // namespace
+
+extern "C" int eden_encode_host(eden_ctx* ctx, const float* x_host, uint64_t ld_x, uint64_t d, uint32_t n,
+                                const double* bits, const uint64_t* seeds,
+                                uint8_t* const* codes_host, float* scales_host)
+{
+    if (!ctx || !x_host || !bits || !seeds || !codes_host || !scales_host || ld_x < d || d == 0 || n == 0)
+        return EDEN_ERR_INVALID_ARG;
+    for (uint32_t c = 0; c < n; ++c)
+        if (eden_code_width(bits[c]) == 0) return EDEN_ERR_UNSUPPORTED_BITS;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    Staging st{ctx->ws, ctx->ws_bytes};
+    const uint64_t row = align_up(d * sizeof(float), 256) / sizeof(float);
+    float* x_dev = (float*)st.take((uint64_t)n * row * sizeof(float));
+    float* scales_dev = (float*)st.take(n * sizeof(float));
+    if (!x_dev || !scales_dev) return EDEN_ERR_WORKSPACE;
+    std::vector<uint8_t*> codes_dev(n);
+    for (uint32_t c = 0; c < n; ++c) {
+        codes_dev[c] = (uint8_t*)st.take(eden_code_bytes(d, bits[c]));
+        if (!codes_dev[c]) return EDEN_ERR_WORKSPACE;
+    }
+    CUDA_OK(cudaMemcpy2DAsync(x_dev, row * sizeof(float), x_host, ld_x * sizeof(float),
+                              d * sizeof(float), n, cudaMemcpyHostToDevice, ctx->stream));
+    const uint64_t saved = ctx->ws_bytes;
+    ctx->ws_bytes = st.left;
+    const int rc = eden_encode(ctx, x_dev, row, d, n, bits, seeds, codes_dev.data(), scales_dev);
+    ctx->ws_bytes = saved;
+    if (rc) return rc;
+    for (uint32_t c = 0; c < n; ++c)
+        CUDA_OK(cudaMemcpyAsync(codes_host[c], codes_dev[c], eden_code_bytes(d, bits[c]),
+                                cudaMemcpyDeviceToHost, ctx->stream));
+    CUDA_OK(cudaMemcpyAsync(scales_host, scales_dev, n * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    return EDEN_OK;
+}
+
+extern "C" int eden_mean_host(eden_ctx* ctx, const uint8_t* const* codes_host, const float* scales_host,
+                              const double* bits, const uint64_t* seeds,
+                              const uint32_t* const* recv_masks_host,
+                              uint64_t d, uint32_t n, float* mean_host)
+{
+    if (!ctx || !codes_host || !scales_host || !bits || !seeds || !mean_host || d == 0 || n == 0)
+        return EDEN_ERR_INVALID_ARG;
+    for (uint32_t c = 0; c < n; ++c)
+        if (eden_code_width(bits[c]) == 0) return EDEN_ERR_UNSUPPORTED_BITS;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    Staging st{ctx->ws, ctx->ws_bytes};
+    float* mean_dev = (float*)st.take(d * sizeof(float));
+    float* scales_dev = (float*)st.take(n * sizeof(float));
+    if (!mean_dev || !scales_dev) return EDEN_ERR_WORKSPACE;
+    std::vector<const uint8_t*> codes_dev(n);
+    std::vector<const uint32_t*> masks_dev(n, nullptr);
+    for (uint32_t c = 0; c < n; ++c) {
+        const uint64_t cb = eden_code_bytes(d, bits[c]);
+        uint8_t* p = (uint8_t*)st.take(cb);
+        if (!p) return EDEN_ERR_WORKSPACE;
+        CUDA_OK(cudaMemcpyAsync(p, codes_host[c], cb, cudaMemcpyHostToDevice, ctx->stream));
+        codes_dev[c] = p;
+        if (recv_masks_host && recv_masks_host[c]) {
+            const uint64_t mb = eden_recv_mask_words(d, bits[c]) * 4;
+            uint32_t* m = (uint32_t*)st.take(mb);
+            if (!m) return EDEN_ERR_WORKSPACE;
+            CUDA_OK(cudaMemcpyAsync(m, recv_masks_host[c], mb, cudaMemcpyHostToDevice, ctx->stream));
+            masks_dev[c] = m;
+        }
+    }
+    CUDA_OK(cudaMemcpyAsync(scales_dev, scales_host, n * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+    const uint64_t saved = ctx->ws_bytes;
+    ctx->ws_bytes = st.left;
+    const int rc = eden_mean(ctx, codes_dev.data(), scales_dev, bits, seeds,
+                             recv_masks_host ? masks_dev.data() : nullptr, d, n, mean_dev);
+    ctx->ws_bytes = saved;
+    if (rc) return rc;
+    CUDA_OK(cudaMemcpyAsync(mean_host, mean_dev, d * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    return EDEN_OK;
+}

@@ -1,0 +1,364 @@
+// Shape-generic transform kernels: any rotation dimension, any pass split.  A tile of
+// 2^lt floats is staged in shared memory and a range of its index bits is transformed
+// with radix-8 register butterflies between barriers.  These kernels serve the small and
+// odd shapes; the register-blocked kernels in kernels_fast.cuh take over the large
+// power-of-two shapes.
+//
+// Tile geometry (PassGeom): a tile is 2^lr rows of 2^lw consecutive coordinates, the rows
+// 2^lo coordinates apart.  With lr = 0 and lw = lo = lt it is a contiguous run (a "row
+// pass" over index bits [0, lt)); otherwise the pass transforms the row bits
+// [lo, lo + lr) of the global index (a "column pass").
+#pragma once
+#include "eden_device.cuh"
+
+namespace eden {
+
+struct PassGeom {
+    int lt;   // log2 of the tile size
+    int lw;   // log2 of the contiguous run
+    int lo;   // log2 of the distance between rows
+    int lr;   // log2 of the number of rows
+};
+
+constexpr int kGenericThreads = 256;
+constexpr int kGenericTileLog = 13;                      // largest generic tile: 8192 floats
+constexpr int kGenericPerThread = (1 << kGenericTileLog) / kGenericThreads;
+
+__device__ __forceinline__ uint64_t tile_coord(const PassGeom& g, uint64_t tile, int e)
+{
+    const int chunk_bits = g.lo - g.lw;
+    const uint64_t outer = tile >> chunk_bits;
+    const uint64_t chunk = tile & ((1ull << chunk_bits) - 1);
+    const uint64_t r = (uint64_t)(e >> g.lw);
+    const uint64_t c = (uint64_t)(e & ((1 << g.lw) - 1));
+    return (outer << (g.lo + g.lr)) + (r << g.lo) + (chunk << g.lw) + c;
+}
+
+// Walsh-Hadamard butterflies over index bits [b0, b1) of a shared-memory tile of 2^lt
+// floats: pair (a, b) -> (a + b, a - b), up to three bits per barrier.
+__device__ __forceinline__ void tile_fwht(float* s, int lt, int b0, int b1)
+{
+    for (int sh = b0; sh < b1; sh += 3) {
+        const int nb = min(3, b1 - sh);
+        const int groups = (1 << lt) >> nb;
+        for (int gi = threadIdx.x; gi < groups; gi += blockDim.x) {
+            const int lo = gi & ((1 << sh) - 1);
+            const int e0 = ((gi >> sh) << (sh + nb)) | lo;
+            float v[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k < (1 << nb)) v[k] = s[e0 + (k << sh)];
+#pragma unroll
+            for (int b = 0; b < 3; ++b) {
+                if (b < nb) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (!(k & (1 << b)) && (k | (1 << b)) < (1 << nb)) {
+                            const float a = v[k], c = v[k | (1 << b)];
+                            v[k] = a + c;
+                            v[k | (1 << b)] = a - c;
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (k < (1 << nb)) s[e0 + (k << sh)] = v[k];
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// Quantiser tables in constant memory: for each width W the 2^(W-1) - 1 positive
+// interval boundaries and the 2^(W-1) positive values (Section 3).  Widths 1..8 are
+// laid out one after the other: width W starts at offset 2^(W-1) - 1 in both arrays
+// (the boundary array of width W has one unused slot at its end).
+// ---------------------------------------------------------------------------------
+__constant__ float c_pos_boundary[256];
+__constant__ float c_pos_value[256];
+
+__device__ __forceinline__ int table_offset(int W) { return (1 << (W - 1)) - 1; }
+
+// Interval rule of Section 2.2.1 on one normalised coordinate: magnitude index m =
+// number of positive boundaries strictly below |z| (an endpoint belongs to the interval
+// nearer zero), by a branch-free binary search over the sorted boundaries in `tb`.
+__device__ __forceinline__ int magnitude_index(float az, const float* tb, int half)
+{
+    int m = 0;
+    for (int step = half >> 1; step >= 1; step >>= 1)
+        m += (az > tb[m + step - 1]) ? step : 0;
+    return m;
+}
+
+// =================================================================================
+// Sender
+// =================================================================================
+
+// First pass of a multi-pass encode (a column pass over the top bits): reads the input
+// (zero beyond `valid`), flips signs (Diag(s), Section 5), accumulates ||y||^2 and writes
+// the partially transformed tile to the work buffer.
+__global__ void __launch_bounds__(kGenericThreads)
+k_enc_first(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, PassGeom g)
+{
+    extern __shared__ float s[];
+    __shared__ double red[32];
+    const ClientDesc cd = descs[blockIdx.y];
+    const int T = 1 << g.lt;
+    float local = 0.f;
+    for (int e = threadIdx.x; e < T; e += blockDim.x) {
+        const uint64_t i = tile_coord(g, blockIdx.x, e);
+        float v = i < cd.valid ? cd.src[i] : 0.f;
+        local = fmaf(v, v, local);
+        const uint32_t sw = sign_word(cd.seed, i >> 5);
+        if ((sw >> (i & 31)) & 1u) v = -v;
+        s[e] = v;
+    }
+    __syncthreads();
+    tile_fwht(s, g.lt, g.lw, g.lw + g.lr);
+    for (int e = threadIdx.x; e < T; e += blockDim.x)
+        cd.work[tile_coord(g, blockIdx.x, e)] = s[e];
+    const double tot = block_sum((double)local, red);
+    if (threadIdx.x == 0) atomicAdd(&states[blockIdx.y].norm2, tot);
+}
+
+// Middle pass, in place on the work buffer (used by sender and receiver).
+__global__ void __launch_bounds__(kGenericThreads)
+k_mid(const ClientDesc* __restrict__ descs, PassGeom g)
+{
+    extern __shared__ float s[];
+    const ClientDesc cd = descs[blockIdx.y];
+    const int T = 1 << g.lt;
+    for (int e = threadIdx.x; e < T; e += blockDim.x) s[e] = cd.work[tile_coord(g, blockIdx.x, e)];
+    __syncthreads();
+    tile_fwht(s, g.lt, g.lw, g.lw + g.lr);
+    for (int e = threadIdx.x; e < T; e += blockDim.x) cd.work[tile_coord(g, blockIdx.x, e)] = s[e];
+}
+
+// Last pass of the encode (a row pass over the low bits): finishes the transform,
+// normalises (z = h / ||y||, i.e. eta_x R(x) of Section 2.2.1), finds each coordinate's
+// interval, accumulates sum h_i Q(z_i) for the scale (Section 2.3) and writes the packed
+// codes, one ballot per bit-plane.  SINGLE: the whole vector is one tile, so this kernel
+// also loads the input, flips the signs and computes the norm.
+template <bool SINGLE>
+__global__ void __launch_bounds__(kGenericThreads)
+k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, PassGeom g)
+{
+    extern __shared__ float s[];
+    __shared__ double red[32];
+    __shared__ double s_norm2;
+    __shared__ float s_tb[128], s_tv[128];
+    const ClientDesc cd = descs[blockIdx.y];
+    const int T = 1 << g.lt;
+    const int W = (int)cd.W, half = 1 << (W - 1);
+    for (int j = threadIdx.x; j < half; j += blockDim.x) {
+        s_tb[j] = c_pos_boundary[table_offset(W) + j];
+        s_tv[j] = c_pos_value[table_offset(W) + j];
+    }
+    const uint64_t base = (uint64_t)blockIdx.x << g.lt;
+    if (SINGLE) {
+        float local = 0.f;
+        for (int e = threadIdx.x; e < T; e += blockDim.x) {
+            const uint64_t i = base + e;
+            float v = i < cd.valid ? cd.src[i] : 0.f;
+            local = fmaf(v, v, local);
+            const uint32_t sw = sign_word(cd.seed, i >> 5);
+            if ((sw >> (i & 31)) & 1u) v = -v;
+            s[e] = v;
+        }
+        const double tot = block_sum((double)local, red);
+        if (threadIdx.x == 0) { s_norm2 = tot; states[blockIdx.y].norm2 = tot; }
+    } else {
+        for (int e = threadIdx.x; e < T; e += blockDim.x) s[e] = cd.work[base + e];
+        if (threadIdx.x == 0) s_norm2 = states[blockIdx.y].norm2;
+    }
+    __syncthreads();
+    tile_fwht(s, g.lt, 0, g.lt);
+    const double n2 = s_norm2;
+    const bool live = n2 > 0.0 && n2 < INFINITY;
+    const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
+    const int lane = threadIdx.x & 31;
+    float dot = 0.f;
+    const int Tr = (T + 31) & ~31;                     // whole warps take part in the ballots
+    for (int e = threadIdx.x; e < Tr; e += blockDim.x) {
+        const float h = e < T ? s[e] : 0.f;
+        const float z = h * inv_norm;
+        const int m = magnitude_index(fabsf(z), s_tb, half);
+        const bool neg = z < 0.f;
+        uint32_t code = neg ? (uint32_t)(half - 1 - m) : (uint32_t)(half + m);
+        const float q = neg ? -s_tv[m] : s_tv[m];
+        if (e < T) dot = fmaf(h, q, dot); else code = 0u;
+        if (!live) code = 0u;
+        uint32_t mine = 0u;
+        for (int j = 0; j < W; ++j) {
+            const uint32_t word = __ballot_sync(0xffffffffu, (code >> j) & 1u);
+            if (lane == j) mine = word;
+        }
+        if (lane < W) cd.codes[((base + e) >> 5) * W + lane] = mine;
+    }
+    const double tot = block_sum((double)dot, red);
+    if (threadIdx.x == 0) {
+        if (SINGLE) states[blockIdx.y].dot = tot;
+        else atomicAdd(&states[blockIdx.y].dot, tot);
+    }
+}
+
+// S_c = ||y||^2 / <R(y), Q> = ||y||^2 sqrt(D) / sum h_i Q(z_i), times d/k below one bit.
+__global__ void k_enc_scale(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states,
+                            float* __restrict__ scales, uint32_t n,
+                            uint32_t* __restrict__ status)
+{
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= n) return;
+    const ClientDesc cd = descs[c];
+    ClientState st = states[c];
+    uint32_t flags = 0;
+    double S = 0.0;
+    if (!(st.norm2 < INFINITY)) flags |= 0x2u;             // inf or nan
+    else if (st.norm2 == 0.0) flags |= 0x1u;
+    else S = cd.extra_scale * st.norm2 * sqrt((double)(1ull << cd.L)) / st.dot;
+    scales[cd.index] = (float)S;
+    states[c].flags = flags;
+    if (flags) atomicOr(status, flags);
+}
+
+// =================================================================================
+// Receiver
+// =================================================================================
+
+// Per client: received fraction p (Section 4.2) and the factor S / (p sqrt D) that the
+// last pass applies (times 1/n for the mean).  One block per client.
+__global__ void __launch_bounds__(256)
+k_dec_prep(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states,
+           const float* __restrict__ scales, uint32_t* __restrict__ status)
+{
+    __shared__ double red[32];
+    const ClientDesc cd = descs[blockIdx.x];
+    const uint64_t D = 1ull << cd.L;
+    const uint64_t packets = (D + 1023) >> 10;
+    double cnt = 0.0;
+    if (cd.recv) {
+        const uint64_t words = (packets + 31) >> 5;
+        for (uint64_t w = threadIdx.x; w < words; w += blockDim.x) {
+            uint32_t v = cd.recv[w];
+            const uint64_t left = packets - (w << 5);
+            if (left < 32) v &= (1u << left) - 1u;
+            cnt += (double)__popc(v);
+        }
+    } else if (threadIdx.x == 0) {
+        cnt = (double)packets;
+    }
+    const double tot = block_sum(cnt, red);
+    if (threadIdx.x == 0) {
+        const double coords = D >= 1024 ? tot * 1024.0 : tot * (double)D;
+        const double p = coords / (double)D;
+        uint32_t flags = 0;
+        float f = 0.f;
+        if (coords == 0.0) flags = 0x4u;
+        else f = (float)((double)scales[cd.index] / (p * sqrt((double)D)) * cd.mean_scale);
+        states[blockIdx.x].received = p;
+        states[blockIdx.x].factor = f;
+        states[blockIdx.x].flags = flags;
+        if (flags) atomicOr(status, flags);
+    }
+}
+
+// Value of coordinate i of the received message: centroid of its code, 0 if its packet
+// was lost (Section 4.2).  `tv` holds the 2^(W-1) positive values.
+__device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i, const float* tv)
+{
+    if (cd.recv) {
+        const uint64_t pkt = i >> 10;
+        if (!((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u)) return 0.f;
+    }
+    const int W = (int)cd.W, half = 1 << (W - 1);
+    const uint32_t* wp = cd.codes + (i >> 5) * W;
+    uint32_t code = 0;
+    for (int j = 0; j < W; ++j) code |= ((wp[j] >> (i & 31)) & 1u) << j;
+    return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
+}
+
+enum OutMode { OUT_WRITE = 0, OUT_ACC = 1, OUT_YHAT = 2 };
+
+// First pass of the decode (a row pass over the low bits): unpack, centroid lookup,
+// lost packets to zero, low stages; writes the work buffer.
+__global__ void __launch_bounds__(kGenericThreads)
+k_dec_first(const ClientDesc* __restrict__ descs, PassGeom g)
+{
+    extern __shared__ float s[];
+    __shared__ float s_tv[128];
+    const ClientDesc cd = descs[blockIdx.y];
+    const int T = 1 << g.lt;
+    const int half = 1 << (cd.W - 1);
+    for (int j = threadIdx.x; j < half; j += blockDim.x) s_tv[j] = c_pos_value[table_offset(cd.W) + j];
+    __syncthreads();
+    const uint64_t base = (uint64_t)blockIdx.x << g.lt;
+    for (int e = threadIdx.x; e < T; e += blockDim.x) s[e] = received_value(cd, base + e, s_tv);
+    __syncthreads();
+    tile_fwht(s, g.lt, 0, g.lt);
+    for (int e = threadIdx.x; e < T; e += blockDim.x) cd.work[base + e] = s[e];
+}
+
+// Last pass of the decode: for each client of the group finish the inverse transform of
+// this tile, apply the client's signs and factor (x_hat = (S/p) Diag(s) H q / sqrt D,
+// Sections 2.2.2 and 4.2) and add it to a running sum kept in registers; the tile of the
+// sum is written once.  FROM_CODES: the whole vector is one tile and the kernel starts
+// from the packed codes.  OUT_YHAT stores one client's estimate of the compacted vector
+// (b < 1) for the scatter kernel.
+template <bool FROM_CODES>
+__global__ void __launch_bounds__(kGenericThreads)
+k_dec_last(const ClientDesc* __restrict__ descs, const ClientState* __restrict__ states,
+           uint32_t n_group, PassGeom g, float* __restrict__ out, uint64_t d, int mode)
+{
+    extern __shared__ float s[];
+    __shared__ float s_tv[128];
+    const int T = 1 << g.lt;
+    float acc[kGenericPerThread];
+#pragma unroll
+    for (int k = 0; k < kGenericPerThread; ++k) acc[k] = 0.f;
+    for (uint32_t c = 0; c < n_group; ++c) {
+        const ClientDesc cd = descs[c];
+        const float f = states[c].factor;
+        if (FROM_CODES) {
+            const int half = 1 << (cd.W - 1);
+            __syncthreads();
+            for (int j = threadIdx.x; j < half; j += blockDim.x)
+                s_tv[j] = c_pos_value[table_offset(cd.W) + j];
+            __syncthreads();
+            for (int e = threadIdx.x; e < T; e += blockDim.x)
+                s[e] = received_value(cd, tile_coord(g, blockIdx.x, e), s_tv);
+        } else {
+            for (int e = threadIdx.x; e < T; e += blockDim.x)
+                s[e] = cd.work[tile_coord(g, blockIdx.x, e)];
+        }
+        __syncthreads();
+        if (FROM_CODES) tile_fwht(s, g.lt, 0, g.lt);
+        else tile_fwht(s, g.lt, g.lw, g.lw + g.lr);
+#pragma unroll
+        for (int k = 0; k < kGenericPerThread; ++k) {
+            const int e = threadIdx.x + k * kGenericThreads;
+            if (e < T) {
+                const uint64_t i = tile_coord(g, blockIdx.x, e);
+                const uint32_t sw = sign_word(cd.seed, i >> 5);
+                const float v = s[e] * f;
+                acc[k] += ((sw >> (i & 31)) & 1u) ? -v : v;
+            }
+        }
+        __syncthreads();
+    }
+    const uint64_t limit = mode == OUT_YHAT ? (1ull << descs[0].L) : d;
+    float* dst = mode == OUT_YHAT ? descs[0].work : out;
+#pragma unroll
+    for (int k = 0; k < kGenericPerThread; ++k) {
+        const int e = threadIdx.x + k * kGenericThreads;
+        if (e < T) {
+            const uint64_t i = tile_coord(g, blockIdx.x, e);
+            if (i < limit) {
+                if (mode == OUT_ACC) dst[i] += acc[k];
+                else dst[i] = acc[k];
+            }
+        }
+    }
+}
+
+}  // namespace eden

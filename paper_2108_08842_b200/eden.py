@@ -1,0 +1,263 @@
+"""Thin ctypes binding over ``libeden.so`` (declared in ``include/eden.h``).
+
+Argument marshalling only: every step of EDEN's sender and receiver runs in the CUDA
+kernels of the library.  PyTorch supplies device memory and the stream.  Importing this
+module fails loudly if the library has not been built (``python -m
+paper_2108_08842_b200.build``); there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libeden.so")
+
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        "libeden.so is missing: build it with `python -m paper_2108_08842_b200.build` "
+        "(needs nvcc); this package has no CPU fallback")
+
+_lib = ctypes.CDLL(_LIB_PATH)
+
+_u32, _u64, _f64, _vp, _int = ctypes.c_uint32, ctypes.c_uint64, ctypes.c_double, ctypes.c_void_p, ctypes.c_int
+
+
+class ClientStat(ctypes.Structure):
+    _fields_ = [("norm2", _f64), ("dot", _f64), ("received", _f64), ("flags", _u32), ("reserved", _u32)]
+
+
+def _sig(name, restype, argtypes):
+    fn = getattr(_lib, name)
+    fn.restype = restype
+    fn.argtypes = argtypes
+    return fn
+
+
+_sig("eden_kept_count", _u64, [_u64, _f64])
+_sig("eden_rot_dim", _u64, [_u64, _f64])
+_sig("eden_code_width", _u32, [_f64])
+_sig("eden_code_bytes", _u64, [_u64, _f64])
+_sig("eden_num_packets", _u64, [_u64, _f64])
+_sig("eden_recv_mask_words", _u64, [_u64, _f64])
+_sig("eden_workspace_bytes", _u64, [_u64, _u32])
+_sig("eden_host_workspace_bytes", _u64, [_u64, _u32])
+_sig("eden_table", _int, [_u32, _vp, _vp])
+_sig("eden_create", _int, [ctypes.POINTER(_vp), _int, _vp, _vp, _u64])
+_sig("eden_destroy", _int, [_vp])
+_sig("eden_encode", _int, [_vp, _vp, _u64, _u64, _u32, _vp, _vp, _vp, _vp])
+_sig("eden_decode_accumulate", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp, _vp])
+_sig("eden_mean", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp])
+_sig("eden_sparsification_mask", _int, [_vp, _u64, _u64, _f64, _vp])
+_sig("eden_encode_host", _int, [_vp, _vp, _u64, _u64, _u32, _vp, _vp, _vp, _vp])
+_sig("eden_mean_host", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp])
+_sig("eden_status", _int, [_vp, ctypes.POINTER(_u32)])
+_sig("eden_client_stats", _int, [_vp, _u32, _vp])
+_sig("eden_launch_count", _u64, [_vp])
+_sig("eden_strerror", ctypes.c_char_p, [_int])
+
+STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA = 1, 2, 4
+PACKET_COORDS = 1024
+
+
+class EdenError(RuntimeError):
+    def __init__(self, code: int):
+        self.code = code
+        super().__init__("eden: %s (%d)" % (_lib.eden_strerror(code).decode(), code))
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise EdenError(rc)
+
+
+# ---------------------------------------------------------------------------- size rules
+def kept_count(d: int, bits: float) -> int:
+    return int(_lib.eden_kept_count(d, bits))
+
+
+def rot_dim(d: int, bits: float) -> int:
+    return int(_lib.eden_rot_dim(d, bits))
+
+
+def code_width(bits: float) -> int:
+    return int(_lib.eden_code_width(bits))
+
+
+def code_bytes(d: int, bits: float) -> int:
+    return int(_lib.eden_code_bytes(d, bits))
+
+
+def num_packets(d: int, bits: float) -> int:
+    return int(_lib.eden_num_packets(d, bits))
+
+
+def recv_mask_words(d: int, bits: float) -> int:
+    return int(_lib.eden_recv_mask_words(d, bits))
+
+
+def workspace_bytes(d_max: int, n_batch: int) -> int:
+    return int(_lib.eden_workspace_bytes(d_max, n_batch))
+
+
+def host_workspace_bytes(d: int, n: int) -> int:
+    return int(_lib.eden_host_workspace_bytes(d, n))
+
+
+def table(W: int):
+    """(values float32[2^W], boundaries float32[2^W - 1]) the kernels quantise with."""
+    c = np.zeros(1 << W, dtype=np.float32)
+    b = np.zeros(max((1 << W) - 1, 1), dtype=np.float32)
+    _check(_lib.eden_table(W, c.ctypes.data, b.ctypes.data))
+    return c, b[: (1 << W) - 1]
+
+
+def _f64s(v) -> np.ndarray:
+    return np.ascontiguousarray(v, dtype=np.float64)
+
+
+def _u64s(v) -> np.ndarray:
+    return np.ascontiguousarray(v, dtype=np.uint64)
+
+
+def _ptr_table(tensors: Sequence[Optional[torch.Tensor]]):
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = None if t is None else t.data_ptr()
+    return arr
+
+
+class Context:
+    """One device, one stream, one caller-owned workspace (a torch uint8 tensor)."""
+
+    def __init__(self, device: int = 0, workspace_bytes_: Optional[int] = None,
+                 d_max: int = 1 << 20, n_batch: int = 1, stream: Optional[torch.cuda.Stream] = None,
+                 host_staging: bool = False):
+        if not torch.cuda.is_available():
+            raise RuntimeError("eden: no CUDA device; this library has no CPU path")
+        self.device = device
+        if workspace_bytes_ is None:
+            workspace_bytes_ = (host_workspace_bytes if host_staging else workspace_bytes)(d_max, n_batch)
+        with torch.cuda.device(device):
+            self.stream = stream if stream is not None else torch.cuda.current_stream()
+            self.workspace = torch.empty(int(workspace_bytes_) + 256, dtype=torch.uint8, device="cuda:%d" % device)
+        base = self.workspace.data_ptr()
+        aligned = (base + 255) // 256 * 256
+        self._h = _vp()
+        self.workspace_bytes = int(workspace_bytes_)
+        _check(_lib.eden_create(ctypes.byref(self._h), device, self.stream.cuda_stream,
+                                aligned, self.workspace_bytes))
+
+    def close(self):
+        if self._h:
+            _lib.eden_destroy(self._h)
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ sender
+    def alloc_codes(self, d: int, bits) -> List[torch.Tensor]:
+        return [torch.empty(code_bytes(d, float(b)), dtype=torch.uint8, device="cuda:%d" % self.device)
+                for b in bits]
+
+    def encode(self, x: torch.Tensor, bits, seeds, codes: Optional[List[torch.Tensor]] = None,
+               scales: Optional[torch.Tensor] = None):
+        """eden_encode: x is a CUDA fp32 [n, d] tensor (row stride >= d).  Returns (codes, scales)."""
+        assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1
+        n, d = x.shape
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        assert len(bits) == n and len(seeds) == n
+        if codes is None:
+            codes = self.alloc_codes(d, bits)
+        if scales is None:
+            scales = torch.empty(n, dtype=torch.float32, device=x.device)
+        tab = _ptr_table(codes)
+        _check(_lib.eden_encode(self._h, x.data_ptr(), x.stride(0), d, n, bits.ctypes.data,
+                                seeds.ctypes.data, tab, scales.data_ptr()))
+        return codes, scales
+
+    # ------------------------------------------------------------------ receiver
+    def _decode(self, fn, codes, scales, bits, seeds, recv_masks, d, out, extra=()):
+        n = len(codes)
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        assert len(bits) == n and len(seeds) == n and scales.is_cuda and scales.dtype == torch.float32
+        tab = _ptr_table(codes)
+        mtab = None if recv_masks is None else _ptr_table(recv_masks)
+        _check(fn(self._h, tab, scales.data_ptr(), bits.ctypes.data, seeds.ctypes.data, mtab,
+                  d, n, out.data_ptr(), *extra))
+        return out
+
+    def mean(self, codes, scales, bits, seeds, d: int, recv_masks=None, out: Optional[torch.Tensor] = None):
+        """eden_mean: (1/n) sum_c x_hat_c as a CUDA fp32 [d] tensor."""
+        if out is None:
+            out = torch.empty(d, dtype=torch.float32, device=scales.device)
+        return self._decode(_lib.eden_mean, codes, scales, bits, seeds, recv_masks, d, out)
+
+    def decode_accumulate(self, codes, scales, bits, seeds, d: int, acc: torch.Tensor, recv_masks=None):
+        """eden_decode_accumulate: acc += sum_c x_hat_c; returns the number of clients counted."""
+        used = _u32(0)
+        self._decode(_lib.eden_decode_accumulate, codes, scales, bits, seeds, recv_masks, d, acc,
+                     extra=(ctypes.byref(used),))
+        return int(used.value)
+
+    def sparsification_mask(self, seed: int, d: int, bits: float) -> torch.Tensor:
+        """Bitmap (int32 words, bit i of word i/32) of the coordinates kept for b < 1."""
+        out = torch.zeros((d + 31) // 32, dtype=torch.int32, device="cuda:%d" % self.device)
+        _check(_lib.eden_sparsification_mask(self._h, int(seed), d, float(bits), out.data_ptr()))
+        return out
+
+    # ------------------------------------------------------------------ host-buffer variants
+    def encode_host(self, x: np.ndarray, bits, seeds, codes: List[np.ndarray], scales: np.ndarray):
+        """eden_encode_host: numpy/pinned host buffers in, host buffers out (synchronous)."""
+        n, d = x.shape
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        tab = (ctypes.c_void_p * n)(*[c.ctypes.data for c in codes])
+        _check(_lib.eden_encode_host(self._h, x.ctypes.data, x.strides[0] // 4, d, n, bits.ctypes.data,
+                                     seeds.ctypes.data, tab, scales.ctypes.data))
+
+    def mean_host(self, codes: List[np.ndarray], scales: np.ndarray, bits, seeds, d: int,
+                  recv_masks: Optional[List[Optional[np.ndarray]]], out: np.ndarray):
+        n = len(codes)
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        tab = (ctypes.c_void_p * n)(*[c.ctypes.data for c in codes])
+        mtab = None
+        if recv_masks is not None:
+            mtab = (ctypes.c_void_p * n)(*[None if m is None else m.ctypes.data for m in recv_masks])
+        _check(_lib.eden_mean_host(self._h, tab, scales.ctypes.data, bits.ctypes.data, seeds.ctypes.data,
+                                   mtab, d, n, out.ctypes.data))
+
+    # ------------------------------------------------------------------ status
+    def status(self) -> int:
+        w = _u32(0)
+        _check(_lib.eden_status(self._h, ctypes.byref(w)))
+        return int(w.value)
+
+    def client_stats(self, n: int):
+        arr = (ClientStat * n)()
+        _check(_lib.eden_client_stats(self._h, n, arr))
+        return [dict(norm2=a.norm2, dot=a.dot, received=a.received, flags=a.flags) for a in arr]
+
+    @property
+    def launch_count(self) -> int:
+        return int(_lib.eden_launch_count(self._h))
+
+
+# module-level calls with the names of the C entry points ---------------------------------
+def eden_encode(ctx: Context, x, bits, seeds, codes=None, scales=None):
+    return ctx.encode(x, bits, seeds, codes, scales)
+
+
+def eden_mean(ctx: Context, codes, scales, bits, seeds, d, recv_masks=None, out=None):
+    return ctx.mean(codes, scales, bits, seeds, d, recv_masks, out)
+
+
+def eden_decode_accumulate(ctx: Context, codes, scales, bits, seeds, d, acc, recv_masks=None):
+    return ctx.decode_accumulate(codes, scales, bits, seeds, d, acc, recv_masks)

@@ -1,0 +1,47 @@
+"""Helpers that compare the CUDA library with the CPU oracle on one workload."""
+from __future__ import annotations
+
+import numpy as np
+
+import oracle as O
+
+
+def unpack_codes(words: np.ndarray, D: int, W: int) -> np.ndarray:
+    """Per-coordinate codes from the packed wire layout (word g*W + j = bit-plane j of group g)."""
+    groups = (D + 31) // 32
+    w = words[: groups * W].reshape(groups, W)
+    shifts = np.arange(32, dtype=np.uint32)
+    codes = np.zeros((groups, 32), dtype=np.uint32)
+    for j in range(W):
+        codes |= ((w[:, j:j + 1] >> shifts) & 1) << np.uint32(j)
+    return codes.reshape(-1)[:D]
+
+
+def near_boundary(z: np.ndarray, W: int) -> np.ndarray:
+    """|z - t| <= 1e-6 * max(1, |t|) for some interval boundary t of the 2^W-value table."""
+    _, b = O.table(W)
+    out = np.zeros(z.shape, dtype=bool)
+    for t in b:
+        out |= np.abs(z - t) <= 1e-6 * max(1.0, abs(t))
+    return out
+
+
+def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, bits: float, seed: int):
+    """Returns (mismatching coordinates, all inside the boundary window?, scale rel. error, oracle result)."""
+    enc = O.encode(x, bits, seed, want_z=True)
+    d = x.shape[0]
+    D, W = O.rot_dim(d, bits), O.code_width(bits)
+    nw = len(enc["codes"])
+    diff = np.nonzero(gpu_words[:nw] != enc["codes"])[0]
+    mism = 0
+    ok = True
+    if diff.size:
+        g = unpack_codes(gpu_words, D, W)
+        o = unpack_codes(enc["codes"], D, W)
+        bad = np.nonzero(g != o)[0]
+        mism = int(bad.size)
+        ok = bool(np.all(near_boundary(enc["z"][bad], W)))
+        # a mismatch may only move the code to the neighbouring interval
+        ok = ok and bool(np.all(np.abs(g[bad].astype(np.int64) - o[bad].astype(np.int64)) == 1))
+    rel = abs(gpu_scale - enc["scale"]) / abs(enc["scale"]) if enc["scale"] != 0 else abs(gpu_scale)
+    return mism, ok, rel, enc

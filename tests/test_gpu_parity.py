@@ -1,0 +1,281 @@
+"""Parity of the CUDA library against the CPU oracle, through the C ABI (via the thin
+binding), on seeded synthetic inputs.
+
+Tolerances (the ones the task fixes):
+  * packed codes and sparsification masks bit-exact, except coordinates whose normalised
+    value lies within 1e-6 * max(1, |t|) of an interval boundary t; those are counted and
+    may only land in the neighbouring interval;
+  * scales within 1e-5 relative;
+  * decoded mean: max abs error <= 1e-4 * ||mean||_inf.
+The receiver is always fed the ORACLE's codes and scales (rounded to fp32, the wire
+format), so a legitimately different boundary decision on the sender cannot leak into
+the receiver comparison.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2108_08842_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+SCALE_TOL = 1e-5
+MEAN_TOL = 1e-4
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2108_08842_b200 import eden
+    return eden
+
+
+def _ctx(E, d, n):
+    return E.Context(0, d_max=d, n_batch=n)
+
+
+def run_workload(E, work, threads=8, check_clients=None):
+    """Encode parity for the chosen clients, decode+mean parity for all of them."""
+    n, d = work.n, work.d
+    xs = work.vectors()
+    ctx = _ctx(E, d, n)
+    x_gpu = torch.from_numpy(xs).cuda()
+    codes, scales = ctx.encode(x_gpu, work.bits, work.seeds)
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    scales_h = scales.cpu().numpy()
+    check_clients = range(n) if check_clients is None else check_clients
+
+    total_mism = 0
+    encs = {}
+    for c in check_clients:
+        words = codes[c].cpu().numpy().view(np.uint32)
+        mism, ok, rel, enc = parity.check_encode_client(words, float(scales_h[c]), xs[c],
+                                                       float(work.bits[c]), int(work.seeds[c]))
+        assert ok, "client %d: %d code mismatches outside the boundary window" % (c, mism)
+        assert rel <= SCALE_TOL, "client %d: scale off by %g" % (c, rel)
+        total_mism += mism
+        encs[c] = enc
+
+    # receiver: oracle's message in, both sides decode it
+    clients = list(check_clients)
+    o_codes = [encs[c]["codes"] for c in clients]
+    o_scales = np.array([np.float32(encs[c]["scale"]) for c in clients], dtype=np.float32)
+    bits = [float(work.bits[c]) for c in clients]
+    seeds = [int(work.seeds[c]) for c in clients]
+    masks_np = masks_t = None
+    if work.drop_prob > 0:
+        masks_np = [work.recv_mask(c, O.num_packets(O.rot_dim(d, float(work.bits[c])))) for c in clients]
+        masks_t = [torch.from_numpy(m.view(np.int32)).cuda() for m in masks_np]
+    g_codes = []
+    for c, w in zip(clients, o_codes):
+        buf = np.zeros(E.code_bytes(d, float(work.bits[c])), dtype=np.uint8)
+        buf[: w.nbytes] = w.view(np.uint8)
+        g_codes.append(torch.from_numpy(buf).cuda())
+    mean_gpu = ctx.mean(g_codes, torch.from_numpy(o_scales).cuda(), bits, seeds, d, masks_t).cpu().numpy()
+    assert ctx.status() == 0
+    mean_ref, used = O.mean(o_codes, [float(s) for s in o_scales], bits, seeds, d, masks_np, threads=threads)
+    assert used == len(clients)
+    err = np.max(np.abs(mean_gpu.astype(np.float64) - mean_ref))
+    assert err <= MEAN_TOL * np.max(np.abs(mean_ref)), (err, np.max(np.abs(mean_ref)))
+
+    # accumulate entry point: acc += sum of estimates
+    acc = torch.full((d,), 0.5, dtype=torch.float32, device="cuda")
+    used = ctx.decode_accumulate(g_codes, torch.from_numpy(o_scales).cuda(), bits, seeds, d, acc, masks_t)
+    assert used == len(clients)
+    err = np.max(np.abs(acc.cpu().numpy().astype(np.float64) - 0.5 - mean_ref * len(clients)))
+    assert err <= MEAN_TOL * np.max(np.abs(mean_ref)) * len(clients) + 1e-6
+
+    # if the sender agreed bit for bit, the GPU-only round trip must give the same mean
+    if total_mism == 0 and len(clients) == n:
+        mean_rt = ctx.mean(codes, scales, work.bits, work.seeds, d, masks_t).cpu().numpy()
+        err = np.max(np.abs(mean_rt.astype(np.float64) - mean_ref))
+        assert err <= 2 * MEAN_TOL * np.max(np.abs(mean_ref))
+    ctx.close()
+    return total_mism, xs, mean_ref
+
+
+# ----------------------------------------------------------------------------- the five configurations
+def test_cfg1_small_normal_one_bit(E):
+    mism, xs, mean = run_workload(E, synth.make("cfg1"))
+    assert mism <= 2
+
+
+def test_cfg2_layered_laplace_two_bits(E):
+    mism, xs, mean = run_workload(E, synth.make("cfg2"))
+    assert mism <= 20
+    # NMSE of the estimate against the true mean: vNMSE/n with vNMSE(b=2) = 0.1331 (Lemma 2.2)
+    true = xs.astype(np.float64).mean(axis=0)
+    nmse = np.sum((mean - true) ** 2) / (np.sum(xs.astype(np.float64) ** 2) / xs.shape[0])
+    assert abs(nmse - 0.1331 / 10) < 0.25 * 0.1331 / 10
+
+
+def test_cfg3_heterogeneous_budgets_reduced(E):
+    # same law and budget mix, d = 2^17 so that the oracle checks all 32 clients
+    work = synth.make("cfg3", d=1 << 17)
+    assert set(np.unique(work.bits)) <= {0.1, 0.5, 1.0, 2.0, 4.0} and len(np.unique(work.bits)) >= 4
+    mism, _, _ = run_workload(E, work)
+    assert mism <= 20
+
+
+def test_cfg4_packet_loss_reduced(E):
+    work = synth.make("cfg4", d=1 << 18, n=16)
+    mism, _, _ = run_workload(E, work)
+    assert mism <= 20
+
+
+def test_cfg5_padding_four_bits_loss_reduced(E):
+    work = synth.make("cfg5", d=1_000_003, n=4)      # ragged: pads to 2^20
+    mism, _, _ = run_workload(E, work)
+    assert mism <= 40
+
+
+# ----------------------------------------------------------------------------- shapes and edge cases
+@pytest.mark.parametrize("d", [1, 2, 5, 31, 32, 33, 100, 1023, 1024, 1025, 4097, 8192, 8193,
+                               16384, 20000, 65536, 100000, (1 << 21) + 7])
+@pytest.mark.parametrize("bits", [1.0, 3.0])
+def test_shapes_and_ragged_tails(E, d, bits):
+    rng = np.random.default_rng(d)
+    n = 3
+    xs = (rng.standard_normal((n, d)) * rng.uniform(0.01, 100)).astype(np.float32)
+    seeds = synth.client_seeds(d, n)
+    work = synth.Workload("adhoc", n, d, np.full(n, bits), seeds, 0.0, lambda c: xs[c], d)
+    run_workload(E, work)
+
+
+@pytest.mark.parametrize("W", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_every_code_width(E, W):
+    d, n = 40000, 2
+    rng = np.random.default_rng(W)
+    xs = np.exp(rng.standard_normal((n, d))).astype(np.float32)      # LogNormal(0,1), the paper's sweep law
+    work = synth.Workload("adhoc", n, d, np.full(n, float(W)), synth.client_seeds(W, n), 0.0,
+                          lambda c: xs[c], W)
+    mism, _, _ = run_workload(E, work)
+    assert mism <= 8 * W
+
+
+@pytest.mark.parametrize("bits,d", [(0.1, 1 << 16), (0.5, 3000), (0.25, 70001), (0.9, 9), (0.01, 50)])
+def test_sub_bit_budgets_and_mask(E, bits, d):
+    n = 3
+    rng = np.random.default_rng(int(bits * 1000) + d)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    seeds = synth.client_seeds(d + 1, n)
+    ctx = _ctx(E, d, n)
+    k = O.kept_count(d, bits)
+    for c in range(n):
+        got = ctx.sparsification_mask(int(seeds[c]), d, bits).cpu().numpy().view(np.uint32)
+        bits_got = ((got[:, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(-1)[:d]
+        want = O.mask(int(seeds[c]), d, k)
+        assert bits_got.sum() == k
+        assert np.array_equal(bits_got.astype(np.uint8), want)           # masks are bit-exact
+    ctx.close()
+    work = synth.Workload("adhoc", n, d, np.full(n, bits), seeds, 0.0, lambda c: xs[c], d)
+    run_workload(E, work)
+
+
+def test_mixed_budgets_in_one_call(E):
+    d, n = 50000, 7
+    rng = np.random.default_rng(5)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    bits = np.array([0.3, 1.0, 2.0, 0.1, 4.0, 8.0, 1.0])
+    work = synth.Workload("adhoc", n, d, bits, synth.client_seeds(9, n), 0.2, lambda c: xs[c], 9)
+    run_workload(E, work)
+
+
+def test_zero_vector_and_status_word(E):
+    d, n = 5000, 3
+    xs = np.random.default_rng(1).standard_normal((n, d)).astype(np.float32)
+    xs[1] = 0.0
+    ctx = _ctx(E, d, n)
+    codes, scales = ctx.encode(torch.from_numpy(xs).cuda(), [2.0] * n, [11, 12, 13])
+    assert ctx.status() == E.STATUS_ZERO_VECTOR
+    assert ctx.status() == 0                                  # reading clears it
+    assert float(scales[1]) == 0.0 and not codes[1].any()
+    stats = ctx.client_stats(n)
+    assert stats[1]["flags"] == E.STATUS_ZERO_VECTOR and stats[0]["flags"] == 0
+    ref = O.encode(xs[0], 2.0, 11)
+    assert abs(stats[0]["norm2"] - float(np.sum(xs[0].astype(np.float64) ** 2))) < 1e-6 * stats[0]["norm2"]
+    # the zero client decodes to zero: the mean is the mean of the other two estimates / 3
+    mean = ctx.mean(codes, scales, [2.0] * n, [11, 12, 13], d).cpu().numpy()
+    parts = [O.decode(O.encode(xs[c], 2.0, s)["codes"], float(np.float32(O.encode(xs[c], 2.0, s)["scale"])),
+                      2.0, s, d)[0] for c, s in ((0, 11), (2, 13))]
+    want = (parts[0] + parts[1]) / 3
+    assert np.max(np.abs(mean - want)) <= 1e-3 * np.max(np.abs(want))
+    # non-finite input is reported, not fatal
+    xs[2, 7] = np.inf
+    ctx.encode(torch.from_numpy(xs).cuda(), [2.0] * n, [11, 12, 13])
+    assert ctx.status() & E.STATUS_NONFINITE
+    ctx.close()
+
+
+def test_all_packets_lost_is_reported_not_fatal(E):
+    d, n = 4096, 2
+    xs = np.random.default_rng(2).standard_normal((n, d)).astype(np.float32)
+    ctx = _ctx(E, d, n)
+    codes, scales = ctx.encode(torch.from_numpy(xs).cuda(), [1.0, 1.0], [5, 6])
+    none = torch.zeros(1, dtype=torch.int32, device="cuda")
+    full = torch.full((1,), 0xF, dtype=torch.int32, device="cuda")
+    mean = ctx.mean(codes, scales, [1.0, 1.0], [5, 6], d, [none, full]).cpu().numpy()
+    assert ctx.status() == E.STATUS_NO_DATA
+    stats = ctx.client_stats(n)
+    assert stats[0]["received"] == 0.0 and stats[1]["received"] == 1.0
+    enc = O.encode(xs[1], 1.0, 6)
+    want = O.decode(enc["codes"], float(np.float32(enc["scale"])), 1.0, 6, d)[0] / 2   # divisor stays n
+    assert np.max(np.abs(mean - want)) <= 1e-3 * np.max(np.abs(want))
+    ctx.close()
+
+
+def test_bad_arguments(E):
+    ctx = _ctx(E, 1024, 2)
+    x = torch.zeros(2, 1024, device="cuda")
+    with pytest.raises(E.EdenError) as e:
+        ctx.encode(x, [1.5, 1.0], [1, 2])
+    assert e.value.code == -2
+    with pytest.raises(E.EdenError) as e:
+        ctx.encode(x, [0.0, 1.0], [1, 2])
+    assert e.value.code == -2
+    small = E.Context(0, workspace_bytes_=E.workspace_bytes(1024, 1))
+    big = torch.zeros(1, 1 << 20, device="cuda")
+    with pytest.raises(E.EdenError) as e:
+        small.encode(big, [1.0], [1])
+    assert e.value.code == -4
+    small.close()
+    ctx.close()
+
+
+def test_small_workspace_runs_in_several_groups(E):
+    d, n = 1 << 16, 6
+    xs = np.random.default_rng(3).standard_normal((n, d)).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.full(n, 2.0), synth.client_seeds(3, n), 0.0, lambda c: xs[c], 3)
+    import paper_2108_08842_b200.eden as eden_mod
+    orig = eden_mod.workspace_bytes
+    try:
+        eden_mod.workspace_bytes = lambda d_max, n_batch: orig(d_max, 2)   # room for two clients at a time
+        run_workload(E, work)
+    finally:
+        eden_mod.workspace_bytes = orig
+
+
+def test_host_buffer_entry_points(E):
+    work = synth.make("cfg4", d=1 << 16, n=5)
+    n, d = work.n, work.d
+    xs = work.vectors()
+    ctx = E.Context(0, d_max=d, n_batch=n, host_staging=True)
+    codes = [np.zeros(E.code_bytes(d, float(b)), dtype=np.uint8) for b in work.bits]
+    scales = np.zeros(n, dtype=np.float32)
+    ctx.encode_host(xs, work.bits, work.seeds, codes, scales)
+    x_gpu = torch.from_numpy(xs).cuda()
+    dcodes, dscales = ctx.encode(x_gpu, work.bits, work.seeds)
+    assert np.array_equal(dscales.cpu().numpy(), scales)
+    for c in range(n):
+        assert np.array_equal(dcodes[c].cpu().numpy(), codes[c])
+    masks = [work.recv_mask(c, O.num_packets(O.rot_dim(d, 1.0))) for c in range(n)]
+    out = np.zeros(d, dtype=np.float32)
+    ctx.mean_host(codes, scales, work.bits, work.seeds, d, masks, out)
+    dev = ctx.mean(dcodes, dscales, work.bits, work.seeds, d,
+                   [torch.from_numpy(m.view(np.int32)).cuda() for m in masks]).cpu().numpy()
+    assert np.array_equal(out, dev)
+    ctx.close()

@@ -1,0 +1,107 @@
+"""CPU-only checks of the CUDA library: it loads, exports every symbol the header
+declares, its host-side size rules and quantiser tables agree with the oracle, and the
+package refuses to run without a GPU instead of falling back."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle as O
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2108_08842_b200 import build
+    return ctypes.CDLL(build.build())
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "eden.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(eden_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert {"eden_encode", "eden_decode_accumulate", "eden_mean", "eden_create"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), name
+
+
+def test_size_rules_match_oracle(lib):
+    lib.eden_kept_count.restype = ctypes.c_uint64
+    lib.eden_rot_dim.restype = ctypes.c_uint64
+    lib.eden_code_bytes.restype = ctypes.c_uint64
+    lib.eden_num_packets.restype = ctypes.c_uint64
+    lib.eden_code_width.restype = ctypes.c_uint32
+    for f in (lib.eden_kept_count, lib.eden_rot_dim, lib.eden_code_bytes, lib.eden_num_packets):
+        f.argtypes = [ctypes.c_uint64, ctypes.c_double]
+    lib.eden_code_width.argtypes = [ctypes.c_double]
+    for d in (1, 2, 31, 32, 33, 1000, 1024, 1025, 10 ** 6, 2 ** 23, 10 ** 8):
+        for bits in (0.001, 0.1, 0.5, 0.999, 1.0, 2.0, 3.0, 4.0, 8.0):
+            assert lib.eden_kept_count(d, bits) == O.kept_count(d, bits)
+            D = O.rot_dim(d, bits)
+            assert lib.eden_rot_dim(d, bits) == D
+            assert lib.eden_code_width(bits) == O.code_width(bits)
+            assert lib.eden_num_packets(d, bits) == O.num_packets(D)
+            words = O.code_words(d, bits)
+            cb = lib.eden_code_bytes(d, bits)
+            assert cb % 16 == 0 and 4 * words <= cb < 4 * words + 16
+    for bad in (0.0, -1.0, 1.5, 2.5, 9.0, float("nan")):
+        assert lib.eden_code_width(bad) == 0
+
+
+def test_library_tables_match_oracle_tables(lib):
+    lib.eden_table.argtypes = [ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p]
+    for W in range(1, 9):
+        c = np.zeros(1 << W, dtype=np.float32)
+        b = np.zeros(max((1 << W) - 1, 1), dtype=np.float32)
+        assert lib.eden_table(W, c.ctypes.data, b.ctypes.data) == 0
+        oc, ob = O.table(W)
+        # two independent double-precision solvers, compared after rounding to fp32:
+        # equal up to one unit in the last place
+        assert np.all(np.abs(c - oc.astype(np.float32)) <= np.spacing(np.abs(oc).astype(np.float32)))
+        assert np.all(np.abs(b[: (1 << W) - 1] - ob.astype(np.float32))
+                      <= np.spacing(np.abs(ob).astype(np.float32)))
+    assert lib.eden_table(0, c.ctypes.data, b.ctypes.data) < 0
+    assert lib.eden_table(9, c.ctypes.data, b.ctypes.data) < 0
+
+
+def test_bad_arguments_are_rejected_without_a_gpu(lib):
+    lib.eden_create.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64]
+    h = ctypes.c_void_p()
+    assert lib.eden_create(ctypes.byref(h), 0, None, None, 1 << 20) == -1        # no workspace
+    assert lib.eden_create(ctypes.byref(h), 0, None, ctypes.c_void_p(256 + 8), 1 << 30) == -1   # misaligned
+    assert lib.eden_create(ctypes.byref(h), 0, None, ctypes.c_void_p(4096), 16) == -4  # too small
+    lib.eden_strerror.restype = ctypes.c_char_p
+    assert b"workspace" in lib.eden_strerror(-4)
+    lib.eden_encode.restype = ctypes.c_int
+    assert lib.eden_encode(None, None, 0, 0, 0, None, None, None, None) == -1
+    assert lib.eden_mean(None, None, None, None, None, None, 0, 0, None) == -1
+    assert lib.eden_status(None, None) == -1
+
+
+def test_product_package_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2108_08842_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".cpp", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower().replace("eden_oracle", "oracle") or f == "synth.py", f
+    text = open(os.path.join(pkg, "synth.py")).read()
+    assert "import oracle" not in text and "from oracle" not in text
+
+
+def test_binding_refuses_to_run_without_cuda():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    from paper_2108_08842_b200 import build
+    build.build()
+    from paper_2108_08842_b200 import eden
+    with pytest.raises(RuntimeError):
+        eden.Context(0)

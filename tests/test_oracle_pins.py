@@ -212,7 +212,7 @@ def test_encode_decode_against_dense_reference(d, bits):
     codes_ref, S_ref, xhat_ref, r, _ = _dense_reference(x.astype(np.float64), bits, seed)
     enc = O.encode(x, bits, seed, want_z=True)
     D, W = O.rot_dim(d, bits), O.code_width(bits)
-    assert len(enc["codes"]) == D * W // 32
+    assert len(enc["codes"]) == (D + 31) // 32 * W
     assert np.array_equal(_unpack(enc["codes"], D, W), codes_ref)
     assert abs(enc["scale"] - S_ref) < 1e-10 * abs(S_ref)
     xhat, nodata = O.decode(enc["codes"], enc["scale"], bits, seed, d)
