@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the EDEN hot path (encode + decode+mean) on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input: eden_encode
+of all n client vectors followed by eden_mean of the n messages.  The metric is GB/s of
+fp32 input (n*d*4 bytes per step).  One JSON line is printed by rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--impl reference]
+
+With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica of the workload (no collective on the data path; only the timing is reduced).
+--impl reference times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "encode and decode+mean GB/s (fp32 in)"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def config_of(work, extra=None):
+    bits = sorted(set(float(b) for b in work.bits))
+    cfg = {"workload": work.name, "n_clients": int(work.n), "d": int(work.d), "bits": bits,
+           "packet_drop_prob": work.drop_prob, "value_law": work.description,
+           "l2_policy": "inputs larger than L2 (no flush)"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+# ------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                 r[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(mx)) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------- inputs
+def generate_vectors(work, out: np.ndarray, threads: int):
+    def one(c):
+        out[c] = work.vector(c)
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(one, range(work.n)))
+
+
+# ------------------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(work, clients, threads):
+    """Times the oracle (as it stands) on `clients` of the workload: encode, then
+    decode + mean of those clients.  Returns (seconds, bytes of fp32 input)."""
+    import oracle as O
+    xs = [work.vector(c) for c in clients]
+    bits = [float(work.bits[c]) for c in clients]
+    seeds = [int(work.seeds[c]) for c in clients]
+    masks = None
+    if work.drop_prob > 0:
+        masks = [work.recv_mask(c, O.num_packets(O.rot_dim(work.d, bits[i]))) for i, c in enumerate(clients)]
+    O.table(1)  # build tables outside the timed region
+    for b in set(bits):
+        O.table(O.code_width(b))
+    t0 = time.perf_counter()
+    enc = O.encode_all(xs, bits, seeds, threads=threads)
+    mean, _ = O.mean([e["codes"] for e in enc], [float(np.float32(e["scale"])) for e in enc],
+                     bits, seeds, work.d, masks, threads=threads)
+    dt = time.perf_counter() - t0
+    return dt, len(clients) * work.d * 4, mean
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2108_08842_b200 import synth
+    work = synth.make(args.workload)
+    cores = host_cores()
+    # bounded sample per step: `threads` clients, each cut to its first d_s coordinates
+    threads = min(cores, work.n, 8)
+    d_s = min(work.d, 1 << 21)
+    sample = synth.make(args.workload, d=d_s, n=threads)
+    times = []
+    for step in range(args.warmup + args.steps):
+        dt, nbytes, _ = oracle_sample(sample, list(range(threads)), threads)
+        if step >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = threads * d_s * 4 / (ms * 1e-3) / 1e9
+    desc = "%d clients x first %d coordinates of %s per step, %d threads" % (threads, d_s, work.name, threads)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_of(work),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------- GPU arm
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2108_08842_b200 import eden, synth
+
+    work = synth.make(args.workload, seed=rank)
+    n, d = work.n, work.d
+    cores = host_cores()
+    dev = torch.device("cuda", local_rank)
+
+    # inputs: generated on the host (pinned, also used by the end-to-end leg), then resident in HBM
+    x_host = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+    generate_vectors(work, x_host.numpy(), min(cores, 16))
+    x_gpu = x_host.to(dev, non_blocking=True)
+    bits, seeds = work.bits, work.seeds
+    masks_np = masks_gpu = None
+    if work.drop_prob > 0:
+        masks_np = [work.recv_mask(c, eden.num_packets(d, float(bits[c]))) for c in range(n)]
+        masks_gpu = [torch.from_numpy(m.view(np.int32)).to(dev) for m in masks_np]
+    ctx = eden.Context(local_rank, d_max=d, n_batch=n, host_staging=True)
+    codes = ctx.alloc_codes(d, bits)
+    scales = torch.empty(n, dtype=torch.float32, device=dev)
+    mean = torch.empty(d, dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+
+    def step():
+        ctx.encode(x_gpu, bits, seeds, codes, scales)
+        ctx.mean(codes, scales, bits, seeds, d, masks_gpu, mean)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- timed region: K steps, CUDA events on the library's stream, clocks sampled meanwhile
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = ctx.launch_count
+    ctx.profile(True)
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    enc_ms = dec_ms = 0.0
+    barrier()
+    t_events = []
+    for _ in range(args.steps):
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        a.record()
+        ctx.encode(x_gpu, bits, seeds, codes, scales)
+        b.record()
+        ctx.mean(codes, scales, bits, seeds, d, masks_gpu, mean)
+        c.record()
+        t_events.append((a, b, c))
+    barrier()
+    kernels = ctx.profile_collect()
+    ctx.profile(False)
+    launches = ctx.launch_count - launches0
+    clocks = sampler.stop()
+    total_ms = t_events[0][0].elapsed_time(t_events[-1][2])
+    enc_ms = sum(a.elapsed_time(b) for a, b, c in t_events) / args.steps
+    dec_ms = sum(b.elapsed_time(c) for a, b, c in t_events) / args.steps
+    t = torch.tensor([total_ms, enc_ms, dec_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, enc_ms, dec_ms = (float(v) for v in t.tolist())
+    ms_per_step = total_ms / args.steps
+    in_bytes = n * d * 4
+    value = world * in_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- roofline of the dominant kernel (by event time inside the timed region)
+    peak, peak_kind = measured_hbm_peak()
+    top_name = max(kernels, key=lambda k: kernels[k]["ms"])
+    top = kernels[top_name]
+    achieved = top["bytes"] / top["launches"] / (top["ms"] / top["launches"] * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": top_name, "achieved": achieved, "peak": peak,
+                "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None,
+                "algorithmic_bytes_per_launch": top["bytes"] / top["launches"],
+                "ms_per_launch": top["ms"] / top["launches"]}
+    kernel_table = {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
+                        "share": round(v["ms"] / sum(x["ms"] for x in kernels.values()), 4),
+                        "algo_GBps": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
+                    for k, v in sorted(kernels.items(), key=lambda kv: -kv[1]["ms"])}
+
+    # ---- accuracy of the GPU estimate against the true mean (untimed)
+    true_mean = x_gpu.double().mean(dim=0)
+    nmse = float(((mean.double() - true_mean) ** 2).sum() / ((x_gpu.double() ** 2).sum() / n))
+    del true_mean
+    status = ctx.status()
+
+    # ---- end to end: same step through the host-buffer entry points (pinned memory),
+    #      host->device and device->host copies inside the timed region
+    e2e = None
+    if rank == 0 or world > 1:
+        codes_h = [torch.empty(eden.code_bytes(d, float(b)), dtype=torch.uint8, pin_memory=True).numpy()
+                   for b in bits]
+        scales_h = torch.empty(n, dtype=torch.float32, pin_memory=True).numpy()
+        mean_h = torch.empty(d, dtype=torch.float32, pin_memory=True).numpy()
+        xh = x_host.numpy()
+
+        def e2e_step():
+            ctx.encode_host(xh, bits, seeds, codes_h, scales_h)
+            ctx.mean_host(codes_h, scales_h, bits, seeds, d, masks_np, mean_h)
+
+        e2e_step()
+        barrier()
+        es = max(2, min(args.steps, 5))
+        s_ev, t_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s_ev.record()
+        for _ in range(es):
+            e2e_step()
+        t_ev.record()
+        barrier()
+        e_ms = s_ev.elapsed_time(t_ev) / es
+        tt = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e_ms = float(tt.item())
+        code_bytes = sum(int(c.nbytes) for c in codes_h)
+        mask_bytes = sum(int(m.nbytes) for m in masks_np) if masks_np else 0
+        e2e = {"value": world * in_bytes / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": in_bytes + code_bytes + mask_bytes + 4 * n,
+               "d2h_bytes_per_step": code_bytes + 4 * n + 4 * d, "ms_per_step": e_ms,
+               "check": "max |mean_host - mean_dev| = %g" %
+                        float(np.max(np.abs(mean_h - mean.cpu().numpy())))}
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        threads = min(cores, n, 8)
+        d_s = min(d, 1 << 26)       # about 10-30 s of CPU work
+        sample = synth.make(args.workload, d=d_s, n=threads, seed=rank)
+        dt, nbytes, _ = oracle_sample(sample, list(range(threads)), threads)
+        cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "%d clients x first %d coordinates of %s, encode + decode+mean, %.1f s" %
+                         (threads, d_s, work.name, dt)}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": config_of(work, {"parallelism": "replicas x%d" % world}),
+                "encode_gbs": in_bytes / (enc_ms * 1e-3) / 1e9, "decode_mean_gbs": in_bytes / (dec_ms * 1e-3) / 1e9,
+                "encode_ms": enc_ms, "decode_mean_ms": dec_ms,
+                "roofline": roofline, "kernels": kernel_table, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": int(launches), "clocks": clocks, "nmse_vs_true_mean": nmse,
+                "status_word": status}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg5",
+                    choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "sweep"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

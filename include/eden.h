@@ -177,6 +177,16 @@ int eden_status(eden_ctx* ctx, uint32_t* device_status_word);
 int eden_client_stats(eden_ctx* ctx, uint32_t n, eden_client_stat* out);
 /* Number of kernels the library has launched on this context so far. */
 uint64_t eden_launch_count(const eden_ctx* ctx);
+
+/* Optional per-kernel timing for benchmarks: while enabled, every kernel launch is
+ * bracketed by CUDA events on the context's stream.  eden_profile_collect synchronises
+ * and folds the records since eden_profile_enable(ctx, 1) into one entry per kernel
+ * name; eden_profile_get returns entry i: launches, summed event time (ms) and summed
+ * algorithmic bytes (what the step must read and write, not what it happened to move). */
+int eden_profile_enable(eden_ctx* ctx, int on);
+int eden_profile_collect(eden_ctx* ctx, uint32_t* n_kernels);
+int eden_profile_get(eden_ctx* ctx, uint32_t i, const char** name, uint64_t* launches,
+                     double* ms_total, double* bytes_total);
 const char* eden_strerror(int code);
 
 #ifdef __cplusplus

@@ -154,6 +154,18 @@ extern "C" const char* eden_strerror(int code)
 // ------------------------------------------------------------------------------------
 // context
 // ------------------------------------------------------------------------------------
+struct ProfileRecord {
+    const char* name;
+    double bytes;                    // algorithmic bytes of this launch
+    cudaEvent_t start, stop;
+};
+
+struct ProfileSummary {
+    const char* name;
+    uint64_t launches;
+    double ms, bytes;
+};
+
 struct eden_ctx {
     int device;
     cudaStream_t stream;
@@ -162,16 +174,46 @@ struct eden_ctx {
     uint64_t launches;
     std::vector<uint32_t> order;     // processing order of the last call: order[j] = client
     uint64_t states_off;             // where the last call put its ClientState array
+    bool profiling;
+    std::vector<ProfileRecord> records;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
+    std::vector<ProfileSummary> summary;
 };
+
+static void profile_begin(eden_ctx* ctx, const char* name, double bytes)
+{
+    if (!ctx->profiling) return;
+    ProfileRecord r;
+    r.name = name;
+    r.bytes = bytes;
+    if (ctx->records.size() < ctx->event_pool.size()) {
+        r.start = ctx->event_pool[ctx->records.size()].first;
+        r.stop = ctx->event_pool[ctx->records.size()].second;
+    } else {
+        if (cudaEventCreate(&r.start) != cudaSuccess || cudaEventCreate(&r.stop) != cudaSuccess) return;
+        ctx->event_pool.push_back({r.start, r.stop});
+    }
+    cudaEventRecord(r.start, ctx->stream);
+    ctx->records.push_back(r);
+}
+
+static void profile_end(eden_ctx* ctx)
+{
+    if (!ctx->profiling || ctx->records.empty()) return;
+    cudaEventRecord(ctx->records.back().stop, ctx->stream);
+}
 
 #define CUDA_OK(expr)                                 \
     do {                                              \
         if ((expr) != cudaSuccess) return EDEN_ERR_CUDA; \
     } while (0)
 
-#define LAUNCH(ctx, kernel, grid, block, smem, ...)                          \
+// name and algorithmic bytes feed the optional per-kernel event timing (eden_profile_*)
+#define LAUNCH(ctx, name, bytes, kernel, grid, block, smem, ...)             \
     do {                                                                     \
+        profile_begin(ctx, name, (double)(bytes));                           \
         kernel<<<grid, block, smem, (ctx)->stream>>>(__VA_ARGS__);           \
+        profile_end(ctx);                                                    \
         ++(ctx)->launches;                                                   \
         if (cudaGetLastError() != cudaSuccess) return EDEN_ERR_CUDA;         \
     } while (0)
@@ -190,6 +232,7 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->ws_bytes = workspace_bytes;
     ctx->launches = 0;
     ctx->states_off = 0;
+    ctx->profiling = false;
     const Tables& t = tables();
     if (cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_pos_value, t.pos_value, sizeof(t.pos_value)) != cudaSuccess ||
@@ -205,11 +248,61 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
 extern "C" int eden_destroy(eden_ctx* ctx)
 {
     if (!ctx) return EDEN_ERR_INVALID_ARG;
+    for (auto& e : ctx->event_pool) {
+        cudaEventDestroy(e.first);
+        cudaEventDestroy(e.second);
+    }
     delete ctx;
     return EDEN_OK;
 }
 
 extern "C" uint64_t eden_launch_count(const eden_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int eden_profile_enable(eden_ctx* ctx, int on)
+{
+    if (!ctx) return EDEN_ERR_INVALID_ARG;
+    ctx->profiling = on != 0;
+    ctx->records.clear();
+    ctx->summary.clear();
+    return EDEN_OK;
+}
+
+extern "C" int eden_profile_collect(eden_ctx* ctx, uint32_t* n_kernels)
+{
+    if (!ctx || !n_kernels) return EDEN_ERR_INVALID_ARG;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    CUDA_OK(cudaStreamSynchronize(ctx->stream));
+    ctx->summary.clear();
+    for (const ProfileRecord& r : ctx->records) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) return EDEN_ERR_CUDA;
+        ProfileSummary* s = nullptr;
+        for (ProfileSummary& t : ctx->summary)
+            if (std::strcmp(t.name, r.name) == 0) s = &t;
+        if (!s) {
+            ctx->summary.push_back(ProfileSummary{r.name, 0, 0.0, 0.0});
+            s = &ctx->summary.back();
+        }
+        s->launches += 1;
+        s->ms += ms;
+        s->bytes += r.bytes;
+    }
+    ctx->records.clear();
+    *n_kernels = (uint32_t)ctx->summary.size();
+    return EDEN_OK;
+}
+
+extern "C" int eden_profile_get(eden_ctx* ctx, uint32_t i, const char** name, uint64_t* launches,
+                                double* ms_total, double* bytes_total)
+{
+    if (!ctx || i >= ctx->summary.size() || !name || !launches || !ms_total || !bytes_total)
+        return EDEN_ERR_INVALID_ARG;
+    *name = ctx->summary[i].name;
+    *launches = ctx->summary[i].launches;
+    *ms_total = ctx->summary[i].ms;
+    *bytes_total = ctx->summary[i].bytes;
+    return EDEN_OK;
+}
 
 extern "C" int eden_status(eden_ctx* ctx, uint32_t* word)
 {
@@ -331,6 +424,14 @@ int make_groups(const std::vector<ClientPlan>& plan, uint64_t work_bytes, std::v
     return EDEN_OK;
 }
 
+// Mean code width of a group's members (bits per rotated coordinate on the wire).
+double code_bits_per_coord(const std::vector<ClientPlan>& plan, const Group& g)
+{
+    double w = 0.0;
+    for (uint32_t m : g.members) w += plan[m].W;
+    return w / (double)g.members.size();
+}
+
 // Column passes over the bits above the row pass, top range first.
 struct BitRange { int lo, lr; };
 
@@ -369,12 +470,12 @@ int run_selection(eden_ctx* ctx, const FixedLayout& f, uint64_t seed, uint64_t d
     const uint64_t calls = (d + 3) / 4;
     const unsigned grid = (unsigned)((calls + kSelThreads - 1) / kSelThreads);
     CUDA_OK(cudaMemsetAsync(hist, 0, kHistBytes, ctx->stream));
-    LAUNCH(ctx, k_sel_hist, grid, kSelThreads, 0, seed, d, 0, sel, hist);
-    LAUNCH(ctx, k_sel_find, 1, 1024, 0, hist, k, 0, sel);
-    LAUNCH(ctx, k_sel_hist, grid, kSelThreads, 0, seed, d, 1, sel, hist + 65536);
-    LAUNCH(ctx, k_sel_find, 1, 1024, 0, hist + 65536, k, 1, sel);
-    LAUNCH(ctx, k_sel_chunk_count, grid, kSelThreads, 0, seed, d, sel, chunks);
-    LAUNCH(ctx, k_sel_chunk_scan, 1, 1024, 0, chunks, (uint64_t)grid);
+    LAUNCH(ctx, "sel_hist", 0, k_sel_hist, grid, kSelThreads, 0, seed, d, 0, sel, hist);
+    LAUNCH(ctx, "sel_find", 65536 * 4, k_sel_find, 1, 1024, 0, hist, k, 0, sel);
+    LAUNCH(ctx, "sel_hist", 0, k_sel_hist, grid, kSelThreads, 0, seed, d, 1, sel, hist + 65536);
+    LAUNCH(ctx, "sel_find", 65536 * 4, k_sel_find, 1, 1024, 0, hist + 65536, k, 1, sel);
+    LAUNCH(ctx, "sel_chunk_count", grid * 8.0, k_sel_chunk_count, grid, kSelThreads, 0, seed, d, sel, chunks);
+    LAUNCH(ctx, "sel_chunk_scan", grid * 16.0, k_sel_chunk_scan, 1, 1024, 0, chunks, (uint64_t)grid);
     return EDEN_OK;
 }
 
@@ -447,13 +548,13 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
             rc = run_selection(ctx, f, seeds[p.index], d, p.k);
             if (rc) return rc;
             const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
-            LAUNCH(ctx, k_sel_apply<SEL_COMPACT>, grid, kSelThreads, 0, seeds[p.index], d,
+            LAUNCH(ctx, "sel_compact", 4.0 * d + 4.0 * p.k, k_sel_apply<SEL_COMPACT>, grid, kSelThreads, 0, seeds[p.index], d,
                    (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
                    x + (uint64_t)p.index * ld_x, descs[first].work, (uint32_t*)nullptr);
         }
         if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);
-            LAUNCH(ctx, k_enc_last<true>, dim3(1, gn), kGenericThreads, sizeof(float) << g.L,
+            LAUNCH(ctx, "enc_single", gn * (4.0 * std::min<uint64_t>(d, 1ull << g.L) + (double)(1ull << g.L) / 8), k_enc_last<true>, dim3(1, gn), kGenericThreads, sizeof(float) << g.L,
                    d_descs + first, d_states + first, rg);
         } else {
             const int lc = kGenericTileLog;
@@ -463,18 +564,18 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
                 const PassGeom cg = column_geom(cols[pi]);
                 const unsigned tiles = (unsigned)((1ull << g.L) >> cg.lt);
                 if (pi == 0)
-                    LAUNCH(ctx, k_enc_first, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
+                    LAUNCH(ctx, "enc_first", gn * (4.0 * std::min<uint64_t>(d, 1ull << g.L) + 4.0 * (double)(1ull << g.L)), k_enc_first, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
                            d_descs + first, d_states + first, cg);
                 else
-                    LAUNCH(ctx, k_mid, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
+                    LAUNCH(ctx, "mid", gn * 8.0 * (double)(1ull << g.L), k_mid, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
                            d_descs + first, cg);
             }
             const PassGeom rg = row_geom(lc);
-            LAUNCH(ctx, k_enc_last<false>, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
+            LAUNCH(ctx, "enc_last", gn * (4.0 + code_bits_per_coord(plan, g) / 8.0) * (double)(1ull << g.L), k_enc_last<false>, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
                    sizeof(float) << lc, d_descs + first, d_states + first, rg);
         }
     }
-    LAUNCH(ctx, k_enc_scale, (n + 127) / 128, 128, 0, d_descs, d_states, scales, n, d_status);
+    LAUNCH(ctx, "enc_scale", n * 20.0, k_enc_scale, (n + 127) / 128, 128, 0, d_descs, d_states, scales, n, d_status);
     return EDEN_OK;
 }
 
@@ -536,7 +637,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
     ctx->states_off = lay.states_off;
     CUDA_OK(cudaMemcpyAsync(d_descs, descs.data(), sizeof(ClientDesc) * n, cudaMemcpyHostToDevice, ctx->stream));
     CUDA_OK(cudaMemsetAsync(d_states, 0, sizeof(ClientState) * n, ctx->stream));
-    LAUNCH(ctx, k_dec_prep, n, 256, 0, d_descs, d_states, scales, d_status);
+    LAUNCH(ctx, "dec_prep", n * 8.0, k_dec_prep, n, 256, 0, d_descs, d_states, scales, d_status);
 
     // the first group with b >= 1 covers every output coordinate, so for the mean it may
     // overwrite; everything after it accumulates
@@ -556,11 +657,11 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         }
         if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);
-            LAUNCH(ctx, k_dec_last<true>, dim3(1), kGenericThreads, sizeof(float) << g.L,
+            LAUNCH(ctx, "dec_single", gn * code_bits_per_coord(plan, g) / 8.0 * (double)(1ull << g.L) + 4.0 * d, k_dec_last<true>, dim3(1), kGenericThreads, sizeof(float) << g.L,
                    d_descs + first, d_states + first, gn, rg, out, d, mode);
         } else {
             const int lc = kGenericTileLog;
-            LAUNCH(ctx, k_dec_first, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
+            LAUNCH(ctx, "dec_first", gn * (4.0 + code_bits_per_coord(plan, g) / 8.0) * (double)(1ull << g.L), k_dec_first, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
                    sizeof(float) << lc, d_descs + first, row_geom(lc));
             std::vector<BitRange> cols;
             column_ranges(g.L, lc, 8, cols);
@@ -568,17 +669,17 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
                 const PassGeom cg = column_geom(cols[pi]);
                 const unsigned tiles = (unsigned)((1ull << g.L) >> cg.lt);
                 if (pi + 1 < cols.size())
-                    LAUNCH(ctx, k_mid, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
+                    LAUNCH(ctx, "mid", gn * 8.0 * (double)(1ull << g.L), k_mid, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
                            d_descs + first, cg);
                 else
-                    LAUNCH(ctx, k_dec_last<false>, dim3(tiles), kGenericThreads, sizeof(float) << cg.lt,
+                    LAUNCH(ctx, "dec_last", gn * 4.0 * (double)(1ull << g.L) + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<uint64_t>(d, 1ull << g.L), k_dec_last<false>, dim3(tiles), kGenericThreads, sizeof(float) << cg.lt,
                            d_descs + first, d_states + first, gn, cg, out, d, mode);
             }
         }
         if (g.subbit) {
             const ClientPlan& p = plan[g.members[0]];
             const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
-            LAUNCH(ctx, k_sel_apply<SEL_SCATTER_ACC>, grid, kSelThreads, 0, seeds[p.index], d,
+            LAUNCH(ctx, "sel_scatter", 8.0 * p.k + 4.0 * p.k, k_sel_apply<SEL_SCATTER_ACC>, grid, kSelThreads, 0, seeds[p.index], d,
                    (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
                    (const float*)descs[first].work, out, (uint32_t*)nullptr);
         } else {
@@ -617,7 +718,7 @@ extern "C" int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d
     const int rc = run_selection(ctx, f, seed, d, eden_kept_count(d, bits));
     if (rc) return rc;
     const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
-    LAUNCH(ctx, k_sel_apply<SEL_MASK_BITS>, grid, kSelThreads, 0, seed, d,
+    LAUNCH(ctx, "sel_mask_bits", d / 8.0, k_sel_apply<SEL_MASK_BITS>, grid, kSelThreads, 0, seed, d,
            (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
            (const float*)nullptr, (float*)nullptr, mask_bits);
     return EDEN_OK;

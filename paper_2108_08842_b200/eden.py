@@ -59,6 +59,10 @@ _sig("eden_status", _int, [_vp, ctypes.POINTER(_u32)])
 _sig("eden_client_stats", _int, [_vp, _u32, _vp])
 _sig("eden_launch_count", _u64, [_vp])
 _sig("eden_strerror", ctypes.c_char_p, [_int])
+_sig("eden_profile_enable", _int, [_vp, _int])
+_sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
+_sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(_u64),
+                                ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
 
 STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA = 1, 2, 4
 PACKET_COORDS = 1024
@@ -244,6 +248,22 @@ class Context:
         arr = (ClientStat * n)()
         _check(_lib.eden_client_stats(self._h, n, arr))
         return [dict(norm2=a.norm2, dot=a.dot, received=a.received, flags=a.flags) for a in arr]
+
+    def profile(self, on: bool):
+        _check(_lib.eden_profile_enable(self._h, 1 if on else 0))
+
+    def profile_collect(self):
+        """Per-kernel totals since profile(True): name -> dict(launches, ms, bytes)."""
+        n = _u32(0)
+        _check(_lib.eden_profile_collect(self._h, ctypes.byref(n)))
+        out = {}
+        for i in range(n.value):
+            name, launches, ms, nbytes = ctypes.c_char_p(), _u64(0), _f64(0), _f64(0)
+            _check(_lib.eden_profile_get(self._h, i, ctypes.byref(name), ctypes.byref(launches),
+                                         ctypes.byref(ms), ctypes.byref(nbytes)))
+            out[name.value.decode()] = dict(launches=int(launches.value), ms=float(ms.value),
+                                            bytes=float(nbytes.value))
+        return out
 
     @property
     def launch_count(self) -> int:
