@@ -151,6 +151,29 @@ int eden_mean(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
 int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bits,
                              uint32_t* mask_bits);
 
+/* The same mask as eden_sparsification_mask, for callers that cannot allocate device
+ * memory and therefore have no workspace to build a context on: code running inside a
+ * host application whose own allocator already holds the whole card, a service that
+ * fixes its memory map at start-up, a loop that cannot afford the device-wide stall of
+ * an allocation.  (The paper has no counterpart: this entry point exists for those
+ * callers only.)  It needs no eden_ctx and calls no cudaMalloc/cudaFree or any other
+ * allocating routine: its scratch (selection state, two 65536-bin histograms, per-chunk
+ * counts; about 0.65 MB) is a fixed array inside the library, resident on every GPU that
+ * loads the library until the process exits.
+ *   cuda_device, cuda_stream   where to run (stream as void*, NULL = default stream)
+ *   seed, d, bits              as for eden_sparsification_mask; 0 < bits < 1
+ *   mask_bits                  dev, ceil(d/32) words, caller-owned, overwritten
+ * Limits and rules: d <= EDEN_NOALLOC_MAX_DIM, larger d returns EDEN_ERR_TOO_LARGE.  The
+ * first call on a device looks up the array's device address (once per device, with that
+ * device made current); make that first call before any stream capture begins.  All
+ * calls on a device share the one array, which keeps the previous call's contents (the
+ * entry point clears what must start at zero): two calls whose GPU work overlaps -- two
+ * streams, two threads -- race on it; run them on one stream or order them yourself.
+ * Asynchronous on cuda_stream like the other entry points. */
+#define EDEN_NOALLOC_MAX_DIM (1ull << 24)
+int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stream, uint64_t seed,
+                                     uint64_t d, double bits, uint32_t* mask_bits);
+
 /* ---- the same two steps on host memory (copies included) --------------------------- */
 
 /* x, codes (array of n host pointers), scales are HOST buffers (pinned memory makes the

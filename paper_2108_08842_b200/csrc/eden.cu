@@ -827,3 +827,76 @@ extern "C" int eden_mean_host(eden_ctx* ctx, const uint8_t* const* codes_host, c
     CUDA_OK(cudaStreamSynchronize(ctx->stream));
     return EDEN_OK;
 }
+
+// ------------------------------------------------------------------------------------
+// Sparsification mask without any allocation or context.
+//
+// Some callers cannot hand this library a workspace because they cannot allocate device
+// memory at the moment they need the mask: a receiver thread inside a host application
+// whose caching allocator has already claimed the whole card (a raw cudaMalloc fails
+// there), a service that freezes its memory map after start-up, or a latency-critical
+// loop that must not take the device-wide synchronisation an allocation implies.  For
+// them the scratch of the mask selection lives in the array below, which every GPU that
+// loads this library carries until the process exits.
+// ------------------------------------------------------------------------------------
+namespace {
+
+constexpr uint64_t kNoallocMaxDim = EDEN_NOALLOC_MAX_DIM;
+constexpr uint64_t kNoallocSelOff = 0;
+constexpr uint64_t kNoallocHistOff = 256;
+constexpr uint64_t kNoallocChunkOff = kNoallocHistOff + kHistBytes;
+constexpr uint64_t kNoallocBytes =
+    kNoallocChunkOff + (kNoallocMaxDim / kSelChunk) * sizeof(unsigned long long);
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocBytes];
+
+// In host code the name g_noalloc_scratch is only a handle: the device address has to be
+// asked for, once per device, with that device current.
+constexpr int kNoallocMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+unsigned char* g_noalloc_ptr[kNoallocMaxDevices];
+
+int noalloc_scratch(int device, unsigned char** out)
+{
+    if (device < 0 || device >= kNoallocMaxDevices) return EDEN_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[device]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return EDEN_ERR_CUDA;
+        g_noalloc_ptr[device] = (unsigned char*)p;
+    }
+    *out = g_noalloc_ptr[device];
+    return EDEN_OK;
+}
+
+}  // namespace
+
+extern "C" int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stream, uint64_t seed,
+                                                uint64_t d, double bits, uint32_t* mask_bits)
+{
+    if (!mask_bits || d == 0 || !(bits > 0.0) || !(bits < 1.0)) return EDEN_ERR_INVALID_ARG;
+    if (d > kNoallocMaxDim) return EDEN_ERR_TOO_LARGE;
+    CUDA_OK(cudaSetDevice(cuda_device));
+    unsigned char* base = nullptr;
+    const int rc = noalloc_scratch(cuda_device, &base);
+    if (rc) return rc;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    MaskSelect* sel = (MaskSelect*)(base + kNoallocSelOff);
+    uint32_t* hist = (uint32_t*)(base + kNoallocHistOff);
+    unsigned long long* chunks = (unsigned long long*)(base + kNoallocChunkOff);
+    const uint64_t k = eden_kept_count(d, bits);
+    const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
+    // the array keeps the previous call's contents: the histograms must start at zero;
+    // everything else is overwritten before it is read
+    CUDA_OK(cudaMemsetAsync(hist, 0, kHistBytes, stream));
+    k_sel_hist<<<grid, kSelThreads, 0, stream>>>(seed, d, 0, sel, hist);
+    k_sel_find<<<1, 1024, 0, stream>>>(hist, k, 0, sel);
+    k_sel_hist<<<grid, kSelThreads, 0, stream>>>(seed, d, 1, sel, hist + 65536);
+    k_sel_find<<<1, 1024, 0, stream>>>(hist + 65536, k, 1, sel);
+    k_sel_chunk_count<<<grid, kSelThreads, 0, stream>>>(seed, d, sel, chunks);
+    k_sel_chunk_scan<<<1, 1024, 0, stream>>>(chunks, (uint64_t)grid);
+    k_sel_apply<SEL_MASK_BITS><<<grid, kSelThreads, 0, stream>>>(
+        seed, d, sel, chunks, (const float*)nullptr, (float*)nullptr, mask_bits);
+    if (cudaGetLastError() != cudaSuccess) return EDEN_ERR_CUDA;
+    return EDEN_OK;
+}

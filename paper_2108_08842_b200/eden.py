@@ -58,6 +58,7 @@ _sig("eden_mean_host", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp])
 _sig("eden_status", _int, [_vp, ctypes.POINTER(_u32)])
 _sig("eden_client_stats", _int, [_vp, _u32, _vp])
 _sig("eden_launch_count", _u64, [_vp])
+_sig("eden_sparsification_mask_noalloc", _int, [_int, _vp, _u64, _u64, _f64, _vp])
 _sig("eden_strerror", ctypes.c_char_p, [_int])
 _sig("eden_profile_enable", _int, [_vp, _int])
 _sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
@@ -268,6 +269,22 @@ class Context:
     @property
     def launch_count(self) -> int:
         return int(_lib.eden_launch_count(self._h))
+
+
+NOALLOC_MAX_DIM = 1 << 24
+
+
+def sparsification_mask_noalloc(seed: int, d: int, bits: float, out: torch.Tensor,
+                                device: int = 0, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """eden_sparsification_mask_noalloc: the b < 1 mask bitmap for callers that cannot
+    allocate device memory (no context, no workspace; scratch is a fixed array inside the
+    library).  `out` is a caller-owned CUDA int32 tensor of ceil(d/32) words.  Calls that
+    overlap on the GPU share that scratch and race; keep them on one stream."""
+    assert out.is_cuda and out.dtype == torch.int32 and out.numel() >= (d + 31) // 32
+    s = stream if stream is not None else torch.cuda.current_stream(device)
+    _check(_lib.eden_sparsification_mask_noalloc(device, s.cuda_stream, int(seed), int(d), float(bits),
+                                                 out.data_ptr()))
+    return out
 
 
 # module-level calls with the names of the C entry points ---------------------------------
