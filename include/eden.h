@@ -201,6 +201,10 @@ int eden_client_stats(eden_ctx* ctx, uint32_t n, eden_client_stat* out);
 /* Number of kernels the library has launched on this context so far. */
 uint64_t eden_launch_count(const eden_ctx* ctx);
 
+/* Cross-checking aid: with on != 0 every call on this context uses the shape-generic
+ * kernels instead of the register-blocked ones (same results, slower). */
+int eden_force_generic_kernels(eden_ctx* ctx, int on);
+
 /* Optional per-kernel timing for benchmarks: while enabled, every kernel launch is
  * bracketed by CUDA events on the context's stream.  eden_profile_collect synchronises
  * and folds the records since eden_profile_enable(ctx, 1) into one entry per kernel

@@ -11,6 +11,7 @@
 
 #include "eden_device.cuh"
 #include "kernels_generic.cuh"
+#include "kernels_fast.cuh"
 #include "kernels_select.cuh"
 #include "lloyd_max.h"
 
@@ -175,6 +176,7 @@ struct eden_ctx {
     std::vector<uint32_t> order;     // processing order of the last call: order[j] = client
     uint64_t states_off;             // where the last call put its ClientState array
     bool profiling;
+    bool force_generic;
     std::vector<ProfileRecord> records;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
     std::vector<ProfileSummary> summary;
@@ -233,6 +235,7 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->launches = 0;
     ctx->states_off = 0;
     ctx->profiling = false;
+    ctx->force_generic = false;
     const Tables& t = tables();
     if (cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_pos_value, t.pos_value, sizeof(t.pos_value)) != cudaSuccess ||
@@ -257,6 +260,13 @@ extern "C" int eden_destroy(eden_ctx* ctx)
 }
 
 extern "C" uint64_t eden_launch_count(const eden_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int eden_force_generic_kernels(eden_ctx* ctx, int on)
+{
+    if (!ctx) return EDEN_ERR_INVALID_ARG;
+    ctx->force_generic = on != 0;
+    return EDEN_OK;
+}
 
 extern "C" int eden_profile_enable(eden_ctx* ctx, int on)
 {
@@ -395,7 +405,9 @@ int make_groups(const std::vector<ClientPlan>& plan, uint64_t work_bytes, std::v
     std::vector<uint32_t> idx;
     for (uint32_t c = 0; c < plan.size(); ++c)
         if (!plan[c].subbit) idx.push_back(c);
-    std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) { return plan[a].L > plan[b].L; });
+    std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
+        return plan[a].L != plan[b].L ? plan[a].L > plan[b].L : plan[a].W < plan[b].W;
+    });
     size_t i = 0;
     while (i < idx.size()) {
         Group g;
@@ -460,6 +472,127 @@ PassGeom column_geom(const BitRange& r)
 
 PassGeom row_geom(int lc) { return PassGeom{lc, lc, lc, 0}; }
 
+// Column passes of the register-blocked path: the bits above the 13-bit row pass, split
+// into passes of at most kFastMaxColBits bits, top range first.
+void fast_column_ranges(int L, std::vector<BitRange>& out)
+{
+    const int cb = L - kFastTileLog;
+    const int passes = (cb + kFastMaxColBits - 1) / kFastMaxColBits;
+    int hi = L;
+    for (int p = 0; p < passes; ++p) {
+        const int lr = (hi - kFastTileLog + (passes - p) - 1) / (passes - p);
+        out.push_back({hi - lr, lr});
+        hi -= lr;
+    }
+}
+
+#define EDEN_DISPATCH_LR(lr, CALL)                \
+    switch (lr) {                                 \
+        case 1: { constexpr int LR_ = 1; CALL; } break; \
+        case 2: { constexpr int LR_ = 2; CALL; } break; \
+        case 3: { constexpr int LR_ = 3; CALL; } break; \
+        case 4: { constexpr int LR_ = 4; CALL; } break; \
+        case 5: { constexpr int LR_ = 5; CALL; } break; \
+        case 6: { constexpr int LR_ = 6; CALL; } break; \
+        case 7: { constexpr int LR_ = 7; CALL; } break; \
+        default: return EDEN_ERR_INVALID_ARG;     \
+    }
+
+#define EDEN_DISPATCH_W(w, CALL)                  \
+    switch (w) {                                  \
+        case 1: { constexpr int W_ = 1; CALL; } break; \
+        case 2: { constexpr int W_ = 2; CALL; } break; \
+        case 3: { constexpr int W_ = 3; CALL; } break; \
+        case 4: { constexpr int W_ = 4; CALL; } break; \
+        case 5: { constexpr int W_ = 5; CALL; } break; \
+        case 6: { constexpr int W_ = 6; CALL; } break; \
+        case 7: { constexpr int W_ = 7; CALL; } break; \
+        case 8: { constexpr int W_ = 8; CALL; } break; \
+        default: return EDEN_ERR_INVALID_ARG;     \
+    }
+
+// Runs of equal code width inside a group (members are sorted by width within a group).
+struct WidthRun { uint32_t first, count; int W; };
+
+void width_runs(const std::vector<ClientPlan>& plan, const Group& g, std::vector<WidthRun>& runs)
+{
+    for (uint32_t j = 0; j < g.members.size(); ++j) {
+        const int W = plan[g.members[j]].W;
+        if (!runs.empty() && runs.back().W == W) ++runs.back().count;
+        else runs.push_back({j, 1u, W});
+    }
+}
+
+// Sender passes of one group on the register-blocked path.
+int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g,
+                      ClientDesc* d_descs, ClientState* d_states, uint64_t d)
+{
+    const uint32_t gn = (uint32_t)g.members.size();
+    const double D = (double)(1ull << g.L);
+    const unsigned tiles = (unsigned)((1ull << g.L) >> kFastTileLog);
+    std::vector<BitRange> cols;
+    fast_column_ranges(g.L, cols);
+    for (size_t pi = 0; pi < cols.size(); ++pi) {
+        const int lo = cols[pi].lo;
+        if (pi == 0) {
+            EDEN_DISPATCH_LR(cols[pi].lr,
+                LAUNCH(ctx, "f_enc_first", gn * (4.0 * std::min<double>((double)d, D) + 4.0 * D),
+                       k_f_enc_first<LR_>, dim3(tiles, gn), kFastThreads, 0, d_descs, d_states, lo));
+        } else {
+            EDEN_DISPATCH_LR(cols[pi].lr,
+                LAUNCH(ctx, "f_mid", gn * 8.0 * D, k_f_mid<LR_>, dim3(tiles, gn), kFastThreads, 0,
+                       d_descs, lo));
+        }
+    }
+    std::vector<WidthRun> runs;
+    width_runs(plan, g, runs);
+    for (const WidthRun& r : runs) {
+        EDEN_DISPATCH_W(r.W,
+            LAUNCH(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, k_f_enc_last<W_>,
+                   dim3(tiles, r.count), kFastThreads, 0, d_descs + r.first, d_states + r.first));
+    }
+    return EDEN_OK;
+}
+
+// Receiver passes of one group on the register-blocked path.
+int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g,
+                      ClientDesc* d_descs, ClientState* d_states, float* out, uint64_t d, int mode)
+{
+    const uint32_t gn = (uint32_t)g.members.size();
+    const double D = (double)(1ull << g.L);
+    const unsigned tiles = (unsigned)((1ull << g.L) >> kFastTileLog);
+    std::vector<WidthRun> runs;
+    width_runs(plan, g, runs);
+    for (const WidthRun& r : runs) {
+        EDEN_DISPATCH_W(r.W,
+            LAUNCH(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, k_f_dec_first<W_>,
+                   dim3(tiles, r.count), kFastThreads, 0, d_descs + r.first));
+    }
+    std::vector<BitRange> cols;
+    fast_column_ranges(g.L, cols);
+    // the receiver walks the column ranges bottom-up so that the top range comes last
+    for (size_t pi = cols.size(); pi-- > 0;) {
+        const int lo = cols[pi].lo;
+        if (pi > 0) {
+            EDEN_DISPATCH_LR(cols[pi].lr,
+                LAUNCH(ctx, "f_mid", gn * 8.0 * D, k_f_mid<LR_>, dim3(tiles, gn), kFastThreads, 0,
+                       d_descs, lo));
+        } else {
+            EDEN_DISPATCH_LR(cols[pi].lr,
+                LAUNCH(ctx, "f_dec_last",
+                       gn * 4.0 * D + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<double>((double)d, D),
+                       k_f_dec_last<LR_>, dim3(tiles), kFastThreads, 0, d_descs, d_states, gn, lo,
+                       out, d, mode));
+        }
+    }
+    return EDEN_OK;
+}
+
+bool fast_eligible(const eden_ctx* ctx, const Group& g)
+{
+    return !ctx->force_generic && g.L > kFastTileLog && g.L <= kFastTileLog + 3 * kFastMaxColBits;
+}
+
 // Exact-size mask selection for one client (Section 4.1): fills the MaskSelect and the
 // scanned chunk offsets in the fixed scratch.
 int run_selection(eden_ctx* ctx, const FixedLayout& f, uint64_t seed, uint64_t d, uint64_t k)
@@ -502,6 +635,7 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
     rc = make_groups(plan, lay.work_bytes, groups);
     if (rc) return rc;
     const FixedLayout f = fixed_layout(d);
+    const bool x_aligned = ((uintptr_t)x & 15u) == 0 && (ld_x & 3u) == 0;
 
     // descriptors in processing order
     std::vector<ClientDesc> descs;
@@ -552,7 +686,10 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
                    (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
                    x + (uint64_t)p.index * ld_x, descs[first].work, (uint32_t*)nullptr);
         }
-        if (g.L <= kGenericTileLog) {
+        if (fast_eligible(ctx, g) && x_aligned) {
+            rc = fast_encode_group(ctx, plan, g, d_descs + first, d_states + first, d);
+            if (rc) return rc;
+        } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);
             LAUNCH(ctx, "enc_single", gn * (4.0 * std::min<uint64_t>(d, 1ull << g.L) + (double)(1ull << g.L) / 8), k_enc_last<true>, dim3(1, gn), kGenericThreads, sizeof(float) << g.L,
                    d_descs + first, d_states + first, rg);
@@ -655,7 +792,10 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             rc = run_selection(ctx, f, seeds[p.index], d, p.k);
             if (rc) return rc;
         }
-        if (g.L <= kGenericTileLog) {
+        if (fast_eligible(ctx, g)) {
+            rc = fast_decode_group(ctx, plan, g, d_descs + first, d_states + first, out, d, mode);
+            if (rc) return rc;
+        } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);
             LAUNCH(ctx, "dec_single", gn * code_bits_per_coord(plan, g) / 8.0 * (double)(1ull << g.L) + 4.0 * d, k_dec_last<true>, dim3(1), kGenericThreads, sizeof(float) << g.L,
                    d_descs + first, d_states + first, gn, rg, out, d, mode);

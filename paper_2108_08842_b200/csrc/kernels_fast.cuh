@@ -1,0 +1,536 @@
+// Register-blocked transform kernels for rotation dimensions of 2^14 and more.
+//
+// Every kernel works on a tile of 8192 floats with 256 threads, 32 values per thread,
+// four resident blocks per SM.  Butterflies run in registers as packed fp32 pairs
+// (add.rn.f32x2 / sub.rn.f32x2: one instruction per two coordinates); between register
+// steps the tile is transposed through shared memory with 64- or 128-bit conflict-free
+// accesses; global loads and stores are 64- or 128-bit and fully coalesced.
+//
+//  * column pass (k_f_enc_first, k_f_mid, k_f_dec_last): the tile is 2^LR rows of
+//    8192/2^LR consecutive coordinates, rows 2^lo apart; the LR row bits are transformed.
+//    Values travel as float4 (four neighbouring columns), so every stage is two packed
+//    instructions per float4 pair.
+//  * row pass (k_f_enc_last, k_f_dec_first): the tile is 8192 consecutive coordinates; all
+//    13 index bits are transformed in three register steps (5 + 4 + 4 bits) on float2
+//    units.  At the message side of the pass a thread owns 32 consecutive coordinates, so
+//    it builds (or reads) whole 32-bit code words by itself.
+#pragma once
+#include "eden_device.cuh"
+#include "kernels_generic.cuh"
+
+namespace eden {
+
+constexpr int kFastThreads = 256;
+constexpr int kFastTileLog = 13;
+constexpr int kFastMaxColBits = 7;
+
+typedef unsigned long long u64;
+
+// ---------------------------------------------------------------------------------
+// packed fp32 pairs
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ u64 pack2(float lo, float hi)
+{
+    u64 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// (a, b) -> (a + b, a - b) on both halves
+__device__ __forceinline__ void bfly2(u64& a, u64& b)
+{
+    u64 s, d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(s) : "l"(a), "l"(b));
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    a = s;
+    b = d;
+}
+// butterfly between the two halves of one pair: (x, y) -> (x + y, x - y)
+__device__ __forceinline__ u64 bfly_inner(u64 v)
+{
+    float x, y;
+    unpack2(v, x, y);
+    return pack2(x + y, x - y);
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c)
+{
+    u64 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// flips the sign of each half where the matching bit of `bits` (bit 0 -> lo, bit 1 -> hi) is set
+__device__ __forceinline__ u64 flip2(u64 v, uint32_t bits)
+{
+    const u64 m = ((u64)(bits & 1u) << 31) | ((u64)(bits & 2u) << 62);
+    return v ^ m;
+}
+
+// Butterflies over the register index bits [0, NB) of 8 float4 values (as 16 packed pairs:
+// v[2*k], v[2*k+1] are the halves of float4 k).  Only the top `nb_live` of the NB = 3 index
+// bits are transformed (bits below belong to columns).
+template <int LIVE>
+__device__ __forceinline__ void col_step(u64 (&v)[16])
+{
+#pragma unroll
+    for (int b = 3 - LIVE; b < 3; ++b) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            if (!(k & (1 << b))) {
+                bfly2(v[2 * k], v[2 * (k | (1 << b))]);
+                bfly2(v[2 * k + 1], v[2 * (k | (1 << b)) + 1]);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// Column-pass tile: float4 index q in [0, 2048); row = q >> (11 - LR).  Three register
+// arrangements (thread -> the 8 float4 it holds), arrangement s holding q bits
+// [10-3s, 8-3s] in registers:
+//   0: q = t + 256 k                         (coalesced; used for all global traffic in)
+//   1: q = (t >> 5) << 8 | k << 5 | (t & 31)
+//   2: q = (t >> 2) << 5 | k << 2 | (t & 3)
+// Shared memory holds float4 q at f(q) = q ^ (bit 5 of q) << 2, which makes the 128-bit
+// accesses of all three arrangements conflict-free.
+// ---------------------------------------------------------------------------------
+template <int ARR>
+__device__ __forceinline__ int col_q(int t, int k)
+{
+    if (ARR == 0) return t + 256 * k;
+    if (ARR == 1) return ((t >> 5) << 8) | (k << 5) | (t & 31);
+    return ((t >> 2) << 5) | (k << 2) | (t & 3);
+}
+__device__ __forceinline__ int col_swz(int q) { return q ^ (((q >> 5) & 1) << 2); }
+
+template <int FROM, int TO>
+__device__ __forceinline__ void col_exchange(u64 (&v)[16], ulonglong2* s)
+{
+    const int t = threadIdx.x;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s[col_swz(col_q<FROM>(t, k))] = make_ulonglong2(v[2 * k], v[2 * k + 1]);
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const ulonglong2 w = s[col_swz(col_q<TO>(t, k))];
+        v[2 * k] = w.x;
+        v[2 * k + 1] = w.y;
+    }
+}
+
+// number of register steps of a column pass and the arrangement it ends in
+template <int LR> struct ColSteps { static constexpr int n = (LR + 2) / 3; static constexpr int last = n - 1; };
+
+// All LR row stages of a column tile held in arrangement 0; returns in arrangement
+// ColSteps<LR>::last.  `s` is a 32 KB shared buffer.  The caller must __syncthreads()
+// before reusing `s` after this returns (the last read of `s` may still be in flight in
+// other warps).
+template <int LR>
+__device__ __forceinline__ void col_transform(u64 (&v)[16], ulonglong2* s)
+{
+    col_step<(LR >= 3 ? 3 : LR)>(v);
+    if (LR > 3) {
+        col_exchange<0, 1>(v, s);
+        col_step<(LR >= 6 ? 3 : LR - 3)>(v);
+    }
+    if (LR > 6) {
+        __syncthreads();
+        col_exchange<1, 2>(v, s);
+        col_step<LR - 6>(v);
+    }
+}
+
+struct ColTile {
+    uint64_t base;      // global index of float 0 of row 0 of this tile
+    int lo;             // log2 of the distance between rows (in floats)
+};
+
+template <int LR>
+__device__ __forceinline__ ColTile col_tile(uint64_t tile, int lo)
+{
+    constexpr int LWC = kFastTileLog - LR;            // log2 columns per row
+    const int chunk_bits = lo - LWC;
+    const uint64_t outer = tile >> chunk_bits;
+    const uint64_t chunk = tile & ((1ull << chunk_bits) - 1);
+    ColTile ct;
+    ct.base = (outer << (lo + LR)) + (chunk << LWC);
+    ct.lo = lo;
+    return ct;
+}
+
+// global float index of component 0 of float4 q of the tile
+template <int LR>
+__device__ __forceinline__ uint64_t col_index(const ColTile& ct, int q)
+{
+    constexpr int LCQ = 11 - LR;                      // log2 float4 per row
+    const uint64_t r = (uint64_t)(q >> LCQ);
+    const uint64_t cq = (uint64_t)(q & ((1 << LCQ) - 1));
+    return ct.base + (r << ct.lo) + (cq << 2);
+}
+
+// The 256 sign words (32 coordinates each) of a column tile, word w = row * (Wc/32) + j,
+// computed by the first warps (one Philox call yields four words) into shared memory.
+template <int LR>
+__device__ __forceinline__ void col_sign_words(uint64_t seed, const ColTile& ct, uint32_t* s_sign)
+{
+    constexpr int LWR = kFastTileLog - LR - 5;        // log2 words per row (Wc / 32); >= 1 for LR <= 7
+    constexpr int CALLS = LWR >= 2 ? 64 : 128;        // Philox calls per tile
+    const int t = threadIdx.x;
+    if (t < CALLS) {
+        if (LWR >= 2) {
+            // call c covers words 4c .. 4c+3 of the tile (same row, since rows hold >= 4 words)
+            const int w0 = 4 * t;
+            const uint64_t r = (uint64_t)(w0 >> LWR);
+            const uint64_t g = (ct.base + (r << ct.lo)) / 32 + (uint64_t)(w0 & ((1 << LWR) - 1));
+            const uint4 p = philox_stream(seed, 0u, g >> 2);
+            s_sign[w0] = p.x; s_sign[w0 + 1] = p.y; s_sign[w0 + 2] = p.z; s_sign[w0 + 3] = p.w;
+        } else {
+            // rows hold two words: half a call per row
+            const int w0 = 2 * t;
+            const uint64_t r = (uint64_t)(w0 >> LWR);
+            const uint64_t g = (ct.base + (r << ct.lo)) / 32;
+            const uint4 p = philox_stream(seed, 0u, g >> 2);
+            const bool upper = (g & 2) != 0;
+            s_sign[w0] = upper ? p.z : p.x;
+            s_sign[w0 + 1] = upper ? p.w : p.y;
+        }
+    }
+}
+
+// the four sign bits of float4 q of the tile
+template <int LR>
+__device__ __forceinline__ uint32_t col_sign_nibble(const uint32_t* s_sign, int q)
+{
+    constexpr int LCQ = 11 - LR;
+    const int r = q >> LCQ, cq = q & ((1 << LCQ) - 1);
+    const uint32_t w = s_sign[(r << (LCQ - 3)) + (cq >> 3)];
+    return (w >> ((cq & 7) * 4)) & 0xFu;
+}
+
+// =================================================================================
+// Sender, first pass: x -> sign flip -> ||y||^2 -> LR top stages -> work
+// =================================================================================
+template <int LR>
+__global__ void __launch_bounds__(kFastThreads, 3)
+k_f_enc_first(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo)
+{
+    __shared__ ulonglong2 s[2048];
+    __shared__ uint32_t s_sign[256];
+    __shared__ double red[32];
+    const ClientDesc cd = descs[blockIdx.y];
+    const ColTile ct = col_tile<LR>(blockIdx.x, lo);
+    const int t = threadIdx.x;
+    col_sign_words<LR>(cd.seed, ct, s_sign);
+    u64 v[16];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const uint64_t i = col_index<LR>(ct, col_q<0>(t, k));
+        float4 x;
+        if (i + 3 < cd.valid) {
+            x = *reinterpret_cast<const float4*>(cd.src + i);
+        } else {
+            x.x = i < cd.valid ? cd.src[i] : 0.f;
+            x.y = i + 1 < cd.valid ? cd.src[i + 1] : 0.f;
+            x.z = i + 2 < cd.valid ? cd.src[i + 2] : 0.f;
+            x.w = 0.f;
+        }
+        v[2 * k] = pack2(x.x, x.y);
+        v[2 * k + 1] = pack2(x.z, x.w);
+    }
+    u64 acc = 0ull;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc = fma2(v[k], v[k], acc);
+    __syncthreads();                                   // sign words ready
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const uint32_t nib = col_sign_nibble<LR>(s_sign, col_q<0>(t, k));
+        v[2 * k] = flip2(v[2 * k], nib);
+        v[2 * k + 1] = flip2(v[2 * k + 1], nib >> 2);
+    }
+    col_transform<LR>(v, s);
+    constexpr int ARR = ColSteps<LR>::last;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const uint64_t i = col_index<LR>(ct, col_q<ARR>(t, k));
+        *reinterpret_cast<ulonglong2*>(cd.work + i) = make_ulonglong2(v[2 * k], v[2 * k + 1]);
+    }
+    float a0, a1;
+    unpack2(acc, a0, a1);
+    const double tot = block_sum((double)a0 + (double)a1, red);
+    if (t == 0) atomicAdd(&states[blockIdx.y].norm2, tot);
+}
+
+// Middle pass, in place on the work buffer.
+template <int LR>
+__global__ void __launch_bounds__(kFastThreads, 3)
+k_f_mid(const ClientDesc* __restrict__ descs, int lo)
+{
+    __shared__ ulonglong2 s[2048];
+    const ClientDesc cd = descs[blockIdx.y];
+    const ColTile ct = col_tile<LR>(blockIdx.x, lo);
+    const int t = threadIdx.x;
+    u64 v[16];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const ulonglong2 w = *reinterpret_cast<const ulonglong2*>(cd.work + col_index<LR>(ct, col_q<0>(t, k)));
+        v[2 * k] = w.x;
+        v[2 * k + 1] = w.y;
+    }
+    col_transform<LR>(v, s);
+    constexpr int ARR = ColSteps<LR>::last;
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        *reinterpret_cast<ulonglong2*>(cd.work + col_index<LR>(ct, col_q<ARR>(t, k))) =
+            make_ulonglong2(v[2 * k], v[2 * k + 1]);
+}
+
+// =================================================================================
+// Receiver, last pass: for every client of the group finish the inverse transform of the
+// tile, apply sign and factor, add into registers; store the sum once (Sections 2.2.2,
+// 4.2).  mode: OUT_WRITE / OUT_ACC into out[0, d), or OUT_YHAT into the client's own work
+// buffer (b < 1, single client).
+// =================================================================================
+template <int LR>
+__global__ void __launch_bounds__(kFastThreads, 2)
+k_f_dec_last(const ClientDesc* __restrict__ descs, const ClientState* __restrict__ states,
+             uint32_t n_group, int lo, float* __restrict__ out, uint64_t d, int mode)
+{
+    __shared__ ulonglong2 s[2048];
+    __shared__ uint32_t s_sign[256];
+    const ColTile ct = col_tile<LR>(blockIdx.x, lo);
+    const int t = threadIdx.x;
+    constexpr int ARR = ColSteps<LR>::last;
+    u64 acc[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) acc[k] = 0ull;
+    for (uint32_t c = 0; c < n_group; ++c) {
+        const float* __restrict__ work = descs[c].work;
+        const uint64_t seed = descs[c].seed;
+        const float f = states[c].factor;
+        u64 v[16];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const ulonglong2 w = *reinterpret_cast<const ulonglong2*>(work + col_index<LR>(ct, col_q<0>(t, k)));
+            v[2 * k] = w.x;
+            v[2 * k + 1] = w.y;
+        }
+        __syncthreads();                               // previous client's s / s_sign reads are done
+        col_sign_words<LR>(seed, ct, s_sign);
+        col_transform<LR>(v, s);
+        if (LR <= 3) __syncthreads();                  // no exchange inside: publish the sign words
+        const u64 f2 = pack2(f, f);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t nib = col_sign_nibble<LR>(s_sign, col_q<ARR>(t, k));
+            acc[2 * k] = fma2(flip2(v[2 * k], nib), f2, acc[2 * k]);
+            acc[2 * k + 1] = fma2(flip2(v[2 * k + 1], nib >> 2), f2, acc[2 * k + 1]);
+        }
+    }
+    const uint64_t limit = mode == OUT_YHAT ? (1ull << descs[0].L) : d;
+    float* dst = mode == OUT_YHAT ? descs[0].work : out;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const uint64_t i = col_index<LR>(ct, col_q<ARR>(t, k));
+        float a[4];
+        unpack2(acc[2 * k], a[0], a[1]);
+        unpack2(acc[2 * k + 1], a[2], a[3]);
+        if (i + 3 < limit) {
+            float4* p = reinterpret_cast<float4*>(dst + i);
+            if (mode == OUT_ACC) {
+                const float4 o = *p;
+                a[0] += o.x; a[1] += o.y; a[2] += o.z; a[3] += o.w;
+            }
+            *p = make_float4(a[0], a[1], a[2], a[3]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (i + e < limit) {
+                    if (mode == OUT_ACC) dst[i + e] += a[e];
+                    else dst[i + e] = a[e];
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// Row-pass tile: 8192 consecutive floats = 4096 float2 units u; element e = 2u + half.
+// Register arrangements (thread -> its 16 units):
+//   A: u = t + 256 k             registers hold u bits 11..8  (e bits 12..9); coalesced
+//   B: u = (t >> 4) << 8 | k << 4 | (t & 15)      registers hold u bits 7..4 (e bits 8..5)
+//   C: u = t << 4 | k            registers hold u bits 3..0  (e bits 4..1): the thread
+//                                owns the 32 consecutive coordinates 32 t .. 32 t + 31
+// Shared memory holds unit u at u + (u >> 4) (one pad per 16), conflict-free for the
+// 64-bit accesses of all three arrangements.
+// ---------------------------------------------------------------------------------
+template <int ARR>
+__device__ __forceinline__ int row_u(int t, int k)
+{
+    if (ARR == 0) return t + 256 * k;
+    if (ARR == 1) return ((t >> 4) << 8) | (k << 4) | (t & 15);
+    return (t << 4) | k;
+}
+__device__ __forceinline__ int row_pad(int u) { return u + (u >> 4); }
+constexpr int kRowSmemUnits = 4096 + 256;
+
+template <int FROM, int TO>
+__device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
+{
+    const int t = threadIdx.x;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) s[row_pad(row_u<FROM>(t, k))] = v[k];
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<TO>(t, k))];
+}
+
+// butterflies over the four register index bits of 16 packed units
+__device__ __forceinline__ void row_step(u64 (&v)[16])
+{
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+#pragma unroll
+        for (int k = 0; k < 16; ++k)
+            if (!(k & (1 << b))) bfly2(v[k], v[k | (1 << b)]);
+}
+__device__ __forceinline__ void row_step_inner(u64 (&v)[16])
+{
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = bfly_inner(v[k]);
+}
+
+// =================================================================================
+// Sender, last pass: work -> 13 low stages -> z = h/||y|| -> interval -> sum h Q(z) ->
+// packed codes.  The thread ends with coordinates 32t..32t+31 of the tile and writes their
+// W code words itself.
+// =================================================================================
+template <int W>
+__device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_norm, bool live,
+                                                 const float* s_tb, const float* s_tv,
+                                                 uint32_t (&words)[W], float& dot)
+{
+    constexpr int half = 1 << (W - 1);
+    uint32_t neg_plane = 0u;
+    uint32_t mag[W > 1 ? W - 1 : 1];
+#pragma unroll
+    for (int j = 0; j < (W > 1 ? W - 1 : 1); ++j) mag[j] = 0u;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        float h[2];
+        unpack2(v[k], h[0], h[1]);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int l = 2 * k + e;
+            const float z = h[e] * inv_norm;
+            const float az = fabsf(z);
+            int m = 0;
+            if (W > 1) {
+#pragma unroll
+                for (int step = half >> 1; step >= 1; step >>= 1)
+                    m += (az > s_tb[m + step - 1]) ? step : 0;
+            }
+            dot = fmaf(fabsf(h[e]), s_tv[m], dot);
+            neg_plane |= (z < 0.f ? 1u : 0u) << l;
+#pragma unroll
+            for (int j = 0; j + 1 < W; ++j) mag[j] |= (((uint32_t)m >> j) & 1u) << l;
+        }
+    }
+    // code = half + m for z >= 0, half - 1 - m otherwise: the low planes of a negative
+    // coordinate are the complement of m's bits, the top plane is "not negative"
+#pragma unroll
+    for (int j = 0; j + 1 < W; ++j) words[j] = live ? (mag[j] ^ neg_plane) : 0u;
+    words[W - 1] = live ? ~neg_plane : 0u;
+}
+
+template <int W>
+__global__ void __launch_bounds__(kFastThreads, 3)
+k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
+{
+    __shared__ u64 s[kRowSmemUnits];
+    __shared__ double red[32];
+    __shared__ float s_tb[128], s_tv[128];
+    const ClientDesc cd = descs[blockIdx.y];
+    const int t = threadIdx.x;
+    constexpr int half = 1 << (W - 1);
+    for (int j = t; j < half; j += kFastThreads) {
+        s_tb[j] = c_pos_boundary[table_offset(W) + j];
+        s_tv[j] = c_pos_value[table_offset(W) + j];
+    }
+    const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
+    const u64* __restrict__ src = reinterpret_cast<const u64*>(cd.work + base);
+    u64 v[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) v[k] = src[row_u<0>(t, k)];
+    row_step(v);                    // e bits 12..9
+    row_exchange<0, 1>(v, s);
+    row_step(v);                    // e bits 8..5
+    __syncthreads();
+    row_exchange<1, 2>(v, s);
+    row_step(v);                    // e bits 4..1
+    row_step_inner(v);              // e bit 0
+    const double n2 = states[blockIdx.y].norm2;
+    const bool live = n2 > 0.0 && n2 < INFINITY;
+    const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
+    uint32_t words[W];
+    float dot = 0.f;
+    quantise_pack_32<W>(v, inv_norm, live, s_tb, s_tv, words, dot);
+    uint32_t* dst = cd.codes + ((base >> 5) + t) * W;
+#pragma unroll
+    for (int j = 0; j < W; ++j) dst[j] = words[j];
+    const double tot = block_sum((double)dot, red);
+    if (t == 0) atomicAdd(&states[blockIdx.y].dot, tot);
+}
+
+// =================================================================================
+// Receiver, first pass: codes -> centroids (lost packets -> 0) -> 13 low stages -> work
+// =================================================================================
+template <int W>
+__global__ void __launch_bounds__(kFastThreads, 3)
+k_f_dec_first(const ClientDesc* __restrict__ descs)
+{
+    __shared__ u64 s[kRowSmemUnits];
+    __shared__ float s_tv[128];
+    const ClientDesc cd = descs[blockIdx.y];
+    const int t = threadIdx.x;
+    constexpr int half = 1 << (W - 1);
+    for (int j = t; j < half; j += kFastThreads) s_tv[j] = c_pos_value[table_offset(W) + j];
+    __syncthreads();
+    const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
+    // the tile is 8 packets of 1024 coordinates; this thread's 32 coordinates lie in one
+    const uint64_t pkt = (base >> 10) + (uint64_t)(t >> 5);
+    const bool arrived = cd.recv ? ((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u) != 0u : true;
+    uint32_t words[W];
+    const uint32_t* src = cd.codes + ((base >> 5) + t) * W;
+#pragma unroll
+    for (int j = 0; j < W; ++j) words[j] = arrived ? src[j] : 0u;
+    u64 v[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        float q[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int l = 2 * k + e;
+            uint32_t code = 0u;
+#pragma unroll
+            for (int j = 0; j < W; ++j) code |= ((words[j] >> l) & 1u) << j;
+            const bool pos = code >= (uint32_t)half;
+            const float c = s_tv[pos ? code - half : half - 1 - code];
+            q[e] = arrived ? (pos ? c : -c) : 0.f;
+        }
+        v[k] = pack2(q[0], q[1]);
+    }
+    row_step_inner(v);              // e bit 0
+    row_step(v);                    // e bits 4..1
+    row_exchange<2, 1>(v, s);
+    row_step(v);                    // e bits 8..5
+    __syncthreads();
+    row_exchange<1, 0>(v, s);
+    row_step(v);                    // e bits 12..9
+    u64* dst = reinterpret_cast<u64*>(cd.work + base);
+#pragma unroll
+    for (int k = 0; k < 16; ++k) dst[row_u<0>(t, k)] = v[k];
+}
+
+}  // namespace eden

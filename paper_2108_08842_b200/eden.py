@@ -61,6 +61,7 @@ _sig("eden_launch_count", _u64, [_vp])
 _sig("eden_sparsification_mask_noalloc", _int, [_int, _vp, _u64, _u64, _f64, _vp])
 _sig("eden_strerror", ctypes.c_char_p, [_int])
 _sig("eden_profile_enable", _int, [_vp, _int])
+_sig("eden_force_generic_kernels", _int, [_vp, _int])
 _sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
 _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(_u64),
                                 ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
@@ -249,6 +250,9 @@ class Context:
         arr = (ClientStat * n)()
         _check(_lib.eden_client_stats(self._h, n, arr))
         return [dict(norm2=a.norm2, dot=a.dot, received=a.received, flags=a.flags) for a in arr]
+
+    def force_generic_kernels(self, on: bool):
+        _check(_lib.eden_force_generic_kernels(self._h, 1 if on else 0))
 
     def profile(self, on: bool):
         _check(_lib.eden_profile_enable(self._h, 1 if on else 0))

@@ -135,7 +135,8 @@ def test_cfg5_padding_four_bits_loss_reduced(E):
 
 # ----------------------------------------------------------------------------- shapes and edge cases
 @pytest.mark.parametrize("d", [1, 2, 5, 31, 32, 33, 100, 1023, 1024, 1025, 4097, 8192, 8193,
-                               16384, 20000, 65536, 100000, (1 << 21) + 7])
+                               16384, 20000, 65536, 100000, 1 << 18, 1 << 19, (1 << 21) + 7,
+                               (1 << 23) + 5])
 @pytest.mark.parametrize("bits", [1.0, 3.0])
 def test_shapes_and_ragged_tails(E, d, bits):
     rng = np.random.default_rng(d)
@@ -183,6 +184,45 @@ def test_mixed_budgets_in_one_call(E):
     bits = np.array([0.3, 1.0, 2.0, 0.1, 4.0, 8.0, 1.0])
     work = synth.Workload("adhoc", n, d, bits, synth.client_seeds(9, n), 0.2, lambda c: xs[c], 9)
     run_workload(E, work)
+
+
+def test_generic_kernels_agree_with_the_oracle_on_large_shapes(E):
+    # the shape-generic kernels stay in the library as the path for odd layouts (for
+    # example an input that is not 16-byte aligned); keep them under the same parity bar
+    d, n = 300000, 3
+    rng = np.random.default_rng(8)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.array([1.0, 4.0, 0.3]), synth.client_seeds(8, n), 0.1,
+                          lambda c: xs[c], 8)
+    import paper_2108_08842_b200.eden as eden_mod
+    orig = eden_mod.Context.__init__
+
+    def patched(self, *a, **k):
+        orig(self, *a, **k)
+        self.force_generic_kernels(True)
+
+    try:
+        eden_mod.Context.__init__ = patched
+        run_workload(E, work)
+    finally:
+        eden_mod.Context.__init__ = orig
+
+
+def test_unaligned_input_rows_take_the_generic_path(E):
+    d, n = 70000, 2
+    rng = np.random.default_rng(9)
+    buf = torch.from_numpy(rng.standard_normal(n * (d + 1) + 1).astype(np.float32)).cuda()
+    x = buf[1: 1 + n * (d + 1)].view(n, d + 1)[:, :d]          # rows start 4 bytes off, odd stride
+    assert x.data_ptr() % 16 != 0
+    ctx = _ctx(E, d, n)
+    codes, scales = ctx.encode(x, [2.0, 2.0], [3, 4])
+    xs = x.cpu().numpy()
+    for c in range(n):
+        mism, ok, rel, _ = parity.check_encode_client(codes[c].cpu().numpy().view(np.uint32),
+                                                      float(scales[c]), np.ascontiguousarray(xs[c]),
+                                                      2.0, 3 + c)
+        assert ok and rel <= SCALE_TOL
+    ctx.close()
 
 
 def test_zero_vector_and_status_word(E):
