@@ -185,7 +185,7 @@ def run_gpu(args):
     __graft_entry__.build()
     from paper_2108_08842_b200 import eden, synth
 
-    work = synth.make(args.workload, seed=rank)
+    work = synth.make(args.workload, n=args.n, seed=rank)
     n, d = work.n, work.d
     cores = host_cores()
     dev = torch.device("cuda", local_rank)
@@ -277,7 +277,7 @@ def run_gpu(args):
     # ---- end to end: same step through the host-buffer entry points (pinned memory),
     #      host->device and device->host copies inside the timed region
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.no_e2e:
         codes_h = [torch.empty(eden.code_bytes(d, float(b)), dtype=torch.uint8, pin_memory=True).numpy()
                    for b in bits]
         scales_h = torch.empty(n, dtype=torch.float32, pin_memory=True).numpy()
@@ -346,6 +346,8 @@ def main():
     ap.add_argument("--workload", default="cfg5",
                     choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "sweep"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--n", type=int, default=None, help="override the number of clients (small profiling runs)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (small profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
