@@ -4,6 +4,7 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -177,6 +178,7 @@ struct eden_ctx {
     uint64_t states_off;             // where the last call put its ClientState array
     bool profiling;
     bool force_generic;
+    int plan_variant;
     std::vector<ProfileRecord> records;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
     std::vector<ProfileSummary> summary;
@@ -236,6 +238,8 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->states_off = 0;
     ctx->profiling = false;
     ctx->force_generic = false;
+    ctx->plan_variant = 0;
+    if (const char* pv = std::getenv("EDEN_PLAN_VARIANT")) ctx->plan_variant = std::atoi(pv);
     const Tables& t = tables();
     if (cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_pos_value, t.pos_value, sizeof(t.pos_value)) != cudaSuccess ||
@@ -472,19 +476,80 @@ PassGeom column_geom(const BitRange& r)
 
 PassGeom row_geom(int lc) { return PassGeom{lc, lc, lc, 0}; }
 
-// Column passes of the register-blocked path: the bits above the 13-bit row pass, split
-// into passes of at most kFastMaxColBits bits, top range first.
-void fast_column_ranges(int L, std::vector<BitRange>& out)
+// Plan of the register-blocked path.  The row pass covers index bits [0, 13 + row_lc);
+// each column pass covers bits [lo, lo + lr + lc), lr of them inside a block and lc (0 or
+// 3) across the 8 blocks of a cluster.  Two sweeps over HBM up to 2^27 coordinates.
+struct FastPass { int lo, lr, lc; };
+struct FastPlan { int row_lc; std::vector<FastPass> cols; };   // cols: top range first
+
+FastPlan fast_plan(int L, int variant)
 {
+    FastPlan pl;
     const int cb = L - kFastTileLog;
-    const int passes = (cb + kFastMaxColBits - 1) / kFastMaxColBits;
-    int hi = L;
-    for (int p = 0; p < passes; ++p) {
-        const int lr = (hi - kFastTileLog + (passes - p) - 1) / (passes - p);
-        out.push_back({hi - lr, lr});
-        hi -= lr;
+    auto one = [](int lo, int bits) {
+        return bits > kFastMaxColBits ? FastPass{lo, bits - kFastClusterLog, kFastClusterLog}
+                                      : FastPass{lo, bits, 0};
+    };
+    if (cb <= kFastMaxColBits) {
+        pl.row_lc = 0;
+        pl.cols.push_back(FastPass{kFastTileLog, cb, 0});
+    } else if (cb <= kFastMaxColBits + kFastClusterLog) {
+        if (variant == 1) {            // cluster on the row pass instead of the column pass
+            pl.row_lc = kFastClusterLog;
+            pl.cols.push_back(FastPass{kFastTileLog + kFastClusterLog, cb - kFastClusterLog, 0});
+        } else if (variant == 2 && cb - 2 * kFastClusterLog >= 1) {   // clusters on both
+            pl.row_lc = kFastClusterLog;
+            pl.cols.push_back(FastPass{kFastTileLog + kFastClusterLog, cb - 2 * kFastClusterLog,
+                                       kFastClusterLog});
+        } else {
+            pl.row_lc = 0;
+            pl.cols.push_back(FastPass{kFastTileLog, cb - kFastClusterLog, kFastClusterLog});
+        }
+    } else {
+        pl.row_lc = kFastClusterLog;
+        const int low = kFastTileLog + kFastClusterLog;
+        const int rest = L - low;
+        const int per = kFastMaxColBits + kFastClusterLog;
+        const int passes = (rest + per - 1) / per;
+        int hi = L;
+        for (int p = 0; p < passes; ++p) {
+            const int bits = (hi - low + (passes - p) - 1) / (passes - p);
+            pl.cols.push_back(one(hi - bits, bits));
+            hi -= bits;
+        }
     }
+    return pl;
 }
+
+// launch with a thread-block cluster of 2^lc blocks along x (lc = 0: ordinary launch)
+template <typename... KArgs, typename... Args>
+cudaError_t launch_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, int lc, cudaStream_t stream,
+                           Args... args)
+{
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1u << lc;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = lc > 0 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+#define LAUNCH_CL(ctx, name, bytes, kernel, grid, block, lc, ...)                            \
+    do {                                                                                     \
+        profile_begin(ctx, name, (double)(bytes));                                           \
+        const cudaError_t e_ = launch_cluster(kernel, grid, block, lc, (ctx)->stream, __VA_ARGS__); \
+        profile_end(ctx);                                                                    \
+        ++(ctx)->launches;                                                                   \
+        if (e_ != cudaSuccess || cudaGetLastError() != cudaSuccess) return EDEN_ERR_CUDA;    \
+    } while (0)
 
 #define EDEN_DISPATCH_LR(lr, CALL)                \
     switch (lr) {                                 \
@@ -495,6 +560,14 @@ void fast_column_ranges(int L, std::vector<BitRange>& out)
         case 5: { constexpr int LR_ = 5; CALL; } break; \
         case 6: { constexpr int LR_ = 6; CALL; } break; \
         case 7: { constexpr int LR_ = 7; CALL; } break; \
+        case 8: { constexpr int LR_ = 8; CALL; } break; \
+        default: return EDEN_ERR_INVALID_ARG;     \
+    }
+
+#define EDEN_DISPATCH_LC(lc, CALL)                \
+    switch (lc) {                                 \
+        case 0: { constexpr int LC_ = 0; CALL; } break; \
+        case 3: { constexpr int LC_ = 3; CALL; } break; \
         default: return EDEN_ERR_INVALID_ARG;     \
     }
 
@@ -530,26 +603,27 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     const uint32_t gn = (uint32_t)g.members.size();
     const double D = (double)(1ull << g.L);
     const unsigned tiles = (unsigned)((1ull << g.L) >> kFastTileLog);
-    std::vector<BitRange> cols;
-    fast_column_ranges(g.L, cols);
-    for (size_t pi = 0; pi < cols.size(); ++pi) {
-        const int lo = cols[pi].lo;
+    const FastPlan pl = fast_plan(g.L, ctx->plan_variant);
+    for (size_t pi = 0; pi < pl.cols.size(); ++pi) {
+        const FastPass& ps = pl.cols[pi];
         if (pi == 0) {
-            EDEN_DISPATCH_LR(cols[pi].lr,
-                LAUNCH(ctx, "f_enc_first", gn * (4.0 * std::min<double>((double)d, D) + 4.0 * D),
-                       k_f_enc_first<LR_>, dim3(tiles, gn), kFastThreads, 0, d_descs, d_states, lo));
+            EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
+                LAUNCH_CL(ctx, "f_enc_first", gn * (4.0 * std::min<double>((double)d, D) + 4.0 * D),
+                          (k_f_col<LR_, LC_, true>), dim3(tiles, gn), dim3(kFastThreads), ps.lc,
+                          (const ClientDesc*)d_descs, d_states, ps.lo)));
         } else {
-            EDEN_DISPATCH_LR(cols[pi].lr,
-                LAUNCH(ctx, "f_mid", gn * 8.0 * D, k_f_mid<LR_>, dim3(tiles, gn), kFastThreads, 0,
-                       d_descs, lo));
+            EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
+                LAUNCH_CL(ctx, "f_mid", gn * 8.0 * D, (k_f_col<LR_, LC_, false>), dim3(tiles, gn),
+                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo)));
         }
     }
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
-        EDEN_DISPATCH_W(r.W,
-            LAUNCH(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, k_f_enc_last<W_>,
-                   dim3(tiles, r.count), kFastThreads, 0, d_descs + r.first, d_states + r.first));
+        EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
+            LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_>),
+                      dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
+                      (const ClientDesc*)(d_descs + r.first), d_states + r.first)));
     }
     return EDEN_OK;
 }
@@ -561,28 +635,28 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     const uint32_t gn = (uint32_t)g.members.size();
     const double D = (double)(1ull << g.L);
     const unsigned tiles = (unsigned)((1ull << g.L) >> kFastTileLog);
+    const FastPlan pl = fast_plan(g.L, ctx->plan_variant);
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
-        EDEN_DISPATCH_W(r.W,
-            LAUNCH(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, k_f_dec_first<W_>,
-                   dim3(tiles, r.count), kFastThreads, 0, d_descs + r.first));
+        EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
+            LAUNCH_CL(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, (k_f_dec_first<W_, LC_>),
+                      dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
+                      (const ClientDesc*)(d_descs + r.first))));
     }
-    std::vector<BitRange> cols;
-    fast_column_ranges(g.L, cols);
     // the receiver walks the column ranges bottom-up so that the top range comes last
-    for (size_t pi = cols.size(); pi-- > 0;) {
-        const int lo = cols[pi].lo;
+    for (size_t pi = pl.cols.size(); pi-- > 0;) {
+        const FastPass& ps = pl.cols[pi];
         if (pi > 0) {
-            EDEN_DISPATCH_LR(cols[pi].lr,
-                LAUNCH(ctx, "f_mid", gn * 8.0 * D, k_f_mid<LR_>, dim3(tiles, gn), kFastThreads, 0,
-                       d_descs, lo));
+            EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
+                LAUNCH_CL(ctx, "f_mid", gn * 8.0 * D, (k_f_col<LR_, LC_, false>), dim3(tiles, gn),
+                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo)));
         } else {
-            EDEN_DISPATCH_LR(cols[pi].lr,
-                LAUNCH(ctx, "f_dec_last",
-                       gn * 4.0 * D + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<double>((double)d, D),
-                       k_f_dec_last<LR_>, dim3(tiles), kFastThreads, 0, d_descs, d_states, gn, lo,
-                       out, d, mode));
+            EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
+                LAUNCH_CL(ctx, "f_dec_last",
+                          gn * 4.0 * D + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<double>((double)d, D),
+                          (k_f_dec_last<LR_, LC_>), dim3(tiles), dim3(kFastThreads), ps.lc,
+                          (const ClientDesc*)d_descs, (const ClientState*)d_states, gn, ps.lo, out, d, mode)));
         }
     }
     return EDEN_OK;
@@ -590,7 +664,7 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
 
 bool fast_eligible(const eden_ctx* ctx, const Group& g)
 {
-    return !ctx->force_generic && g.L > kFastTileLog && g.L <= kFastTileLog + 3 * kFastMaxColBits;
+    return !ctx->force_generic && g.L > kFastTileLog && g.L <= 40;
 }
 
 // Exact-size mask selection for one client (Section 4.1): fills the MaskSelect and the

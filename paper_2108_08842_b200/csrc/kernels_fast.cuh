@@ -14,15 +14,25 @@
 //    13 index bits are transformed in three register steps (5 + 4 + 4 bits) on float2
 //    units.  At the message side of the pass a thread owns 32 consecutive coordinates, so
 //    it builds (or reads) whole 32-bit code words by itself.
+//  * thread-block clusters (template parameter LC > 0): 2^LC blocks of a cluster hold 2^LC
+//    tiles that differ in the LC index bits just above the block's own; those stages are
+//    done by one exchange through distributed shared memory: every block fetches its
+//    1/2^LC slice of all tiles of the cluster, does the LC stages in registers and writes
+//    the results where they belong.  This is what lets 2^24 .. 2^27 coordinates be
+//    transformed in two sweeps over HBM instead of three.
 #pragma once
 #include "eden_device.cuh"
 #include "kernels_generic.cuh"
+#include <cooperative_groups.h>
 
 namespace eden {
 
 constexpr int kFastThreads = 256;
 constexpr int kFastTileLog = 13;
-constexpr int kFastMaxColBits = 7;
+constexpr int kFastMaxColBits = 8;     // row bits one block transforms in a column pass
+constexpr int kFastClusterLog = 3;     // a cluster of 8 blocks adds three more bits to a pass
+
+namespace cg = cooperative_groups;
 
 typedef unsigned long long u64;
 
@@ -143,58 +153,73 @@ __device__ __forceinline__ void col_transform(u64 (&v)[16], ulonglong2* s)
 }
 
 struct ColTile {
-    uint64_t base;      // global index of float 0 of row 0 of this tile
+    uint64_t base;      // global index of float 0 of row 0 of this block's tile
+    uint64_t base0;     // the same for the tile of cluster rank 0
+    uint64_t rank_step; // distance between the tiles of consecutive cluster ranks
     int lo;             // log2 of the distance between rows (in floats)
+    int rank;           // this block's rank in its cluster
 };
 
-template <int LR>
-__device__ __forceinline__ ColTile col_tile(uint64_t tile, int lo)
+// Tile of block blockIdx.x for a pass over index bits [lo, lo + LR + LC): the block's rows
+// are bits [lo, lo + LR); bits [lo + LR, lo + LR + LC) are the cluster rank.
+template <int LR, int LC>
+__device__ __forceinline__ ColTile col_tile(uint64_t block, int lo)
 {
     constexpr int LWC = kFastTileLog - LR;            // log2 columns per row
     const int chunk_bits = lo - LWC;
-    const uint64_t outer = tile >> chunk_bits;
-    const uint64_t chunk = tile & ((1ull << chunk_bits) - 1);
+    const uint64_t super = block >> LC;
+    const uint64_t outer = super >> chunk_bits;
+    const uint64_t chunk = super & ((1ull << chunk_bits) - 1);
     ColTile ct;
-    ct.base = (outer << (lo + LR)) + (chunk << LWC);
+    ct.rank = (int)(block & ((1u << LC) - 1));
+    ct.rank_step = 1ull << (lo + LR);
+    ct.base0 = (outer << (lo + LR + LC)) + (chunk << LWC);
+    ct.base = ct.base0 + (uint64_t)ct.rank * ct.rank_step;
     ct.lo = lo;
     return ct;
 }
 
-// global float index of component 0 of float4 q of the tile
+// offset (in floats) of component 0 of float4 q inside a tile
 template <int LR>
-__device__ __forceinline__ uint64_t col_index(const ColTile& ct, int q)
+__device__ __forceinline__ uint64_t col_offset(const ColTile& ct, int q)
 {
     constexpr int LCQ = 11 - LR;                      // log2 float4 per row
     const uint64_t r = (uint64_t)(q >> LCQ);
     const uint64_t cq = (uint64_t)(q & ((1 << LCQ) - 1));
-    return ct.base + (r << ct.lo) + (cq << 2);
+    return (r << ct.lo) + (cq << 2);
 }
 
-// The 256 sign words (32 coordinates each) of a column tile, word w = row * (Wc/32) + j,
-// computed by the first warps (one Philox call yields four words) into shared memory.
+// The 256 sign words (32 coordinates each) of the block's column tile, word w =
+// row * (Wc/32) + j, computed by the first warps into shared memory (one Philox call
+// yields the four words of 128 consecutive coordinates).
 template <int LR>
 __device__ __forceinline__ void col_sign_words(uint64_t seed, const ColTile& ct, uint32_t* s_sign)
 {
-    constexpr int LWR = kFastTileLog - LR - 5;        // log2 words per row (Wc / 32); >= 1 for LR <= 7
-    constexpr int CALLS = LWR >= 2 ? 64 : 128;        // Philox calls per tile
+    constexpr int LWR = kFastTileLog - LR - 5;        // log2 words per row (Wc / 32)
+    constexpr int CALLS = LWR >= 2 ? 64 : (LWR == 1 ? 128 : 256);
     const int t = threadIdx.x;
     if (t < CALLS) {
         if (LWR >= 2) {
-            // call c covers words 4c .. 4c+3 of the tile (same row, since rows hold >= 4 words)
+            // call t covers words 4t .. 4t+3 of the tile (same row: rows hold >= 4 words)
             const int w0 = 4 * t;
             const uint64_t r = (uint64_t)(w0 >> LWR);
             const uint64_t g = (ct.base + (r << ct.lo)) / 32 + (uint64_t)(w0 & ((1 << LWR) - 1));
             const uint4 p = philox_stream(seed, 0u, g >> 2);
             s_sign[w0] = p.x; s_sign[w0 + 1] = p.y; s_sign[w0 + 2] = p.z; s_sign[w0 + 3] = p.w;
-        } else {
+        } else if (LWR == 1) {
             // rows hold two words: half a call per row
             const int w0 = 2 * t;
-            const uint64_t r = (uint64_t)(w0 >> LWR);
-            const uint64_t g = (ct.base + (r << ct.lo)) / 32;
+            const uint64_t g = (ct.base + ((uint64_t)t << ct.lo)) / 32;
             const uint4 p = philox_stream(seed, 0u, g >> 2);
             const bool upper = (g & 2) != 0;
             s_sign[w0] = upper ? p.z : p.x;
             s_sign[w0 + 1] = upper ? p.w : p.y;
+        } else {
+            // rows hold one word: a quarter of a call per row
+            const uint64_t g = (ct.base + ((uint64_t)t << ct.lo)) / 32;
+            const uint4 p = philox_stream(seed, 0u, g >> 2);
+            const uint32_t w = (uint32_t)g & 3u;
+            s_sign[t] = w == 0 ? p.x : w == 1 ? p.y : w == 2 ? p.z : p.w;
         }
     }
 }
@@ -205,85 +230,113 @@ __device__ __forceinline__ uint32_t col_sign_nibble(const uint32_t* s_sign, int 
 {
     constexpr int LCQ = 11 - LR;
     const int r = q >> LCQ, cq = q & ((1 << LCQ) - 1);
-    const uint32_t w = s_sign[(r << (LCQ - 3)) + (cq >> 3)];
+    const uint32_t w = s_sign[(LCQ >= 3 ? (r << (LCQ - 3)) : r) + (cq >> 3)];
     return (w >> ((cq & 7) * 4)) & 0xFu;
 }
 
+// ---------------------------------------------------------------------------------
+// Cluster stage of a column pass.  In: the block's tile in arrangement ARR.  Out: the
+// "slice" arrangement: register float4 k holds float4 q = slice_q(rank, t, k) of the tile
+// of cluster rank k >> (3 - LC); the LC stages across the ranks are done.  If s_sign is
+// given, nib[k] receives the sign nibble of that float4 from its owner's sign words.
+// ---------------------------------------------------------------------------------
+template <int LC>
+__device__ __forceinline__ int slice_q(int rank, int t, int k)
+{
+    return rank * (2048 >> LC) + t + 256 * (k & ((8 >> LC) - 1));
+}
+
+template <int LR, int LC, int ARR, bool SIGNS>
+__device__ __forceinline__ void col_cluster_stage(u64 (&v)[16], ulonglong2* s, const uint32_t* s_sign,
+                                                  uint32_t (&nib)[8], int rank)
+{
+    cg::cluster_group cluster = cg::this_cluster();
+    const int t = threadIdx.x;
+    __syncthreads();                                   // earlier readers of s are done
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s[col_swz(col_q<ARR>(t, k))] = make_ulonglong2(v[2 * k], v[2 * k + 1]);
+    cluster.sync();                                    // every tile of the cluster is in shared memory
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int owner = k >> (3 - LC);
+        const int q = slice_q<LC>(rank, t, k);
+        const ulonglong2* rs = cluster.map_shared_rank(s, owner);
+        const ulonglong2 w = rs[col_swz(q)];
+        v[2 * k] = w.x;
+        v[2 * k + 1] = w.y;
+        if (SIGNS) nib[k] = col_sign_nibble<LR>(cluster.map_shared_rank(s_sign, owner), q);
+    }
+    cluster.sync();                                    // owners may now reuse their shared memory
+    col_step<LC>(v);                                   // the LC stages across the tiles
+}
+
 // =================================================================================
-// Sender, first pass: x -> sign flip -> ||y||^2 -> LR top stages -> work
+// Sender, first pass: x -> sign flip -> ||y||^2 -> top stages -> work
+// Middle pass (SIGNED = false): work -> stages -> work, in place.
 // =================================================================================
-template <int LR>
+template <int LR, int LC, bool FIRST>
 __global__ void __launch_bounds__(kFastThreads, 3)
-k_f_enc_first(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo)
+k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo)
 {
     __shared__ ulonglong2 s[2048];
     __shared__ uint32_t s_sign[256];
     __shared__ double red[32];
     const ClientDesc cd = descs[blockIdx.y];
-    const ColTile ct = col_tile<LR>(blockIdx.x, lo);
+    const ColTile ct = col_tile<LR, LC>(blockIdx.x, lo);
     const int t = threadIdx.x;
-    col_sign_words<LR>(cd.seed, ct, s_sign);
+    const float* __restrict__ src = FIRST ? cd.src : cd.work;
+    if (FIRST) col_sign_words<LR>(cd.seed, ct, s_sign);
     u64 v[16];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const uint64_t i = col_index<LR>(ct, col_q<0>(t, k));
-        float4 x;
-        if (i + 3 < cd.valid) {
-            x = *reinterpret_cast<const float4*>(cd.src + i);
+        const uint64_t i = ct.base + col_offset<LR>(ct, col_q<0>(t, k));
+        if (!FIRST || i + 3 < cd.valid) {
+            const ulonglong2 w = *reinterpret_cast<const ulonglong2*>(src + i);
+            v[2 * k] = w.x;
+            v[2 * k + 1] = w.y;
         } else {
-            x.x = i < cd.valid ? cd.src[i] : 0.f;
-            x.y = i + 1 < cd.valid ? cd.src[i + 1] : 0.f;
-            x.z = i + 2 < cd.valid ? cd.src[i + 2] : 0.f;
-            x.w = 0.f;
+            const float x0 = i < cd.valid ? src[i] : 0.f;
+            const float x1 = i + 1 < cd.valid ? src[i + 1] : 0.f;
+            const float x2 = i + 2 < cd.valid ? src[i + 2] : 0.f;
+            v[2 * k] = pack2(x0, x1);
+            v[2 * k + 1] = pack2(x2, 0.f);
         }
-        v[2 * k] = pack2(x.x, x.y);
-        v[2 * k + 1] = pack2(x.z, x.w);
     }
     u64 acc = 0ull;
+    if (FIRST) {
 #pragma unroll
-    for (int k = 0; k < 16; ++k) acc = fma2(v[k], v[k], acc);
-    __syncthreads();                                   // sign words ready
+        for (int k = 0; k < 16; ++k) acc = fma2(v[k], v[k], acc);
+        __syncthreads();                               // sign words ready
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const uint32_t nib = col_sign_nibble<LR>(s_sign, col_q<0>(t, k));
-        v[2 * k] = flip2(v[2 * k], nib);
-        v[2 * k + 1] = flip2(v[2 * k + 1], nib >> 2);
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t nib = col_sign_nibble<LR>(s_sign, col_q<0>(t, k));
+            v[2 * k] = flip2(v[2 * k], nib);
+            v[2 * k + 1] = flip2(v[2 * k + 1], nib >> 2);
+        }
     }
     col_transform<LR>(v, s);
     constexpr int ARR = ColSteps<LR>::last;
+    if (LC == 0) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const uint64_t i = col_index<LR>(ct, col_q<ARR>(t, k));
-        *reinterpret_cast<ulonglong2*>(cd.work + i) = make_ulonglong2(v[2 * k], v[2 * k + 1]);
+        for (int k = 0; k < 8; ++k)
+            *reinterpret_cast<ulonglong2*>(cd.work + ct.base + col_offset<LR>(ct, col_q<ARR>(t, k))) =
+                make_ulonglong2(v[2 * k], v[2 * k + 1]);
+    } else {
+        uint32_t nib[8];
+        col_cluster_stage<LR, LC, ARR, false>(v, s, nullptr, nib, ct.rank);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint64_t i = ct.base0 + (uint64_t)(k >> (3 - LC)) * ct.rank_step +
+                               col_offset<LR>(ct, slice_q<LC>(ct.rank, t, k));
+            *reinterpret_cast<ulonglong2*>(cd.work + i) = make_ulonglong2(v[2 * k], v[2 * k + 1]);
+        }
     }
-    float a0, a1;
-    unpack2(acc, a0, a1);
-    const double tot = block_sum((double)a0 + (double)a1, red);
-    if (t == 0) atomicAdd(&states[blockIdx.y].norm2, tot);
-}
-
-// Middle pass, in place on the work buffer.
-template <int LR>
-__global__ void __launch_bounds__(kFastThreads, 3)
-k_f_mid(const ClientDesc* __restrict__ descs, int lo)
-{
-    __shared__ ulonglong2 s[2048];
-    const ClientDesc cd = descs[blockIdx.y];
-    const ColTile ct = col_tile<LR>(blockIdx.x, lo);
-    const int t = threadIdx.x;
-    u64 v[16];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const ulonglong2 w = *reinterpret_cast<const ulonglong2*>(cd.work + col_index<LR>(ct, col_q<0>(t, k)));
-        v[2 * k] = w.x;
-        v[2 * k + 1] = w.y;
+    if (FIRST) {
+        float a0, a1;
+        unpack2(acc, a0, a1);
+        const double tot = block_sum((double)a0 + (double)a1, red);
+        if (t == 0) atomicAdd(&states[blockIdx.y].norm2, tot);
     }
-    col_transform<LR>(v, s);
-    constexpr int ARR = ColSteps<LR>::last;
-#pragma unroll
-    for (int k = 0; k < 8; ++k)
-        *reinterpret_cast<ulonglong2*>(cd.work + col_index<LR>(ct, col_q<ARR>(t, k))) =
-            make_ulonglong2(v[2 * k], v[2 * k + 1]);
 }
 
 // =================================================================================
@@ -292,14 +345,14 @@ k_f_mid(const ClientDesc* __restrict__ descs, int lo)
 // 4.2).  mode: OUT_WRITE / OUT_ACC into out[0, d), or OUT_YHAT into the client's own work
 // buffer (b < 1, single client).
 // =================================================================================
-template <int LR>
+template <int LR, int LC>
 __global__ void __launch_bounds__(kFastThreads, 2)
 k_f_dec_last(const ClientDesc* __restrict__ descs, const ClientState* __restrict__ states,
              uint32_t n_group, int lo, float* __restrict__ out, uint64_t d, int mode)
 {
     __shared__ ulonglong2 s[2048];
     __shared__ uint32_t s_sign[256];
-    const ColTile ct = col_tile<LR>(blockIdx.x, lo);
+    const ColTile ct = col_tile<LR, LC>(blockIdx.x, lo);
     const int t = threadIdx.x;
     constexpr int ARR = ColSteps<LR>::last;
     u64 acc[16];
@@ -312,27 +365,36 @@ k_f_dec_last(const ClientDesc* __restrict__ descs, const ClientState* __restrict
         u64 v[16];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const ulonglong2 w = *reinterpret_cast<const ulonglong2*>(work + col_index<LR>(ct, col_q<0>(t, k)));
+            const ulonglong2 w =
+                *reinterpret_cast<const ulonglong2*>(work + ct.base + col_offset<LR>(ct, col_q<0>(t, k)));
             v[2 * k] = w.x;
             v[2 * k + 1] = w.y;
         }
         __syncthreads();                               // previous client's s / s_sign reads are done
         col_sign_words<LR>(seed, ct, s_sign);
         col_transform<LR>(v, s);
-        if (LR <= 3) __syncthreads();                  // no exchange inside: publish the sign words
+        uint32_t nib[8];
+        if (LC == 0) {
+            if (LR <= 3) __syncthreads();              // no exchange inside: publish the sign words
+#pragma unroll
+            for (int k = 0; k < 8; ++k) nib[k] = col_sign_nibble<LR>(s_sign, col_q<ARR>(t, k));
+        } else {
+            col_cluster_stage<LR, LC, ARR, true>(v, s, s_sign, nib, ct.rank);
+        }
         const u64 f2 = pack2(f, f);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const uint32_t nib = col_sign_nibble<LR>(s_sign, col_q<ARR>(t, k));
-            acc[2 * k] = fma2(flip2(v[2 * k], nib), f2, acc[2 * k]);
-            acc[2 * k + 1] = fma2(flip2(v[2 * k + 1], nib >> 2), f2, acc[2 * k + 1]);
+            acc[2 * k] = fma2(flip2(v[2 * k], nib[k]), f2, acc[2 * k]);
+            acc[2 * k + 1] = fma2(flip2(v[2 * k + 1], nib[k] >> 2), f2, acc[2 * k + 1]);
         }
     }
     const uint64_t limit = mode == OUT_YHAT ? (1ull << descs[0].L) : d;
     float* dst = mode == OUT_YHAT ? descs[0].work : out;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const uint64_t i = col_index<LR>(ct, col_q<ARR>(t, k));
+        const uint64_t i = LC == 0
+            ? ct.base + col_offset<LR>(ct, col_q<ARR>(t, k))
+            : ct.base0 + (uint64_t)(k >> (3 - LC)) * ct.rank_step + col_offset<LR>(ct, slice_q<LC>(ct.rank, t, k));
         float a[4];
         unpack2(acc[2 * k], a[0], a[1]);
         unpack2(acc[2 * k + 1], a[2], a[3]);
@@ -364,6 +426,9 @@ k_f_dec_last(const ClientDesc* __restrict__ descs, const ClientState* __restrict
 //                                owns the 32 consecutive coordinates 32 t .. 32 t + 31
 // Shared memory holds unit u at u + (u >> 4) (one pad per 16), conflict-free for the
 // 64-bit accesses of all three arrangements.
+// With a cluster (LC > 0) the 2^LC tiles of the cluster are consecutive in memory and the
+// LC index bits above the tile are exchanged in the "slice" arrangement: register k holds
+// unit rank * (4096 >> LC) + t + 256 * (k mod (16 >> LC)) of the tile of rank k / (16 >> LC).
 // ---------------------------------------------------------------------------------
 template <int ARR>
 __device__ __forceinline__ int row_u(int t, int k)
@@ -374,6 +439,12 @@ __device__ __forceinline__ int row_u(int t, int k)
 }
 __device__ __forceinline__ int row_pad(int u) { return u + (u >> 4); }
 constexpr int kRowSmemUnits = 4096 + 256;
+
+template <int LC>
+__device__ __forceinline__ int slice_u(int rank, int t, int k)
+{
+    return rank * (4096 >> LC) + t + 256 * (k & ((16 >> LC) - 1));
+}
 
 template <int FROM, int TO>
 __device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
@@ -386,11 +457,12 @@ __device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
     for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<TO>(t, k))];
 }
 
-// butterflies over the four register index bits of 16 packed units
+// butterflies over register index bits [B0, 4) of 16 packed units
+template <int B0>
 __device__ __forceinline__ void row_step(u64 (&v)[16])
 {
 #pragma unroll
-    for (int b = 0; b < 4; ++b)
+    for (int b = B0; b < 4; ++b)
 #pragma unroll
         for (int k = 0; k < 16; ++k)
             if (!(k & (1 << b))) bfly2(v[k], v[k | (1 << b)]);
@@ -402,7 +474,7 @@ __device__ __forceinline__ void row_step_inner(u64 (&v)[16])
 }
 
 // =================================================================================
-// Sender, last pass: work -> 13 low stages -> z = h/||y|| -> interval -> sum h Q(z) ->
+// Sender, last pass: work -> low stages -> z = h/||y|| -> interval -> sum h Q(z) ->
 // packed codes.  The thread ends with coordinates 32t..32t+31 of the tile and writes their
 // W code words itself.
 // =================================================================================
@@ -444,7 +516,7 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
     words[W - 1] = live ? ~neg_plane : 0u;
 }
 
-template <int W>
+template <int W, int LC>
 __global__ void __launch_bounds__(kFastThreads, 3)
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
 {
@@ -459,16 +531,41 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
         s_tv[j] = c_pos_value[table_offset(W) + j];
     }
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
-    const u64* __restrict__ src = reinterpret_cast<const u64*>(cd.work + base);
     u64 v[16];
+    if (LC == 0) {
+        const u64* __restrict__ src = reinterpret_cast<const u64*>(cd.work + base);
 #pragma unroll
-    for (int k = 0; k < 16; ++k) v[k] = src[row_u<0>(t, k)];
-    row_step(v);                    // e bits 12..9
+        for (int k = 0; k < 16; ++k) v[k] = src[row_u<0>(t, k)];
+    } else {
+        // fetch this block's slice of all tiles of the cluster, do the stages across the
+        // tiles, hand every result to the block that owns its tile
+        cg::cluster_group cluster = cg::this_cluster();
+        const int rank = (int)(blockIdx.x & ((1u << LC) - 1));
+        const uint64_t base0 = (uint64_t)(blockIdx.x >> LC) << (kFastTileLog + LC);
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int owner = k >> (4 - LC);
+            v[k] = reinterpret_cast<const u64*>(cd.work + base0 + ((uint64_t)owner << kFastTileLog))
+                       [slice_u<LC>(rank, t, k)];
+        }
+        row_step<4 - LC>(v);
+        cluster.sync();                                // every block of the cluster is running
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            u64* rs = cluster.map_shared_rank(s, k >> (4 - LC));
+            rs[row_pad(slice_u<LC>(rank, t, k))] = v[k];
+        }
+        cluster.sync();                                // the block's own tile is complete
+#pragma unroll
+        for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<0>(t, k))];
+        __syncthreads();                               // s is rewritten by the next exchange
+    }
+    row_step<0>(v);                 // e bits 12..9
     row_exchange<0, 1>(v, s);
-    row_step(v);                    // e bits 8..5
+    row_step<0>(v);                 // e bits 8..5
     __syncthreads();
     row_exchange<1, 2>(v, s);
-    row_step(v);                    // e bits 4..1
+    row_step<0>(v);                 // e bits 4..1
     row_step_inner(v);              // e bit 0
     const double n2 = states[blockIdx.y].norm2;
     const bool live = n2 > 0.0 && n2 < INFINITY;
@@ -484,9 +581,9 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
 }
 
 // =================================================================================
-// Receiver, first pass: codes -> centroids (lost packets -> 0) -> 13 low stages -> work
+// Receiver, first pass: codes -> centroids (lost packets -> 0) -> low stages -> work
 // =================================================================================
-template <int W>
+template <int W, int LC>
 __global__ void __launch_bounds__(kFastThreads, 3)
 k_f_dec_first(const ClientDesc* __restrict__ descs)
 {
@@ -522,15 +619,38 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
         v[k] = pack2(q[0], q[1]);
     }
     row_step_inner(v);              // e bit 0
-    row_step(v);                    // e bits 4..1
+    row_step<0>(v);                 // e bits 4..1
     row_exchange<2, 1>(v, s);
-    row_step(v);                    // e bits 8..5
+    row_step<0>(v);                 // e bits 8..5
     __syncthreads();
     row_exchange<1, 0>(v, s);
-    row_step(v);                    // e bits 12..9
-    u64* dst = reinterpret_cast<u64*>(cd.work + base);
+    row_step<0>(v);                 // e bits 12..9
+    if (LC == 0) {
+        u64* dst = reinterpret_cast<u64*>(cd.work + base);
 #pragma unroll
-    for (int k = 0; k < 16; ++k) dst[row_u<0>(t, k)] = v[k];
+        for (int k = 0; k < 16; ++k) dst[row_u<0>(t, k)] = v[k];
+    } else {
+        cg::cluster_group cluster = cg::this_cluster();
+        const int rank = (int)(blockIdx.x & ((1u << LC) - 1));
+        const uint64_t base0 = (uint64_t)(blockIdx.x >> LC) << (kFastTileLog + LC);
+        __syncthreads();                               // readers of the last exchange are done
+#pragma unroll
+        for (int k = 0; k < 16; ++k) s[row_pad(row_u<0>(t, k))] = v[k];
+        cluster.sync();
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const u64* rs = cluster.map_shared_rank(s, k >> (4 - LC));
+            v[k] = rs[row_pad(slice_u<LC>(rank, t, k))];
+        }
+        cluster.sync();                                // nobody reads this block's tile any more
+        row_step<4 - LC>(v);                           // the LC stages across the tiles
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const int owner = k >> (4 - LC);
+            reinterpret_cast<u64*>(cd.work + base0 + ((uint64_t)owner << kFastTileLog))
+                [slice_u<LC>(rank, t, k)] = v[k];
+        }
+    }
 }
 
 }  // namespace eden

@@ -135,7 +135,7 @@ def test_cfg5_padding_four_bits_loss_reduced(E):
 
 # ----------------------------------------------------------------------------- shapes and edge cases
 @pytest.mark.parametrize("d", [1, 2, 5, 31, 32, 33, 100, 1023, 1024, 1025, 4097, 8192, 8193,
-                               16384, 20000, 65536, 100000, 1 << 18, 1 << 19, (1 << 21) + 7,
+                               16384, 20000, 65536, 100000, 1 << 18, 1 << 19, 1 << 21, (1 << 21) + 7,
                                (1 << 23) + 5])
 @pytest.mark.parametrize("bits", [1.0, 3.0])
 def test_shapes_and_ragged_tails(E, d, bits):
@@ -145,6 +145,22 @@ def test_shapes_and_ragged_tails(E, d, bits):
     seeds = synth.client_seeds(d, n)
     work = synth.Workload("adhoc", n, d, np.full(n, bits), seeds, 0.0, lambda c: xs[c], d)
     run_workload(E, work)
+
+
+@pytest.mark.parametrize("variant", ["0", "1", "2"])
+def test_cluster_plans_at_2_pow_24_and_25(E, variant, monkeypatch):
+    # 2^24 can put the 8-block cluster stage on the column pass, on the row pass or on
+    # both; 2^25 needs both.  All plans must give the same answers.
+    monkeypatch.setenv("EDEN_PLAN_VARIANT", variant)
+    for d, bits in (((1 << 24) - 3, 2.0), (1 << 25, 1.0)):
+        if variant != "0" and d == 1 << 25:
+            continue
+        rng = np.random.default_rng(d % 1000)
+        n = 2
+        xs = rng.standard_normal((n, d)).astype(np.float32)
+        work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(d % 77, n), 0.05,
+                              lambda c: xs[c], d % 77)
+        run_workload(E, work)
 
 
 @pytest.mark.parametrize("W", [1, 2, 3, 4, 5, 6, 7, 8])
