@@ -30,11 +30,11 @@
  *     key = seed, counter = (t, 0, stream, 0): stream 0 call t gives the 128 sign bits
  *     of coordinates 128t..128t+127 (word (i/32)%4, bit i%32, 1 = minus); stream 1
  *     call t gives the 32-bit mask keys of input coordinates 4t..4t+3.
- *   - Message layout: coordinates in groups of 32; 32-bit word g*W + j holds bit j of
- *     the codes of coordinates 32g..32g+31 (bit l = coordinate 32g + l), W the code
- *     width.  A code is the rank of its quantisation value in ascending order.  A
- *     packet is 1024 consecutive rotated coordinates = 128*W bytes.  The scale S
- *     travels beside the codes as one fp32.
+ *   - Message layout: the codes form one little-endian bit stream of W-bit fields (W the
+ *     code width): coordinate i occupies stream bits [i*W, i*W + W), low bit of the code
+ *     first; stream bit b is bit b%32 of 32-bit word b/32.  A code is the rank of its
+ *     quantisation value in ascending order.  A packet is 1024 consecutive rotated
+ *     coordinates = 128*W bytes.  The scale S travels beside the codes as one fp32.
  */
 #ifndef EDEN_H_
 #define EDEN_H_
@@ -81,7 +81,7 @@ uint64_t eden_kept_count(uint64_t d, double bits);
 uint64_t eden_rot_dim(uint64_t d, double bits);
 /* W = 1 for bits <= 1, else (int)bits; 0 if the budget is unsupported (Section 3). */
 uint32_t eden_code_width(double bits);
-/* bytes of one client's packed codes: D*W/8 rounded up to a multiple of 16
+/* bytes of one client's packed codes: ceil(D*W/32) words rounded up to a multiple of 16 bytes
  * (Section 2.2.1: ceil(log2 |I|) * d bits). */
 uint64_t eden_code_bytes(uint64_t d, double bits);
 /* ceil(D / 1024): packets of one client's message (Section 4.2). */

@@ -104,7 +104,7 @@ def num_packets(D: int) -> int:
 
 
 def code_words(d: int, bits: float) -> int:
-    return ((rot_dim(d, bits) + 31) // 32) * code_width(bits)
+    return (rot_dim(d, bits) * code_width(bits) + 31) // 32
 
 
 # --------------------------------------------------------------------------- RNG

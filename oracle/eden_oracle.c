@@ -34,9 +34,9 @@
  *   - An endpoint belongs to the interval nearer zero (Section 2.2.1, footnote);
  *     z = +-0 goes to the non-negative side.                         [tie at 0 unpinned]
  *   - Code of a coordinate = rank of its centroid in ascending order.
- *   - Wire layout: coordinates in groups of 32; word g*W + j holds bit j of the
- *     codes of coordinates 32g..32g+31 (bit l of the word = coordinate 32g+l).
- *                                                                    [layout unpinned]
+ *   - Wire layout: the codes form one little-endian bit stream of W-bit fields,
+ *     coordinate i in stream bits [i*W, i*W + W) (bit b of the stream = bit b%32
+ *     of 32-bit word b/32), low bit of the code first.                [layout unpinned]
  *   - A packet is 1024 consecutive rotated coordinates.
  *   - The interval decision is taken after rounding z and the boundary to fp32,
  *     the precision the GPU kernels decide in; everything else is double.
@@ -310,7 +310,7 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
     uint64_t k = eden_oracle_kept_count(d, bits);
     uint64_t D = eden_oracle_rot_dim(d, bits);
     uint32_t W = eden_oracle_code_width(bits);
-    uint64_t n_words = ((D + 31u) / 32u) * W; /* W words per group of 32 coordinates */
+    uint64_t n_words = (D * W + 31u) / 32u;
 
     double *y = (double *)calloc(D, sizeof(double));
     if (!y) return -1;
@@ -356,10 +356,10 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
         double z = eta * y[i];
         uint32_t code = eden_oracle_quantise(z, W);
         dot += y[i] * eden_oracle_value(code, W);
-        uint64_t g = i / 32u;
-        uint32_t l = (uint32_t)(i % 32u);
-        for (uint32_t j = 0; j < W; ++j)
-            codes[g * W + j] |= ((code >> j) & 1u) << l;
+        for (uint32_t j = 0; j < W; ++j) {           /* field i of the bit stream */
+            uint64_t b = i * W + j;
+            codes[b / 32u] |= ((code >> j) & 1u) << (b % 32u);
+        }
         if (z_out) z_out[i] = z;
     }
     *scale_out = N2 / dot;
@@ -396,11 +396,11 @@ int eden_oracle_decode(const uint32_t *codes, double S, double bits, uint64_t se
         int arrived = recv_mask ? (int)((recv_mask[pkt / 32u] >> (pkt % 32u)) & 1u) : 1;
         if (!arrived) continue; /* lost coordinate counts as 0 */
         ++received;
-        uint64_t g = i / 32u;
-        uint32_t l = (uint32_t)(i % 32u);
         uint32_t code = 0;
-        for (uint32_t j = 0; j < W; ++j)
-            code |= ((codes[g * W + j] >> l) & 1u) << j;
+        for (uint32_t j = 0; j < W; ++j) {
+            uint64_t b = i * W + j;
+            code |= ((codes[b / 32u] >> (b % 32u)) & 1u) << j;
+        }
         q[i] = eden_oracle_value(code, W);
     }
     if (received == 0) { free(q); return 1; }

@@ -53,7 +53,7 @@ extern "C" uint32_t eden_code_width(double bits)
 extern "C" uint64_t eden_code_bytes(uint64_t d, double bits)
 {
     const uint64_t D = eden_rot_dim(d, bits);
-    const uint64_t bytes = ((D + 31) / 32) * eden_code_width(bits) * 4;
+    const uint64_t bytes = ((D * eden_code_width(bits) + 31) / 32) * 4;
     return (bytes + 15) / 16 * 16;
 }
 
@@ -478,7 +478,8 @@ PassGeom row_geom(int lc) { return PassGeom{lc, lc, lc, 0}; }
 
 // Plan of the register-blocked path.  The row pass covers index bits [0, 13 + row_lc);
 // each column pass covers bits [lo, lo + lr + lc), lr of them inside a block and lc (0 or
-// 3) across the 8 blocks of a cluster.  Two sweeps over HBM up to 2^27 coordinates.
+// 3) across the 8 blocks of a cluster.  variant 0 (the default) uses no clusters; 1..3 are
+// the cluster plans (two sweeps over HBM up to 2^27 coordinates), kept for tuning.
 struct FastPass { int lo, lr, lc; };
 struct FastPlan { int row_lc; std::vector<FastPass> cols; };   // cols: top range first
 
@@ -486,26 +487,35 @@ FastPlan fast_plan(int L, int variant)
 {
     FastPlan pl;
     const int cb = L - kFastTileLog;
+    if (variant == 0 || cb <= kFastMaxColBits) {
+        // No clusters: column passes of at most 7 bits each (8-bit passes are slower per
+        // byte), split evenly, top range first.  Measured on B200 this beats every
+        // cluster plan below: one more sweep over HBM costs less than the per-tile
+        // cluster barriers.
+        const int per = cb <= kFastMaxColBits ? kFastMaxColBits : 7;
+        pl.row_lc = 0;
+        const int passes = (cb + per - 1) / per;
+        int hi = L;
+        for (int p = 0; p < passes; ++p) {
+            const int bits = (hi - kFastTileLog + (passes - p) - 1) / (passes - p);
+            pl.cols.push_back(FastPass{hi - bits, bits, 0});
+            hi -= bits;
+        }
+        return pl;
+    }
     auto one = [](int lo, int bits) {
         return bits > kFastMaxColBits ? FastPass{lo, bits - kFastClusterLog, kFastClusterLog}
                                       : FastPass{lo, bits, 0};
     };
-    if (cb <= kFastMaxColBits) {
-        pl.row_lc = 0;
-        pl.cols.push_back(FastPass{kFastTileLog, cb, 0});
-    } else if (cb <= kFastMaxColBits + kFastClusterLog) {
-        if (variant == 1) {            // cluster on the row pass instead of the column pass
-            pl.row_lc = kFastClusterLog;
-            pl.cols.push_back(FastPass{kFastTileLog + kFastClusterLog, cb - kFastClusterLog, 0});
-        } else if (variant == 2 && cb - 2 * kFastClusterLog >= 1) {   // clusters on both
-            pl.row_lc = kFastClusterLog;
-            pl.cols.push_back(FastPass{kFastTileLog + kFastClusterLog, cb - 2 * kFastClusterLog,
-                                       kFastClusterLog});
-        } else {
+    if (cb <= kFastMaxColBits + kFastClusterLog && variant != 3) {
+        if (variant == 1) {            // cluster on the column pass
             pl.row_lc = 0;
             pl.cols.push_back(FastPass{kFastTileLog, cb - kFastClusterLog, kFastClusterLog});
+        } else {                       // variant 2: cluster on the row pass
+            pl.row_lc = kFastClusterLog;
+            pl.cols.push_back(FastPass{kFastTileLog + kFastClusterLog, cb - kFastClusterLog, 0});
         }
-    } else {
+    } else {                           // clusters on both (variant 3, or more than 11 bits)
         pl.row_lc = kFastClusterLog;
         const int low = kFastTileLog + kFastClusterLog;
         const int rest = L - low;

@@ -34,6 +34,26 @@ constexpr int kFastClusterLog = 3;     // a cluster of 8 blocks adds three more 
 
 namespace cg = cooperative_groups;
 
+// Cluster barrier that publishes this block's shared-memory writes to the other blocks
+// of the cluster: the block-wide barrier orders every thread's writes before thread 0,
+// whose cluster-scope fence and (relaxed) arrival form the release; every thread's wait
+// acquires.  One fence per block instead of one per thread.
+__device__ __forceinline__ void cluster_sync_publish()
+{
+    __syncthreads();
+    if (threadIdx.x == 0) asm volatile("fence.acq_rel.cluster;" ::: "memory");
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Cluster barrier that only orders execution: callers use it after they have consumed
+// every value they read from other blocks' shared memory, to tell the owners that the
+// memory may be overwritten.
+__device__ __forceinline__ void cluster_sync_execution()
+{
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+}
+
 typedef unsigned long long u64;
 
 // ---------------------------------------------------------------------------------
@@ -255,7 +275,7 @@ __device__ __forceinline__ void col_cluster_stage(u64 (&v)[16], ulonglong2* s, c
     __syncthreads();                                   // earlier readers of s are done
 #pragma unroll
     for (int k = 0; k < 8; ++k) s[col_swz(col_q<ARR>(t, k))] = make_ulonglong2(v[2 * k], v[2 * k + 1]);
-    cluster.sync();                                    // every tile of the cluster is in shared memory
+    cluster_sync_publish();                            // every tile of the cluster is in shared memory
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         const int owner = k >> (3 - LC);
@@ -266,8 +286,14 @@ __device__ __forceinline__ void col_cluster_stage(u64 (&v)[16], ulonglong2* s, c
         v[2 * k + 1] = w.y;
         if (SIGNS) nib[k] = col_sign_nibble<LR>(cluster.map_shared_rank(s_sign, owner), q);
     }
-    cluster.sync();                                    // owners may now reuse their shared memory
-    col_step<LC>(v);                                   // the LC stages across the tiles
+    col_step<LC>(v);                                   // the LC stages across the tiles (consumes the fetched values)
+    if (SIGNS) {
+        uint32_t any = 0u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) any |= nib[k];
+        asm volatile("" :: "r"(any));                  // the sign nibbles have arrived as well
+    }
+    cluster_sync_execution();                          // owners may now reuse their shared memory
 }
 
 // =================================================================================
@@ -478,16 +504,47 @@ __device__ __forceinline__ void row_step_inner(u64 (&v)[16])
 // packed codes.  The thread ends with coordinates 32t..32t+31 of the tile and writes their
 // W code words itself.
 // =================================================================================
+// Magnitude index of |z| in the 2^(W-1) positive intervals (Section 2.2.1): the number of
+// positive boundaries strictly below |z|.  Up to four bits the boundaries are
+// compile-time-indexed constants and the search is a tree of selects; wider tables are
+// searched in shared memory.
+template <int W>
+__device__ __forceinline__ int fast_magnitude(float az, const float* s_tb)
+{
+    constexpr int off = (1 << (W - 1)) - 1;
+    if (W == 1) return 0;
+    if (W == 2) return az > c_pos_boundary[off] ? 1 : 0;
+    if (W == 3) {
+        const bool b1 = az > c_pos_boundary[off + 1];
+        const float t0 = b1 ? c_pos_boundary[off + 2] : c_pos_boundary[off + 0];
+        return (b1 ? 2 : 0) + (az > t0 ? 1 : 0);
+    }
+    if (W == 4) {
+        const bool b2 = az > c_pos_boundary[off + 3];
+        const float t1 = b2 ? c_pos_boundary[off + 5] : c_pos_boundary[off + 1];
+        const bool b1 = az > t1;
+        const float lo = b1 ? c_pos_boundary[off + 2] : c_pos_boundary[off + 0];
+        const float hi = b1 ? c_pos_boundary[off + 6] : c_pos_boundary[off + 4];
+        const float t0 = b2 ? hi : lo;
+        return (b2 ? 4 : 0) + (b1 ? 2 : 0) + (az > t0 ? 1 : 0);
+    }
+    int m = 0;
+#pragma unroll
+    for (int step = (1 << (W - 1)) >> 1; step >= 1; step >>= 1)
+        m += (az > s_tb[m + step - 1]) ? step : 0;
+    return m;
+}
+
+// The thread's 32 consecutive coordinates -> their W words of the code bit stream
+// (coordinate l in bits [l*W, l*W + W) of the 32*W-bit group), and sum |h| Q(|z|).
 template <int W>
 __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_norm, bool live,
                                                  const float* s_tb, const float* s_tv,
                                                  uint32_t (&words)[W], float& dot)
 {
-    constexpr int half = 1 << (W - 1);
-    uint32_t neg_plane = 0u;
-    uint32_t mag[W > 1 ? W - 1 : 1];
+    constexpr uint32_t half = 1u << (W - 1);
 #pragma unroll
-    for (int j = 0; j < (W > 1 ? W - 1 : 1); ++j) mag[j] = 0u;
+    for (int j = 0; j < W; ++j) words[j] = 0u;
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
         float h[2];
@@ -496,24 +553,19 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
         for (int e = 0; e < 2; ++e) {
             const int l = 2 * k + e;
             const float z = h[e] * inv_norm;
-            const float az = fabsf(z);
-            int m = 0;
-            if (W > 1) {
-#pragma unroll
-                for (int step = half >> 1; step >= 1; step >>= 1)
-                    m += (az > s_tb[m + step - 1]) ? step : 0;
-            }
-            dot = fmaf(fabsf(h[e]), s_tv[m], dot);
-            neg_plane |= (z < 0.f ? 1u : 0u) << l;
-#pragma unroll
-            for (int j = 0; j + 1 < W; ++j) mag[j] |= (((uint32_t)m >> j) & 1u) << l;
+            const int m = fast_magnitude<W>(fabsf(z), s_tb);
+            dot = fmaf(fabsf(h[e]), W <= 2 ? (m ? c_pos_value[half] : c_pos_value[half - 1]) : s_tv[m], dot);
+            // code = half + m for z >= 0 and half - 1 - m otherwise
+            const uint32_t code = (uint32_t)m ^ (z < 0.f ? half - 1u : half);
+            const int a = (l * W) >> 5, off = (l * W) & 31;
+            words[a] |= code << off;
+            if (off + W > 32) words[a + 1] |= code >> (32 - off);
         }
     }
-    // code = half + m for z >= 0, half - 1 - m otherwise: the low planes of a negative
-    // coordinate are the complement of m's bits, the top plane is "not negative"
+    if (!live) {
 #pragma unroll
-    for (int j = 0; j + 1 < W; ++j) words[j] = live ? (mag[j] ^ neg_plane) : 0u;
-    words[W - 1] = live ? ~neg_plane : 0u;
+        for (int j = 0; j < W; ++j) words[j] = 0u;
+    }
 }
 
 template <int W, int LC>
@@ -549,13 +601,13 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
                        [slice_u<LC>(rank, t, k)];
         }
         row_step<4 - LC>(v);
-        cluster.sync();                                // every block of the cluster is running
+        cluster_sync_execution();                      // every block of the cluster is running
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             u64* rs = cluster.map_shared_rank(s, k >> (4 - LC));
             rs[row_pad(slice_u<LC>(rank, t, k))] = v[k];
         }
-        cluster.sync();                                // the block's own tile is complete
+        cluster_sync_publish();                        // the block's own tile is complete
 #pragma unroll
         for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<0>(t, k))];
         __syncthreads();                               // s is rewritten by the next exchange
@@ -588,20 +640,27 @@ __global__ void __launch_bounds__(kFastThreads, 3)
 k_f_dec_first(const ClientDesc* __restrict__ descs)
 {
     __shared__ u64 s[kRowSmemUnits];
-    __shared__ float s_tv[128];
+    __shared__ float s_val[2 << W];                    // the 2^W values by code, then 2^W zeros
     const ClientDesc cd = descs[blockIdx.y];
     const int t = threadIdx.x;
     constexpr int half = 1 << (W - 1);
-    for (int j = t; j < half; j += kFastThreads) s_tv[j] = c_pos_value[table_offset(W) + j];
+    for (int j = t; j < (2 << W); j += kFastThreads) {
+        float c = 0.f;
+        if (j < (1 << W)) c = j >= half ? c_pos_value[table_offset(W) + j - half]
+                                         : -c_pos_value[table_offset(W) + half - 1 - j];
+        s_val[j] = c;
+    }
     __syncthreads();
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
-    // the tile is 8 packets of 1024 coordinates; this thread's 32 coordinates lie in one
+    // the tile is 8 packets of 1024 coordinates; this thread's 32 coordinates lie in one.
+    // A lost packet reads the zero half of the table (Section 4.2: lost coordinates are 0).
     const uint64_t pkt = (base >> 10) + (uint64_t)(t >> 5);
     const bool arrived = cd.recv ? ((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u) != 0u : true;
+    const float* tbl = s_val + (arrived ? 0 : (1 << W));
     uint32_t words[W];
     const uint32_t* src = cd.codes + ((base >> 5) + t) * W;
 #pragma unroll
-    for (int j = 0; j < W; ++j) words[j] = arrived ? src[j] : 0u;
+    for (int j = 0; j < W; ++j) words[j] = src[j];
     u64 v[16];
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
@@ -609,12 +668,10 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
             const int l = 2 * k + e;
-            uint32_t code = 0u;
-#pragma unroll
-            for (int j = 0; j < W; ++j) code |= ((words[j] >> l) & 1u) << j;
-            const bool pos = code >= (uint32_t)half;
-            const float c = s_tv[pos ? code - half : half - 1 - code];
-            q[e] = arrived ? (pos ? c : -c) : 0.f;
+            const int a = (l * W) >> 5, off = (l * W) & 31;
+            uint32_t code = words[a] >> off;
+            if (off + W > 32) code |= words[a + 1] << (32 - off);
+            q[e] = tbl[code & ((1u << W) - 1u)];
         }
         v[k] = pack2(q[0], q[1]);
     }
@@ -636,14 +693,14 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
         __syncthreads();                               // readers of the last exchange are done
 #pragma unroll
         for (int k = 0; k < 16; ++k) s[row_pad(row_u<0>(t, k))] = v[k];
-        cluster.sync();
+        cluster_sync_publish();
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const u64* rs = cluster.map_shared_rank(s, k >> (4 - LC));
             v[k] = rs[row_pad(slice_u<LC>(rank, t, k))];
         }
-        cluster.sync();                                // nobody reads this block's tile any more
-        row_step<4 - LC>(v);                           // the LC stages across the tiles
+        row_step<4 - LC>(v);                           // the LC stages across the tiles (consumes the fetched values)
+        cluster_sync_execution();                      // nobody reads this block's tile any more
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const int owner = k >> (4 - LC);

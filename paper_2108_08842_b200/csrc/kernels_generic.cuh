@@ -138,7 +138,7 @@ k_mid(const ClientDesc* __restrict__ descs, PassGeom g)
 // Last pass of the encode (a row pass over the low bits): finishes the transform,
 // normalises (z = h / ||y||, i.e. eta_x R(x) of Section 2.2.1), finds each coordinate's
 // interval, accumulates sum h_i Q(z_i) for the scale (Section 2.3) and writes the packed
-// codes, one ballot per bit-plane.  SINGLE: the whole vector is one tile, so this kernel
+// codes (a bit stream of W-bit fields, assembled with warp-wide OR reductions).  SINGLE: the whole vector is one tile, so this kernel
 // also loads the input, flips the signs and computes the norm.
 template <bool SINGLE>
 __global__ void __launch_bounds__(kGenericThreads)
@@ -179,7 +179,8 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
     const int lane = threadIdx.x & 31;
     float dot = 0.f;
-    const int Tr = (T + 31) & ~31;                     // whole warps take part in the ballots
+    const int Tr = (T + 31) & ~31;                     // whole warps take part in the reductions
+    const uint64_t total_words = (((uint64_t)1 << cd.L) * W + 31) >> 5;
     for (int e = threadIdx.x; e < Tr; e += blockDim.x) {
         const float h = e < T ? s[e] : 0.f;
         const float z = h * inv_norm;
@@ -189,12 +190,18 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
         const float q = neg ? -s_tv[m] : s_tv[m];
         if (e < T) dot = fmaf(h, q, dot); else code = 0u;
         if (!live) code = 0u;
+        // the 32 lanes hold 32 consecutive W-bit fields = W words of the bit stream:
+        // lane l's field starts at bit l*W of the group
         uint32_t mine = 0u;
         for (int j = 0; j < W; ++j) {
-            const uint32_t word = __ballot_sync(0xffffffffu, (code >> j) & 1u);
+            const int sh = lane * W - 32 * j;
+            uint32_t part = 0u;
+            if (sh > -W && sh < 32) part = sh >= 0 ? code << sh : code >> (-sh);
+            const uint32_t word = __reduce_or_sync(0xffffffffu, part);
             if (lane == j) mine = word;
         }
-        if (lane < W) cd.codes[((base + e) >> 5) * W + lane] = mine;
+        const uint64_t widx = ((base + e) >> 5) * W + lane;
+        if (lane < W && widx < total_words) cd.codes[widx] = mine;
     }
     const double tot = block_sum((double)dot, red);
     if (threadIdx.x == 0) {
@@ -272,9 +279,11 @@ __device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i
         if (!((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u)) return 0.f;
     }
     const int W = (int)cd.W, half = 1 << (W - 1);
-    const uint32_t* wp = cd.codes + (i >> 5) * W;
-    uint32_t code = 0;
-    for (int j = 0; j < W; ++j) code |= ((wp[j] >> (i & 31)) & 1u) << j;
+    const uint64_t bit = i * W;                        // field i of the bit stream
+    const uint32_t off = (uint32_t)(bit & 31);
+    uint32_t code = cd.codes[bit >> 5] >> off;
+    if (off + W > 32) code |= cd.codes[(bit >> 5) + 1] << (32 - off);
+    code &= (1u << W) - 1u;
     return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
 }
 

@@ -7,14 +7,11 @@ import oracle as O
 
 
 def unpack_codes(words: np.ndarray, D: int, W: int) -> np.ndarray:
-    """Per-coordinate codes from the packed wire layout (word g*W + j = bit-plane j of group g)."""
-    groups = (D + 31) // 32
-    w = words[: groups * W].reshape(groups, W)
-    shifts = np.arange(32, dtype=np.uint32)
-    codes = np.zeros((groups, 32), dtype=np.uint32)
-    for j in range(W):
-        codes |= ((w[:, j:j + 1] >> shifts) & 1) << np.uint32(j)
-    return codes.reshape(-1)[:D]
+    """Per-coordinate codes from the wire layout: a little-endian bit stream of W-bit fields."""
+    nw = (D * W + 31) // 32
+    bits = ((words[:nw, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(-1)[: D * W]
+    weights = (np.uint32(1) << np.arange(W, dtype=np.uint32))
+    return (bits.reshape(D, W).astype(np.uint32) * weights).sum(axis=1).astype(np.uint32)
 
 
 def near_boundary(z: np.ndarray, W: int) -> np.ndarray:

@@ -147,13 +147,14 @@ def test_shapes_and_ragged_tails(E, d, bits):
     run_workload(E, work)
 
 
-@pytest.mark.parametrize("variant", ["0", "1", "2"])
-def test_cluster_plans_at_2_pow_24_and_25(E, variant, monkeypatch):
-    # 2^24 can put the 8-block cluster stage on the column pass, on the row pass or on
-    # both; 2^25 needs both.  All plans must give the same answers.
+@pytest.mark.parametrize("variant", ["0", "1", "2", "3"])
+def test_pass_plans_at_2_pow_24_and_25(E, variant, monkeypatch):
+    # plan 0 (default) sweeps three times without clusters; plans 1-3 put an 8-block
+    # cluster stage on the column pass, on the row pass or on both (2^25 always needs
+    # both).  All plans must give the same answers.
     monkeypatch.setenv("EDEN_PLAN_VARIANT", variant)
     for d, bits in (((1 << 24) - 3, 2.0), (1 << 25, 1.0)):
-        if variant != "0" and d == 1 << 25:
+        if variant in ("2", "3") and d == 1 << 25:
             continue
         rng = np.random.default_rng(d % 1000)
         n = 2

@@ -198,9 +198,9 @@ def _dense_reference(x, bits, seed):
 def _unpack(words, D, W):
     codes = np.zeros(D, dtype=np.int64)
     for i in range(D):
-        g, l = divmod(i, 32)
         for j in range(W):
-            codes[i] |= ((int(words[g * W + j]) >> l) & 1) << j
+            b = i * W + j
+            codes[i] |= ((int(words[b // 32]) >> (b % 32)) & 1) << j
     return codes
 
 
@@ -212,7 +212,7 @@ def test_encode_decode_against_dense_reference(d, bits):
     codes_ref, S_ref, xhat_ref, r, _ = _dense_reference(x.astype(np.float64), bits, seed)
     enc = O.encode(x, bits, seed, want_z=True)
     D, W = O.rot_dim(d, bits), O.code_width(bits)
-    assert len(enc["codes"]) == (D + 31) // 32 * W
+    assert len(enc["codes"]) == (D * W + 31) // 32
     assert np.array_equal(_unpack(enc["codes"], D, W), codes_ref)
     assert abs(enc["scale"] - S_ref) < 1e-10 * abs(S_ref)
     xhat, nodata = O.decode(enc["codes"], enc["scale"], bits, seed, d)
@@ -230,17 +230,22 @@ def test_encode_decode_against_dense_reference(d, bits):
 
 
 def test_wire_layout_by_hand():
-    # 64 coordinates, W = 2: word g*2 + j, bit l = bit j of the code of coordinate 32 g + l
-    d, bits, seed = 64, 2, 77
+    # W-bit fields, low bit first, packed into little-endian 32-bit words; 3-bit fields
+    # straddle word boundaries (coordinate 10 occupies stream bits 30..32)
+    d, bits, seed = 64, 3, 77
     x = np.random.default_rng(5).standard_normal(d).astype(np.float32)
     enc = O.encode(x, bits, seed, want_z=True)
-    codes = [O.quantise(z, 2) for z in enc["z"]]
-    for g in range(2):
-        for j in range(2):
-            w = 0
-            for l in range(32):
-                w |= ((codes[32 * g + l] >> j) & 1) << l
-            assert int(enc["codes"][g * 2 + j]) == w
+    codes = [O.quantise(z, 3) for z in enc["z"]]
+    stream = 0
+    for i, c in enumerate(codes):
+        stream |= c << (3 * i)
+    assert len(enc["codes"]) == 6
+    for w in range(6):
+        assert int(enc["codes"][w]) == (stream >> (32 * w)) & 0xFFFFFFFF
+    # one-bit codes: bit i of the stream is "coordinate i is non-negative"
+    e1 = O.encode(x, 1, seed, want_z=True)
+    for i in range(d):
+        assert (int(e1["codes"][i // 32]) >> (i % 32)) & 1 == (1 if e1["z"][i] >= 0 else 0)
 
 
 def test_zero_padding_equals_explicit_padding():
