@@ -94,8 +94,11 @@ __device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c)
 // flips the sign of each half where the matching bit of `bits` (bit 0 -> lo, bit 1 -> hi) is set
 __device__ __forceinline__ u64 flip2(u64 v, uint32_t bits)
 {
-    const u64 m = ((u64)(bits & 1u) << 31) | ((u64)(bits & 2u) << 62);
-    return v ^ m;
+    float lo, hi;
+    unpack2(v, lo, hi);
+    lo = __uint_as_float(__float_as_uint(lo) ^ (bits << 31));
+    hi = __uint_as_float(__float_as_uint(hi) ^ ((bits << 30) & 0x80000000u));
+    return pack2(lo, hi);
 }
 
 // Butterflies over the register index bits [0, NB) of 8 float4 values (as 16 packed pairs:
@@ -301,7 +304,7 @@ __device__ __forceinline__ void col_cluster_stage(u64 (&v)[16], ulonglong2* s, c
 // Middle pass (SIGNED = false): work -> stages -> work, in place.
 // =================================================================================
 template <int LR, int LC, bool FIRST>
-__global__ void __launch_bounds__(kFastThreads, 3)
+__global__ void __launch_bounds__(kFastThreads, 4)
 k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo)
 {
     __shared__ ulonglong2 s[2048];
@@ -569,7 +572,7 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
 }
 
 template <int W, int LC>
-__global__ void __launch_bounds__(kFastThreads, 3)
+__global__ void __launch_bounds__(kFastThreads, 4)
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
 {
     __shared__ u64 s[kRowSmemUnits];
@@ -636,7 +639,7 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
 // Receiver, first pass: codes -> centroids (lost packets -> 0) -> low stages -> work
 // =================================================================================
 template <int W, int LC>
-__global__ void __launch_bounds__(kFastThreads, 3)
+__global__ void __launch_bounds__(kFastThreads, 4)
 k_f_dec_first(const ClientDesc* __restrict__ descs)
 {
     __shared__ u64 s[kRowSmemUnits];
