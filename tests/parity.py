@@ -23,9 +23,12 @@ def near_boundary(z: np.ndarray, W: int) -> np.ndarray:
     return out
 
 
-def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, bits: float, seed: int):
-    """Returns (mismatching coordinates, all inside the boundary window?, scale rel. error, oracle result)."""
-    enc = O.encode(x, bits, seed, want_z=True)
+def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, bits: float, seed: int,
+                        enc=None):
+    """Returns (mismatching coordinates, all inside the boundary window?, scale rel. error, oracle result).
+    `enc` may carry a precomputed oracle result (without z); z is recomputed only on a mismatch."""
+    if enc is None:
+        enc = O.encode(x, bits, seed)
     d = x.shape[0]
     D, W = O.rot_dim(d, bits), O.code_width(bits)
     nw = len(enc["codes"])
@@ -33,11 +36,12 @@ def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, 
     mism = 0
     ok = True
     if diff.size:
+        z = O.encode(x, bits, seed, want_z=True)["z"]
         g = unpack_codes(gpu_words, D, W)
         o = unpack_codes(enc["codes"], D, W)
         bad = np.nonzero(g != o)[0]
         mism = int(bad.size)
-        ok = bool(np.all(near_boundary(enc["z"][bad], W)))
+        ok = bool(np.all(near_boundary(z[bad], W)))
         # a mismatch may only move the code to the neighbouring interval
         ok = ok and bool(np.all(np.abs(g[bad].astype(np.int64) - o[bad].astype(np.int64)) == 1))
     rel = abs(gpu_scale - enc["scale"]) / abs(enc["scale"]) if enc["scale"] != 0 else abs(gpu_scale)

@@ -1,0 +1,99 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration
+bench.py times (all clients of the configuration in one eden_encode / eden_mean call).
+
+The oracle checks every client where that takes seconds (configurations 3 and 4) and a
+sample of clients where one client alone takes the oracle tens of seconds
+(configuration 5); what is not compared coordinate by coordinate is checked through
+properties that hold at any size (NMSE of the mean against Lemma 2.2 / Lemma 4.3).
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2108_08842_b200 import synth
+from tests.test_gpu_parity import run_workload, MEAN_TOL, SCALE_TOL
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+THREADS = min(16, os.cpu_count() or 1)
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_2108_08842_b200 import eden
+    return eden
+
+
+def _nmse(mean, xs):
+    true = xs.astype(np.float64).mean(axis=0)
+    return float(np.sum((mean - true) ** 2) / (np.sum(xs.astype(np.float64) ** 2) / xs.shape[0]))
+
+
+def test_cfg3_full_size_heterogeneous_budgets(E):
+    work = synth.make("cfg3")
+    assert work.n == 32 and work.d == 1 << 23
+    mism, xs, mean = run_workload(E, work, threads=THREADS)
+    assert mism <= 60
+
+
+def test_cfg4_full_size_packet_loss(E):
+    work = synth.make("cfg4")
+    assert work.n == 64 and work.d == 1 << 24
+    mism, xs, mean = run_workload(E, work, threads=THREADS)
+    assert mism <= 120
+    # one bit, 10 % of the packets lost: vNMSE = 1/(p 2/pi) - 1 per client, NMSE = vNMSE/n
+    # weighted by the clients' norms (Lemma 2.2, Lemma 4.3); p is about 0.9 for every client
+    expect = (1 / (0.9 * 2 / np.pi) - 1) / work.n
+    assert abs(_nmse(mean, xs) - expect) < 0.05 * expect
+
+
+def test_cfg5_full_size_sampled_clients(E):
+    work = synth.make("cfg5")
+    n, d = work.n, work.d
+    assert n == 16 and d == 100_000_000
+    xs = np.empty((n, d), dtype=np.float32)
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(THREADS) as ex:
+        list(ex.map(lambda c: xs.__setitem__(c, work.vector(c)), range(n)))
+    ctx = E.Context(0, d_max=d, n_batch=n)
+    x_gpu = torch.from_numpy(xs).cuda()
+    codes, scales = ctx.encode(x_gpu, work.bits, work.seeds)
+    masks_np = [work.recv_mask(c, O.num_packets(O.rot_dim(d, 4.0))) for c in range(n)]
+    masks_t = [torch.from_numpy(m.view(np.int32)).cuda() for m in masks_np]
+    mean_all = ctx.mean(codes, scales, work.bits, work.seeds, d, masks_t).cpu().numpy()
+    assert ctx.status() == 0
+    scales_h = scales.cpu().numpy()
+
+    # sender: four sampled clients against the oracle, coordinate by coordinate
+    sample = [0, 5, 10, 15]
+    pre = O.encode_all([xs[c] for c in sample], [4.0] * 4, [int(work.seeds[c]) for c in sample], threads=4)
+    total = 0
+    for j, c in enumerate(sample):
+        mism, ok, rel, _ = parity.check_encode_client(codes[c].cpu().numpy().view(np.uint32),
+                                                      float(scales_h[c]), xs[c], 4.0, int(work.seeds[c]), pre[j])
+        assert ok and rel <= SCALE_TOL, (c, mism, rel)
+        total += mism
+    assert total <= 400
+
+    # receiver: the same four clients' oracle messages through eden_mean, all coordinates
+    o_scales = np.array([np.float32(e["scale"]) for e in pre], dtype=np.float32)
+    g_codes = [torch.from_numpy(e["codes"].view(np.uint8).copy()).cuda() for e in pre]
+    got = ctx.mean(g_codes, torch.from_numpy(o_scales).cuda(), [4.0] * 4, [int(work.seeds[c]) for c in sample],
+                   d, [masks_t[c] for c in sample]).cpu().numpy()
+    ref, used = O.mean([e["codes"] for e in pre], [float(s) for s in o_scales], [4.0] * 4,
+                       [int(work.seeds[c]) for c in sample], d, [masks_np[c] for c in sample], threads=4)
+    assert used == 4
+    assert np.max(np.abs(got - ref)) <= MEAN_TOL * np.max(np.abs(ref))
+
+    # all 16 clients: NMSE of the mean = vNMSE/n with vNMSE = (1/(p E[Q^2]) - 1) * d/D
+    c, b = O.table(4)
+    edges = np.concatenate(([-np.inf], b, [np.inf]))
+    from scipy.stats import norm
+    eq2 = float(np.sum((norm.cdf(edges[1:]) - norm.cdf(edges[:-1])) * c * c))
+    expect = (1 / (0.99 * eq2) - 1) * d / (1 << 27) / n
+    assert abs(_nmse(mean_all.astype(np.float64), xs) - expect) < 0.05 * expect
+    ctx.close()

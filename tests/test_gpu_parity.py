@@ -47,14 +47,16 @@ def run_workload(E, work, threads=8, check_clients=None):
     torch.cuda.synchronize()
     assert ctx.status() == 0
     scales_h = scales.cpu().numpy()
-    check_clients = range(n) if check_clients is None else check_clients
+    check_clients = list(range(n)) if check_clients is None else list(check_clients)
 
     total_mism = 0
     encs = {}
-    for c in check_clients:
+    pre = O.encode_all([xs[c] for c in check_clients], [float(work.bits[c]) for c in check_clients],
+                       [int(work.seeds[c]) for c in check_clients], threads=threads)
+    for j, c in enumerate(check_clients):
         words = codes[c].cpu().numpy().view(np.uint32)
         mism, ok, rel, enc = parity.check_encode_client(words, float(scales_h[c]), xs[c],
-                                                       float(work.bits[c]), int(work.seeds[c]))
+                                                       float(work.bits[c]), int(work.seeds[c]), pre[j])
         assert ok, "client %d: %d code mismatches outside the boundary window" % (c, mism)
         assert rel <= SCALE_TOL, "client %d: scale off by %g" % (c, rel)
         total_mism += mism
