@@ -174,9 +174,8 @@ def run_gpu(args):
     import torch
     import torch.distributed as dist
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2108_08842_b200 import replicas
+    rank, world, local_rank = replicas.rank_info()
     torch.cuda.set_device(local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
@@ -245,13 +244,10 @@ def run_gpu(args):
     total_ms = t_events[0][0].elapsed_time(t_events[-1][2])
     enc_ms = sum(a.elapsed_time(b) for a, b, c in t_events) / args.steps
     dec_ms = sum(b.elapsed_time(c) for a, b, c in t_events) / args.steps
-    t = torch.tensor([total_ms, enc_ms, dec_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, enc_ms, dec_ms = (float(v) for v in t.tolist())
+    total_ms, enc_ms, dec_ms = replicas.max_over_ranks([total_ms, enc_ms, dec_ms], dev)
     ms_per_step = total_ms / args.steps
     in_bytes = n * d * 4
-    value = world * in_bytes / (ms_per_step * 1e-3) / 1e9
+    value = replicas.whole_job_gbs(world, in_bytes, ms_per_step)
 
     # ---- roofline of the dominant kernel (by event time inside the timed region)
     peak, peak_kind = measured_hbm_peak()
@@ -298,13 +294,10 @@ def run_gpu(args):
         t_ev.record()
         barrier()
         e_ms = s_ev.elapsed_time(t_ev) / es
-        tt = torch.tensor([e_ms], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e_ms = float(tt.item())
+        e_ms = replicas.max_over_ranks([e_ms], dev)[0]
         code_bytes = sum(int(c.nbytes) for c in codes_h)
         mask_bytes = sum(int(m.nbytes) for m in masks_np) if masks_np else 0
-        e2e = {"value": world * in_bytes / (e_ms * 1e-3) / 1e9, "unit": UNIT,
+        e2e = {"value": replicas.whole_job_gbs(world, in_bytes, e_ms), "unit": UNIT,
                "h2d_bytes_per_step": in_bytes + code_bytes + mask_bytes + 4 * n,
                "d2h_bytes_per_step": code_bytes + 4 * n + 4 * d, "ms_per_step": e_ms,
                "check": "max |mean_host - mean_dev| = %g" %
