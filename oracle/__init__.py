@@ -212,9 +212,17 @@ def decode(codes: np.ndarray, scale: float, bits: float, seed: int, d: int, recv
     return xhat, rc == 1
 
 
+def _warm_tables(bits):
+    """The C side builds each table on first use and caches it without locking: build the
+    tables a threaded run needs before the threads start."""
+    for w in sorted(set(code_width(float(b)) for b in bits)):
+        table(w)
+
+
 def encode_all(xs, bits, seeds, threads: int = 1):
     """All senders; ``threads`` > 1 runs independent senders on separate threads."""
     n = len(seeds)
+    _warm_tables(bits)
 
     def one(c):
         return encode(xs[c], bits[c], seeds[c])
@@ -228,6 +236,7 @@ def encode_all(xs, bits, seeds, threads: int = 1):
 def mean(codes, scales, bits, seeds, d: int, recv_masks=None, threads: int = 1):
     """Receiver: (1/n) * sum_c x_hat_c (Section 2.2.2); returns (mean float64[d], n_used)."""
     n = len(seeds)
+    _warm_tables(bits)
 
     def one(c):
         return decode(codes[c], scales[c], bits[c], seeds[c], d,

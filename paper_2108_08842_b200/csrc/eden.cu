@@ -127,8 +127,11 @@ extern "C" uint64_t eden_workspace_bytes(uint64_t d_max, uint32_t n_batch)
 {
     if (n_batch == 0) n_batch = 1;
     const uint64_t D = 1ull << ceil_log2(d_max ? d_max : 1);
+    // per client: descriptors, one intermediate vector, and (b < 1) the mask-selection scratch
+    const uint64_t n_chunks = (d_max + kSelChunk - 1) / kSelChunk;
+    const uint64_t sel = 256 + kHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) + 256;
     return fixed_layout(d_max).end + align_up(per_client_bytes() * n_batch, 256) + 1024 +
-           (uint64_t)n_batch * D * sizeof(float);
+           (uint64_t)n_batch * (align_up(D * sizeof(float), 256) + sel);
 }
 
 extern "C" int eden_table(uint32_t W, float* centroids, float* boundaries)
@@ -402,39 +405,46 @@ int carve(const eden_ctx* ctx, uint64_t d, uint32_t n, CallLayout& lay)
     return EDEN_OK;
 }
 
-// Groups: clients with b >= 1 by rotation dimension, split so that each group's work
-// buffers fit; every client with b < 1 alone (the mask scratch is shared).
-int make_groups(const std::vector<ClientPlan>& plan, uint64_t work_bytes, std::vector<Group>& groups)
+// One client's intermediate vector in the workspace; what follows it stays 256-byte aligned.
+uint64_t work_buffer_bytes(uint64_t D) { return align_up(D * sizeof(float), 256); }
+
+// Scratch of the exact-size mask selection for one client with b < 1.
+uint64_t sel_scratch_bytes(uint64_t d)
 {
-    std::vector<uint32_t> idx;
-    for (uint32_t c = 0; c < plan.size(); ++c)
-        if (!plan[c].subbit) idx.push_back(c);
+    const uint64_t n_chunks = (d + kSelChunk - 1) / kSelChunk;
+    return 256 + kHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) +
+           align_up(sizeof(SelJob), 256);
+}
+
+// Groups: clients of one rotation dimension (and, within it, of one kind: b >= 1 or
+// b < 1) are launched together, split so that each group's work buffers and selection
+// scratch fit the workspace.  Larger dimensions first, so that for the mean a group with
+// b >= 1, which covers every output coordinate, comes before any b < 1 group.
+int make_groups(const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_bytes,
+                std::vector<Group>& groups)
+{
+    std::vector<uint32_t> idx(plan.size());
+    for (uint32_t c = 0; c < plan.size(); ++c) idx[c] = c;
     std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
-        return plan[a].L != plan[b].L ? plan[a].L > plan[b].L : plan[a].W < plan[b].W;
+        if (plan[a].subbit != plan[b].subbit) return !plan[a].subbit;
+        if (plan[a].L != plan[b].L) return plan[a].L > plan[b].L;
+        return plan[a].W < plan[b].W;
     });
     size_t i = 0;
     while (i < idx.size()) {
         Group g;
         g.L = plan[idx[i]].L;
-        g.subbit = false;
-        const uint64_t need = plan[idx[i]].needs_work ? plan[idx[i]].D * sizeof(float) : 0;
+        g.subbit = plan[idx[i]].subbit;
+        const uint64_t need = (plan[idx[i]].needs_work ? work_buffer_bytes(plan[idx[i]].D) : 0) +
+                              (g.subbit ? sel_scratch_bytes(d) : 0);
         if (need > work_bytes) return EDEN_ERR_WORKSPACE;
         uint64_t used = 0;
-        while (i < idx.size() && plan[idx[i]].L == g.L && used + need <= work_bytes &&
-               g.members.size() < 32768) {
+        while (i < idx.size() && plan[idx[i]].L == g.L && plan[idx[i]].subbit == g.subbit &&
+               used + need <= work_bytes && g.members.size() < 32768) {
             g.members.push_back(idx[i]);
             used += need;
             ++i;
         }
-        groups.push_back(g);
-    }
-    for (uint32_t c = 0; c < plan.size(); ++c) {
-        if (!plan[c].subbit) continue;
-        if (plan[c].D * sizeof(float) > work_bytes) return EDEN_ERR_WORKSPACE;
-        Group g;
-        g.L = plan[c].L;
-        g.subbit = true;
-        g.members.push_back(c);
         groups.push_back(g);
     }
     return EDEN_OK;
@@ -665,8 +675,9 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
             EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
                 LAUNCH_CL(ctx, "f_dec_last",
                           gn * 4.0 * D + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<double>((double)d, D),
-                          (k_f_dec_last<LR_, LC_>), dim3(tiles), dim3(kFastThreads), ps.lc,
-                          (const ClientDesc*)d_descs, (const ClientState*)d_states, gn, ps.lo, out, d, mode)));
+                          (k_f_dec_last<LR_, LC_>), dim3(tiles, mode == OUT_YHAT ? gn : 1u), dim3(kFastThreads), ps.lc,
+                          (const ClientDesc*)d_descs, (const ClientState*)d_states, mode == OUT_YHAT ? 1u : gn,
+                          ps.lo, out, d, mode)));
         }
     }
     return EDEN_OK;
@@ -698,6 +709,52 @@ int run_selection(eden_ctx* ctx, const FixedLayout& f, uint64_t seed, uint64_t d
 
 }  // namespace
 
+namespace {
+
+// Selection jobs of a group of clients with b < 1.  The scratch sits behind the group's
+// work buffers: n MaskSelect slots, n double histograms (contiguous, cleared by one
+// memset), n chunk arrays, then the job table itself.
+struct SelBatch {
+    SelJob* d_jobs;
+    uint32_t n;
+    unsigned grid;       // blocks of 1024 coordinates
+};
+
+int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::vector<SelJob>& partial,
+                          SelBatch& batch)
+{
+    const uint32_t n = (uint32_t)partial.size();
+    const uint64_t n_chunks = (d + kSelChunk - 1) / kSelChunk;
+    const uint64_t chunk_bytes = align_up(n_chunks * sizeof(unsigned long long), 256);
+    char* sel_base = region;
+    char* hist_base = sel_base + 256ull * n;
+    char* chunk_base = hist_base + kHistBytes * n;
+    char* job_base = chunk_base + chunk_bytes * n;
+    std::vector<SelJob> jobs(partial);
+    for (uint32_t j = 0; j < n; ++j) {
+        jobs[j].sel = (MaskSelect*)(sel_base + 256ull * j);
+        jobs[j].hist = (uint32_t*)(hist_base + kHistBytes * j);
+        jobs[j].chunks = (unsigned long long*)(chunk_base + chunk_bytes * j);
+    }
+    batch.d_jobs = (SelJob*)job_base;
+    batch.n = n;
+    batch.grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
+    CUDA_OK(cudaMemcpyAsync(batch.d_jobs, jobs.data(), sizeof(SelJob) * n, cudaMemcpyHostToDevice, ctx->stream));
+    CUDA_OK(cudaMemsetAsync(hist_base, 0, kHistBytes * n, ctx->stream));
+    const double keys = (double)n * (double)d;
+    LAUNCH(ctx, "sel_hist", 0, k_selb_hist, dim3(batch.grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs, 0);
+    LAUNCH(ctx, "sel_find", n * 65536.0 * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, 0);
+    LAUNCH(ctx, "sel_hist", 0, k_selb_hist, dim3(batch.grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs, 1);
+    LAUNCH(ctx, "sel_find", n * 65536.0 * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, 1);
+    LAUNCH(ctx, "sel_chunk_count", keys / 128.0, k_selb_chunk_count, dim3(batch.grid, n), kSelThreads, 0,
+           (const SelJob*)batch.d_jobs);
+    LAUNCH(ctx, "sel_chunk_scan", keys / 64.0, k_selb_chunk_scan, n, 1024, 0, (const SelJob*)batch.d_jobs,
+           (uint64_t)batch.grid);
+    return EDEN_OK;
+}
+
+}  // namespace
+
 // ------------------------------------------------------------------------------------
 // sender
 // ------------------------------------------------------------------------------------
@@ -716,7 +773,7 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
     rc = carve(ctx, d, n, lay);
     if (rc) return rc;
     std::vector<Group> groups;
-    rc = make_groups(plan, lay.work_bytes, groups);
+    rc = make_groups(plan, d, lay.work_bytes, groups);
     if (rc) return rc;
     const FixedLayout f = fixed_layout(d);
     const bool x_aligned = ((uintptr_t)x & 15u) == 0 && (ld_x & 3u) == 0;
@@ -734,7 +791,7 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
             ClientDesc cd;
             std::memset(&cd, 0, sizeof(cd));
             cd.work = p.needs_work ? (float*)(ctx->ws + lay.work_off + off) : nullptr;
-            if (p.needs_work) off += p.D * sizeof(float);
+            if (p.needs_work) off += work_buffer_bytes(p.D);
             cd.src = p.subbit ? cd.work : x + (uint64_t)p.index * ld_x;
             cd.codes = (uint32_t*)codes[p.index];
             cd.recv = nullptr;
@@ -762,15 +819,27 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
         const Group& g = groups[gi];
         const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
         if (g.subbit) {
-            const ClientPlan& p = plan[g.members[0]];
-            rc = run_selection(ctx, f, seeds[p.index], d, p.k);
+            // exact-size masks of all members, then gather their kept coordinates
+            std::vector<SelJob> jobs(gn);
+            uint64_t work_end = 0, kept = 0;
+            for (uint32_t j = 0; j < gn; ++j) {
+                const ClientPlan& p = plan[g.members[j]];
+                std::memset(&jobs[j], 0, sizeof(SelJob));
+                jobs[j].seed = seeds[p.index];
+                jobs[j].d = d;
+                jobs[j].k = p.k;
+                jobs[j].in = x + (uint64_t)p.index * ld_x;
+                jobs[j].out = descs[first + j].work;
+                work_end += work_buffer_bytes(p.D);
+                kept += p.k;
+            }
+            SelBatch batch;
+            rc = start_selection_batch(ctx, ctx->ws + lay.work_off + work_end, d, jobs, batch);
             if (rc) return rc;
-            const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
-            LAUNCH(ctx, "sel_compact", 4.0 * d + 4.0 * p.k, k_sel_apply<SEL_COMPACT>, grid, kSelThreads, 0, seeds[p.index], d,
-                   (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
-                   x + (uint64_t)p.index * ld_x, descs[first].work, (uint32_t*)nullptr);
+            LAUNCH(ctx, "sel_compact", 4.0 * gn * (double)d + 4.0 * (double)kept, k_selb_compact,
+                   dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
         }
-        if (fast_eligible(ctx, g) && x_aligned) {
+        if (fast_eligible(ctx, g) && (x_aligned || g.subbit)) {
             rc = fast_encode_group(ctx, plan, g, d_descs + first, d_states + first, d);
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
@@ -819,7 +888,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
     rc = carve(ctx, d, n, lay);
     if (rc) return rc;
     std::vector<Group> groups;
-    rc = make_groups(plan, lay.work_bytes, groups);
+    rc = make_groups(plan, d, lay.work_bytes, groups);
     if (rc) return rc;
     const FixedLayout f = fixed_layout(d);
 
@@ -835,7 +904,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             ClientDesc cd;
             std::memset(&cd, 0, sizeof(cd));
             cd.work = p.needs_work ? (float*)(ctx->ws + lay.work_off + off) : nullptr;
-            if (p.needs_work) off += p.D * sizeof(float);
+            if (p.needs_work) off += work_buffer_bytes(p.D);
             cd.src = nullptr;
             cd.codes = (uint32_t*)codes[p.index];
             cd.recv = recv_masks ? recv_masks[p.index] : nullptr;
@@ -871,18 +940,36 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         const Group& g = groups[gi];
         const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
         int mode = g.subbit ? OUT_YHAT : (written ? OUT_ACC : OUT_WRITE);
+        SelBatch batch{nullptr, 0, 0};
+        uint64_t kept = 0;
         if (g.subbit) {
-            const ClientPlan& p = plan[g.members[0]];
-            rc = run_selection(ctx, f, seeds[p.index], d, p.k);
+            // exact-size masks of all members (the estimates of their kept coordinates will
+            // be written to their work buffers and scattered from there)
+            std::vector<SelJob> jobs(gn);
+            uint64_t work_end = 0;
+            for (uint32_t j = 0; j < gn; ++j) {
+                const ClientPlan& p = plan[g.members[j]];
+                std::memset(&jobs[j], 0, sizeof(SelJob));
+                jobs[j].seed = seeds[p.index];
+                jobs[j].d = d;
+                jobs[j].k = p.k;
+                jobs[j].in = descs[first + j].work;
+                work_end += work_buffer_bytes(p.D);
+                kept += p.k;
+            }
+            rc = start_selection_batch(ctx, ctx->ws + lay.work_off + work_end, d, jobs, batch);
             if (rc) return rc;
         }
+        // with OUT_YHAT every member writes its own estimate: one block row per member
+        const uint32_t loop_n = g.subbit ? 1u : gn;
+        const unsigned rows = g.subbit ? gn : 1u;
         if (fast_eligible(ctx, g)) {
             rc = fast_decode_group(ctx, plan, g, d_descs + first, d_states + first, out, d, mode);
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);
-            LAUNCH(ctx, "dec_single", gn * code_bits_per_coord(plan, g) / 8.0 * (double)(1ull << g.L) + 4.0 * d, k_dec_last<true>, dim3(1), kGenericThreads, sizeof(float) << g.L,
-                   d_descs + first, d_states + first, gn, rg, out, d, mode);
+            LAUNCH(ctx, "dec_single", gn * code_bits_per_coord(plan, g) / 8.0 * (double)(1ull << g.L) + 4.0 * d, k_dec_last<true>, dim3(1, rows), kGenericThreads, sizeof(float) << g.L,
+                   d_descs + first, d_states + first, loop_n, rg, out, d, mode);
         } else {
             const int lc = kGenericTileLog;
             LAUNCH(ctx, "dec_first", gn * (4.0 + code_bits_per_coord(plan, g) / 8.0) * (double)(1ull << g.L), k_dec_first, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
@@ -896,16 +983,13 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
                     LAUNCH(ctx, "mid", gn * 8.0 * (double)(1ull << g.L), k_mid, dim3(tiles, gn), kGenericThreads, sizeof(float) << cg.lt,
                            d_descs + first, cg);
                 else
-                    LAUNCH(ctx, "dec_last", gn * 4.0 * (double)(1ull << g.L) + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<uint64_t>(d, 1ull << g.L), k_dec_last<false>, dim3(tiles), kGenericThreads, sizeof(float) << cg.lt,
-                           d_descs + first, d_states + first, gn, cg, out, d, mode);
+                    LAUNCH(ctx, "dec_last", gn * 4.0 * (double)(1ull << g.L) + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<uint64_t>(d, 1ull << g.L), k_dec_last<false>, dim3(tiles, rows), kGenericThreads, sizeof(float) << cg.lt,
+                           d_descs + first, d_states + first, loop_n, cg, out, d, mode);
             }
         }
         if (g.subbit) {
-            const ClientPlan& p = plan[g.members[0]];
-            const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
-            LAUNCH(ctx, "sel_scatter", 8.0 * p.k + 4.0 * p.k, k_sel_apply<SEL_SCATTER_ACC>, grid, kSelThreads, 0, seeds[p.index], d,
-                   (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
-                   (const float*)descs[first].work, out, (uint32_t*)nullptr);
+            LAUNCH(ctx, "sel_scatter", 8.0 * (double)kept + 4.0 * (double)kept, k_selb_scatter, batch.grid,
+                   kSelThreads, 0, (const SelJob*)batch.d_jobs, gn, d, out);
         } else {
             written = true;
         }

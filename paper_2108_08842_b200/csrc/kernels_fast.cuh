@@ -372,13 +372,16 @@ k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, 
 // Receiver, last pass: for every client of the group finish the inverse transform of the
 // tile, apply sign and factor, add into registers; store the sum once (Sections 2.2.2,
 // 4.2).  mode: OUT_WRITE / OUT_ACC into out[0, d), or OUT_YHAT into the client's own work
-// buffer (b < 1, single client).
+// buffer (b < 1: one block row per client, n_group = 1).
 // =================================================================================
 template <int LR, int LC>
 __global__ void __launch_bounds__(kFastThreads, 2)
-k_f_dec_last(const ClientDesc* __restrict__ descs, const ClientState* __restrict__ states,
+k_f_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restrict__ states_in,
              uint32_t n_group, int lo, float* __restrict__ out, uint64_t d, int mode)
 {
+    // OUT_YHAT: block row y handles member y alone (n_group = 1)
+    const ClientDesc* __restrict__ descs = descs_in + (mode == OUT_YHAT ? blockIdx.y : 0);
+    const ClientState* __restrict__ states = states_in + (mode == OUT_YHAT ? blockIdx.y : 0);
     __shared__ ulonglong2 s[2048];
     __shared__ uint32_t s_sign[256];
     const ColTile ct = col_tile<LR, LC>(blockIdx.x, lo);

@@ -316,9 +316,12 @@ k_dec_first(const ClientDesc* __restrict__ descs, PassGeom g)
 // (b < 1) for the scatter kernel.
 template <bool FROM_CODES>
 __global__ void __launch_bounds__(kGenericThreads)
-k_dec_last(const ClientDesc* __restrict__ descs, const ClientState* __restrict__ states,
+k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restrict__ states_in,
            uint32_t n_group, PassGeom g, float* __restrict__ out, uint64_t d, int mode)
 {
+    // OUT_YHAT: block row y handles member y alone (n_group = 1)
+    const ClientDesc* __restrict__ descs = descs_in + (mode == OUT_YHAT ? blockIdx.y : 0);
+    const ClientState* __restrict__ states = states_in + (mode == OUT_YHAT ? blockIdx.y : 0);
     extern __shared__ float s[];
     __shared__ float s_tv[128];
     const int T = 1 << g.lt;

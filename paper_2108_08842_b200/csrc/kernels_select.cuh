@@ -37,35 +37,72 @@ k_sel_hist(uint64_t seed, uint64_t d, int round, const MaskSelect* __restrict__ 
 
 // Finds the histogram bin that holds the element of 0-based rank r (one block of 1024
 // threads over 65536 bins).  Round 0: r = k - 1, writes bin_hi / below_hi.  Round 1:
-// r = k - 1 - below_hi, writes tau, below and rem.
-__global__ void __launch_bounds__(1024)
-k_sel_find(const uint32_t* __restrict__ hist, uint64_t k, int round, MaskSelect* __restrict__ sel)
+// r = k - 1 - below_hi, writes tau, below and rem.  Each warp sums a run of 2048 bins with
+// coalesced loads; the warp whose run holds rank r then walks it 32 bins at a time.
+__device__ __forceinline__ void sel_find_body(const uint32_t* __restrict__ hist, uint64_t k, int round,
+                                              MaskSelect* __restrict__ sel)
 {
-    __shared__ unsigned long long scratch[33];
+    __shared__ uint32_t warp_total[32];
+    __shared__ uint32_t warp_before[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t r = round ? (uint32_t)(k - 1) - sel->below_hi : (uint32_t)(k - 1);
+    const uint32_t* run = hist + warp * 2048;
     uint32_t mine = 0;
-    for (int j = 0; j < 64; ++j) mine += hist[threadIdx.x * 64 + j];
-    unsigned long long total;
-    const uint32_t before = (uint32_t)block_exclusive_scan(mine, scratch, &total);
-    if (r >= before && r < before + mine) {
-        uint32_t run = before;
-        for (int j = 0; j < 64; ++j) {
-            const uint32_t h = hist[threadIdx.x * 64 + j];
-            if (r < run + h) {
-                const uint32_t bin = threadIdx.x * 64 + j;
-                if (round == 0) {
-                    sel->bin_hi = bin;
-                    sel->below_hi = run;
-                } else {
-                    sel->tau = (sel->bin_hi << 16) | bin;
-                    sel->below = sel->below_hi + run;
-                    sel->rem = (uint32_t)k - (sel->below_hi + run);   // ties to keep, >= 1
+#pragma unroll 8
+    for (int i = 0; i < 64; ++i) mine += run[i * 32 + lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if (lane == 0) warp_total[warp] = mine;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t v = warp_total[lane];
+        uint32_t inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        warp_before[lane] = inc - v;
+    }
+    __syncthreads();
+    const uint32_t before = warp_before[warp];
+    if (r >= before && r < before + warp_total[warp]) {        // exactly one warp
+        uint32_t seen = before;
+        for (int i = 0; i < 64; ++i) {
+            const uint32_t v = run[i * 32 + lane];
+            uint32_t inc = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += t;
+            }
+            const uint32_t chunk_total = __shfl_sync(0xffffffffu, inc, 31);
+            if (r < seen + chunk_total) {
+                const uint32_t hit = __ballot_sync(0xffffffffu, r < seen + inc);
+                const int first = __ffs(hit) - 1;
+                if (lane == first) {
+                    const uint32_t bin = (uint32_t)(warp * 2048 + i * 32 + lane);
+                    const uint32_t below = seen + inc - v;
+                    if (round == 0) {
+                        sel->bin_hi = bin;
+                        sel->below_hi = below;
+                    } else {
+                        sel->tau = (sel->bin_hi << 16) | bin;
+                        sel->below = sel->below_hi + below;
+                        sel->rem = (uint32_t)k - (sel->below_hi + below);   // ties to keep, >= 1
+                    }
                 }
                 break;
             }
-            run += h;
+            seen += chunk_total;
         }
     }
+}
+
+__global__ void __launch_bounds__(1024)
+k_sel_find(const uint32_t* __restrict__ hist, uint64_t k, int round, MaskSelect* __restrict__ sel)
+{
+    sel_find_body(hist, k, round, sel);
 }
 
 // (keys below tau, keys equal to tau) of the four coordinates of Philox call t, as a
@@ -163,6 +200,129 @@ k_sel_apply(uint64_t seed, uint64_t d, const MaskSelect* __restrict__ sel,
         w |= __shfl_xor_sync(0xffffffffu, w, 2);
         w |= __shfl_xor_sync(0xffffffffu, w, 4);
         if ((threadIdx.x & 7) == 0 && t * 4 < d) bits[t >> 3] = w;
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// The same steps for several clients at once: one job per client with b < 1, the job
+// index in blockIdx.y (blockIdx.x for the one-block steps).
+// ---------------------------------------------------------------------------------
+struct SelJob {
+    uint64_t seed, d, k;
+    MaskSelect* sel;
+    uint32_t* hist;                  // 2 x 65536 bins
+    unsigned long long* chunks;      // one packed count per 1024 coordinates
+    const float* in;                 // compact: the client's input row; scatter: its estimate of the kept coordinates
+    float* out;                      // compact: the compacted vector
+};
+
+__global__ void __launch_bounds__(kSelThreads)
+k_selb_hist(const SelJob* __restrict__ jobs, int round)
+{
+    const SelJob job = jobs[blockIdx.y];
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t * 4 >= job.d) return;
+    const uint4 k4 = mask_keys(job.seed, t);
+    const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
+    const uint32_t want = round ? job.sel->bin_hi : 0u;
+    uint32_t* hist = job.hist + (round ? 65536 : 0);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (t * 4 + j >= job.d) break;
+        if (round == 0) atomicAdd(&hist[keys[j] >> 16], 1u);
+        else if ((keys[j] >> 16) == want) atomicAdd(&hist[keys[j] & 0xFFFFu], 1u);
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+k_selb_find(const SelJob* __restrict__ jobs, int round)
+{
+    const SelJob job = jobs[blockIdx.x];
+    sel_find_body(job.hist + (round ? 65536 : 0), job.k, round, job.sel);
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+k_selb_chunk_count(const SelJob* __restrict__ jobs)
+{
+    __shared__ unsigned long long scratch[33];
+    const SelJob job = jobs[blockIdx.y];
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t cls[4];
+    const unsigned long long mine = classify4(job.seed, t, job.d, job.sel->tau, cls);
+    unsigned long long total;
+    block_exclusive_scan(mine, scratch, &total);
+    if (threadIdx.x == 0) job.chunks[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(1024)
+k_selb_chunk_scan(const SelJob* __restrict__ jobs, uint64_t n_chunks)
+{
+    __shared__ unsigned long long scratch[33];
+    unsigned long long* chunk_counts = jobs[blockIdx.x].chunks;
+    const uint64_t per = (n_chunks + blockDim.x - 1) / blockDim.x;
+    const uint64_t lo = min((uint64_t)threadIdx.x * per, n_chunks), hi = min(lo + per, n_chunks);
+    unsigned long long mine = 0;
+    for (uint64_t j = lo; j < hi; ++j) mine += chunk_counts[j];
+    unsigned long long total;
+    unsigned long long run = block_exclusive_scan(mine, scratch, &total);
+    for (uint64_t j = lo; j < hi; ++j) {
+        const unsigned long long v = chunk_counts[j];
+        chunk_counts[j] = run;
+        run += v;
+    }
+}
+
+// Sender: y_c[pos] = x_c[i] for the kept coordinates of every job.
+__global__ void __launch_bounds__(kSelThreads)
+k_selb_compact(const SelJob* __restrict__ jobs)
+{
+    __shared__ unsigned long long scratch[33];
+    const SelJob job = jobs[blockIdx.y];
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t tau = job.sel->tau, rem = job.sel->rem;
+    uint32_t cls[4];
+    const unsigned long long mine = classify4(job.seed, t, job.d, tau, cls);
+    unsigned long long total;
+    const unsigned long long before = block_exclusive_scan(mine, scratch, &total) + job.chunks[blockIdx.x];
+    uint32_t below = (uint32_t)before, ties = (uint32_t)(before >> 32);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint64_t i = t * 4 + j;
+        const bool keep = cls[j] == 1 || (cls[j] == 2 && ties < rem);
+        if (keep) job.out[(uint64_t)below + min(ties, rem)] = job.in[i];
+        if (cls[j] == 1) ++below;
+        if (cls[j] == 2) ++ties;
+    }
+}
+
+// Receiver: out[i] += sum over the jobs of yhat_c[pos_c(i)] for the coordinates job c kept
+// (Section 4.1: the receiver restores through the same mask).  One pass over out.
+__global__ void __launch_bounds__(kSelThreads)
+k_selb_scatter(const SelJob* __restrict__ jobs, uint32_t n_jobs, uint64_t d, float* __restrict__ out)
+{
+    __shared__ unsigned long long scratch[33];
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    float add[4] = {0.f, 0.f, 0.f, 0.f};
+    for (uint32_t c = 0; c < n_jobs; ++c) {
+        const SelJob job = jobs[c];
+        const uint32_t tau = job.sel->tau, rem = job.sel->rem;
+        uint32_t cls[4];
+        const unsigned long long mine = classify4(job.seed, t, d, tau, cls);
+        unsigned long long total;
+        const unsigned long long before = block_exclusive_scan(mine, scratch, &total) + job.chunks[blockIdx.x];
+        uint32_t below = (uint32_t)before, ties = (uint32_t)(before >> 32);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bool keep = cls[j] == 1 || (cls[j] == 2 && ties < rem);
+            if (keep) add[j] += job.in[(uint64_t)below + min(ties, rem)];
+            if (cls[j] == 1) ++below;
+            if (cls[j] == 2) ++ties;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint64_t i = t * 4 + j;
+        if (i < d && add[j] != 0.f) out[i] += add[j];
     }
 }
 
