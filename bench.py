@@ -184,7 +184,9 @@ def run_gpu(args):
     __graft_entry__.build()
     from paper_2108_08842_b200 import eden, synth
 
-    work = synth.make(args.workload, n=args.n, seed=rank)
+    work = synth.make(args.workload, d=args.d, n=args.n, seed=rank)
+    if args.bits is not None:
+        work.bits = np.full(work.n, float(args.bits))
     n, d = work.n, work.d
     cores = host_cores()
     dev = torch.device("cuda", local_rank)
@@ -341,6 +343,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--n", type=int, default=None, help="override the number of clients (small profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (small profiling runs)")
+    ap.add_argument("--d", type=int, default=None, help="override the dimension (sweeps)")
+    ap.add_argument("--bits", type=float, default=None, help="override every client's bit budget (sweeps)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
