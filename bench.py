@@ -31,6 +31,11 @@ if ROOT not in sys.path:
 METRIC = "encode and decode+mean GB/s (fp32 in)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes (read + write) per rotated coordinate and client from the ncu capture in
+# profiles/ncu_full_fast_kernels_cfg5_n1.md (one client of 2^27 coordinates per launch;
+# traffic grows in proportion to the clients a launch covers).  Only kernels that have not
+# changed since that capture are listed.
+NCU_DRAM_BYTES_PER_COORD = {"f_mid": (536.88 + 482.55) * 1e6 / 2 ** 27}
 
 
 def host_cores() -> int:
@@ -258,7 +263,9 @@ def run_gpu(args):
     achieved = top["bytes"] / top["launches"] / (top["ms"] / top["launches"] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": top_name, "achieved": achieved, "peak": peak,
                 "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None,
+                "traffic": (NCU_DRAM_BYTES_PER_COORD[top_name] * n * float(eden.rot_dim(d, float(bits[0])))
+                            if top_name in NCU_DRAM_BYTES_PER_COORD and len(set(map(float, bits))) == 1 else None),
+                "traffic_source": "ncu dram__bytes_read+write, one client, scaled by clients per launch",
                 "algorithmic_bytes_per_launch": top["bytes"] / top["launches"],
                 "ms_per_launch": top["ms"] / top["launches"]}
     kernel_table = {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
