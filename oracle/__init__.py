@@ -56,6 +56,12 @@ def _L():
             getattr(lib, name).restype = u64
         lib.eden_oracle_code_width.argtypes = [f64]
         lib.eden_oracle_code_width.restype = u32
+        lib.eden_oracle_coin_threshold.argtypes = [f64]
+        lib.eden_oracle_coin_threshold.restype = u32
+        lib.eden_oracle_coin.argtypes = [u64, u64, u32]
+        lib.eden_oracle_coin.restype = ctypes.c_int
+        lib.eden_oracle_code_words.argtypes = [u64, f64]
+        lib.eden_oracle_code_words.restype = u64
         lib.eden_oracle_num_packets.argtypes = [u64]
         lib.eden_oracle_num_packets.restype = u64
         lib.eden_oracle_interval_mass.argtypes = [f64, f64]
@@ -104,7 +110,16 @@ def num_packets(D: int) -> int:
 
 
 def code_words(d: int, bits: float) -> int:
-    return (rot_dim(d, bits) * code_width(bits) + 31) // 32
+    return int(_L().eden_oracle_code_words(rot_dim(d, bits), float(bits)))
+
+
+def coin_threshold(bits: float) -> int:
+    """0 for integer and sub-bit budgets, else round(frac(b) * 65536)."""
+    return int(_L().eden_oracle_coin_threshold(float(bits)))
+
+
+def coin(seed: int, i: int, threshold: int) -> bool:
+    return bool(_L().eden_oracle_coin(int(seed), int(i), int(threshold)))
 
 
 # --------------------------------------------------------------------------- RNG

@@ -38,6 +38,16 @@
  *     coordinate i in stream bits [i*W, i*W + W) (bit b of the stream = bit b%32
  *     of 32-bit word b/32), low bit of the code first.                [layout unpinned]
  *   - A packet is 1024 consecutive rotated coordinates.
+ *   - Non-integer budgets b > 1 (Section 4.1): coordinate i is coded with 2^(floor(b)+1)
+ *     values if its coin is set, else with 2^floor(b).  Coins are Philox stream 2:
+ *     call t yields eight 16-bit numbers (low half of word 0, high half of word 0,
+ *     low half of word 1, ...) for rotated coordinates 8t..8t+7; the coin is set iff
+ *     the number is below round((b - floor(b)) * 65536).              [stream layout unpinned]
+ *     Wire layout for such b: groups of 32 coordinates, floor(b)+1 words each: first a
+ *     bit stream of floor(b)-bit fields (the code of an unset coordinate, or the
+ *     upper floor(b) bits of a set coordinate's code), then one word holding the lowest
+ *     code bit of the set coordinates, packed in coordinate order from bit 0.
+ *     Only floor(b)*32 + (number of coins) bits of a group are meaningful.  [layout unpinned]
  *   - The interval decision is taken after rounding z and the boundary to fp32,
  *     the precision the GPU kernels decide in; everything else is double.
  *   - ||x|| = 0: scale 0, all codes 0.  A client with no received packet
@@ -120,10 +130,40 @@ uint64_t eden_oracle_rot_dim(uint64_t d, double bits)
     return D;
 }
 
+/* widest code of a client: 1 for b <= 1, b for integer b, floor(b)+1 otherwise */
 uint32_t eden_oracle_code_width(double bits)
 {
     if (bits <= 1.0) return 1u;
-    return (uint32_t)bits; /* integer budgets 2..8 */
+    if (bits == floor(bits)) return (uint32_t)bits;
+    return (uint32_t)floor(bits) + 1u;
+}
+
+/* 0 for an integer (or sub-bit) budget, else the coin threshold round(frac * 65536) */
+uint32_t eden_oracle_coin_threshold(double bits)
+{
+    if (bits <= 1.0 || bits == floor(bits)) return 0u;
+    uint32_t t = (uint32_t)floor((bits - floor(bits)) * 65536.0 + 0.5);
+    if (t < 1u) t = 1u;
+    if (t > 65535u) t = 65535u;
+    return t;
+}
+
+/* coin of rotated coordinate i for a non-integer budget (Philox stream 2) */
+int eden_oracle_coin(uint64_t seed, uint64_t i, uint32_t threshold)
+{
+    uint32_t w[4];
+    philox_stream(seed, 2u, i / 8u, w);
+    uint32_t word = w[(i % 8u) / 2u];
+    uint32_t half = (i % 2u) ? (word >> 16) : (word & 0xFFFFu);
+    return half < threshold;
+}
+
+/* words of one client's message */
+uint64_t eden_oracle_code_words(uint64_t D, double bits)
+{
+    uint32_t W = eden_oracle_code_width(bits);
+    if (eden_oracle_coin_threshold(bits)) return ((D + 31u) / 32u) * W;   /* padded groups */
+    return (D * W + 31u) / 32u;
 }
 
 /* ------------------------------------------------------------------------- */
@@ -310,7 +350,9 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
     uint64_t k = eden_oracle_kept_count(d, bits);
     uint64_t D = eden_oracle_rot_dim(d, bits);
     uint32_t W = eden_oracle_code_width(bits);
-    uint64_t n_words = (D * W + 31u) / 32u;
+    uint64_t n_words = eden_oracle_code_words(D, bits);
+    uint32_t coin_thr = eden_oracle_coin_threshold(bits);
+    uint32_t W0 = coin_thr ? W - 1u : W;       /* width of the fixed fields */
 
     double *y = (double *)calloc(D, sizeof(double));
     if (!y) return -1;
@@ -352,13 +394,31 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
     /* steps 4-6: z = eta r with eta = sqrt(D)/||y||, code, dot <r, Q(z)> */
     double eta = sqrt((double)D) / sqrt(N2);
     double dot = 0.0;
+    uint32_t extra_pos = 0;                        /* next free bit of the group's extra word */
     for (uint64_t i = 0; i < D; ++i) {
         double z = eta * y[i];
-        uint32_t code = eden_oracle_quantise(z, W);
-        dot += y[i] * eden_oracle_value(code, W);
-        for (uint32_t j = 0; j < W; ++j) {           /* field i of the bit stream */
-            uint64_t b = i * W + j;
-            codes[b / 32u] |= ((code >> j) & 1u) << (b % 32u);
+        if (!coin_thr) {
+            uint32_t code = eden_oracle_quantise(z, W);
+            dot += y[i] * eden_oracle_value(code, W);
+            for (uint32_t j = 0; j < W; ++j) {           /* field i of the bit stream */
+                uint64_t b = i * W + j;
+                codes[b / 32u] |= ((code >> j) & 1u) << (b % 32u);
+            }
+        } else {
+            /* non-integer budget: 2^(W0+1) values if the coin is set, else 2^W0 */
+            uint64_t g = i / 32u, l = i % 32u;
+            uint32_t *grp = codes + g * W;
+            if (l == 0) extra_pos = 0;
+            int coin = eden_oracle_coin(seed, i, coin_thr);
+            uint32_t Wi = coin ? W0 + 1u : W0;
+            uint32_t code = eden_oracle_quantise(z, Wi);
+            dot += y[i] * eden_oracle_value(code, Wi);
+            uint32_t field = coin ? code >> 1 : code;
+            for (uint32_t j = 0; j < W0; ++j) {
+                uint64_t b = l * W0 + j;
+                grp[b / 32u] |= ((field >> j) & 1u) << (b % 32u);
+            }
+            if (coin) grp[W0] |= (code & 1u) << extra_pos++;
         }
         if (z_out) z_out[i] = z;
     }
@@ -385,15 +445,37 @@ int eden_oracle_decode(const uint32_t *codes, double S, double bits, uint64_t se
     uint64_t k = eden_oracle_kept_count(d, bits);
     uint64_t D = eden_oracle_rot_dim(d, bits);
     uint32_t W = eden_oracle_code_width(bits);
+    uint32_t coin_thr = eden_oracle_coin_threshold(bits);
+    uint32_t W0 = coin_thr ? W - 1u : W;
 
     memset(xhat, 0, sizeof(double) * d);
     double *q = (double *)calloc(D, sizeof(double));
     if (!q) return -1;
 
     uint64_t received = 0;
+    uint32_t extra_pos = 0;
     for (uint64_t i = 0; i < D; ++i) {
         uint64_t pkt = i / EDEN_ORACLE_PACKET;
         int arrived = recv_mask ? (int)((recv_mask[pkt / 32u] >> (pkt % 32u)) & 1u) : 1;
+        if (coin_thr) {
+            /* the position of a set coordinate's extra bit depends on the coins before it */
+            uint64_t g = i / 32u, l = i % 32u;
+            const uint32_t *grp = codes + g * W;
+            if (l == 0) extra_pos = 0;
+            int coin = eden_oracle_coin(seed, i, coin_thr);
+            uint32_t my_pos = extra_pos;
+            if (coin) ++extra_pos;
+            if (!arrived) continue;
+            ++received;
+            uint32_t field = 0;
+            for (uint32_t j = 0; j < W0; ++j) {
+                uint64_t b = l * W0 + j;
+                field |= ((grp[b / 32u] >> (b % 32u)) & 1u) << j;
+            }
+            if (coin) q[i] = eden_oracle_value((field << 1) | ((grp[W0] >> my_pos) & 1u), W0 + 1u);
+            else q[i] = eden_oracle_value(field, W0);
+            continue;
+        }
         if (!arrived) continue; /* lost coordinate counts as 0 */
         ++received;
         uint32_t code = 0;

@@ -448,3 +448,98 @@ def test_nmse_of_mean_is_vnmse_over_n():
     c, b, edges, p = _levels(4)
     limit = (1 / (p * c * c).sum() - 1) / n        # Lemma 2.2 with equal budgets
     assert abs(tot / rounds - limit) < 0.15 * limit, (tot / rounds, limit)
+
+
+# ----------------------------------------------------------------------------- non-integer budgets b > 1
+def _coins_from_raw_philox(seed, D, bits):
+    thr = int(math.floor((bits - math.floor(bits)) * 65536 + 0.5))
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    out = np.zeros(D, dtype=bool)
+    for t in range((D + 7) // 8):
+        w = O.philox4x32_10([t, 0, 2, 0], key)
+        halves = []
+        for v in w:
+            halves += [int(v) & 0xFFFF, int(v) >> 16]
+        for j in range(8):
+            if 8 * t + j < D:
+                out[8 * t + j] = halves[j] < thr
+    return out
+
+
+def _unpack_fractional(words, D, W0, coins):
+    codes = np.zeros(D, dtype=np.int64)
+    for g in range((D + 31) // 32):
+        grp = words[g * (W0 + 1):(g + 1) * (W0 + 1)]
+        pos = 0
+        for l in range(min(32, D - 32 * g)):
+            i = 32 * g + l
+            field = 0
+            for j in range(W0):
+                b = l * W0 + j
+                field |= ((int(grp[b // 32]) >> (b % 32)) & 1) << j
+            if coins[i]:
+                codes[i] = (field << 1) | ((int(grp[W0]) >> pos) & 1)
+                pos += 1
+            else:
+                codes[i] = field
+    return codes
+
+
+@pytest.mark.parametrize("d,bits", [(64, 1.5), (100, 2.25), (40, 3.5), (256, 7.75)])
+def test_fractional_budget_against_dense_reference(d, bits):
+    rng = np.random.default_rng(int(d * bits))
+    x = rng.standard_normal(d).astype(np.float32)
+    seed = int(rng.integers(1, 2 ** 63))
+    D, W0 = O.rot_dim(d, bits), int(math.floor(bits))
+    assert O.code_width(bits) == W0 + 1 and O.coin_threshold(bits) == round((bits - W0) * 65536)
+    coins = _coins_from_raw_philox(seed, D, bits)
+    assert all(O.coin(seed, i, O.coin_threshold(bits)) == coins[i] for i in range(D))
+    # independent dense route: rotate, per-coordinate nearest value in its own table (Section 4.1)
+    y = np.zeros(D)
+    y[:d] = x
+    s = O.signs(seed, D)
+    R = scipy.linalg.hadamard(D) / math.sqrt(D) @ np.diag(s)
+    r = R @ y
+    z = math.sqrt(D) * r / np.linalg.norm(y)
+    tabs = {W0: O.table(W0)[0], W0 + 1: O.table(W0 + 1)[0]}
+    codes_ref = np.array([int(np.argmin(np.abs(tabs[W0 + 1 if coins[i] else W0] - z[i]))) for i in range(D)])
+    q = np.array([tabs[W0 + 1 if coins[i] else W0][codes_ref[i]] for i in range(D)])
+    S_ref = np.dot(y, y) / np.dot(r, q)
+    enc = O.encode(x, bits, seed)
+    assert len(enc["codes"]) == (D + 31) // 32 * (W0 + 1)
+    assert np.array_equal(_unpack_fractional(enc["codes"], D, W0, coins), codes_ref)
+    assert abs(enc["scale"] - S_ref) < 1e-10 * S_ref
+    xhat, _ = O.decode(enc["codes"], enc["scale"], bits, seed, d)
+    assert np.allclose(xhat, (S_ref * (R.T @ q))[:d], rtol=1e-10, atol=1e-12)
+
+
+def test_fractional_budget_vnmse_and_bit_usage(golden):
+    K = _const(golden)
+    eq2 = {n: float((_levels(n)[3] * _levels(n)[0] ** 2).sum()) for n in (2, 4, 8)}
+    # b = 1.5: vNMSE -> 1/(E1/2 + E2/2) - 1 = 0.317 (Section 4.1), below the naive split's 0.352
+    got = _vnmse(1 << 14, 1.5, range(300, 312))
+    assert abs(got - K["vnmse_b1p5"][0]) < 0.04 * K["vnmse_b1p5"][0]
+    assert got < K["naive_split_b1p5"][0] - 0.02
+    # b = 2.25: a quarter of the coordinates get three bits
+    limit = 1 / (0.75 * eq2[4] + 0.25 * eq2[8]) - 1
+    got = _vnmse(1 << 14, 2.25, range(320, 332))
+    assert abs(got - limit) < 0.05 * limit
+    # the share of upgraded coordinates concentrates around the fraction (expected budget b)
+    coins = _coins_from_raw_philox(4711, 1 << 15, 2.25)
+    assert abs(coins.mean() - 0.25) < 5 * math.sqrt(0.25 * 0.75 / (1 << 15))
+
+
+def test_fractional_budget_unbiased_at_d64():
+    d, trials = 64, 10000
+    x = np.random.default_rng(12).standard_normal(d).astype(np.float32)
+    xd = x.astype(np.float64)
+    acc = np.zeros(d)
+    err2 = 0.0
+    for s in range(trials):
+        e = O.encode(x, 1.5, 900000 + s)
+        xh, _ = O.decode(e["codes"], e["scale"], 1.5, 900000 + s, d)
+        acc += xh
+        err2 += np.dot(xh - xd, xh - xd)
+    vnmse = err2 / trials / np.dot(xd, xd)
+    bias2 = np.dot(acc / trials - xd, acc / trials - xd) / np.dot(xd, xd)
+    assert bias2 < 3 * vnmse / trials, (bias2, vnmse / trials)
