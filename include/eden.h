@@ -21,8 +21,11 @@
  *     sides and are not stored in the message.  Seeds must differ between clients and
  *     between rounds; that is the caller's duty.
  *   - Supported budgets: 0 < b <= 1 (one-bit codes; b < 1 adds the shared-seed
- *     sparsification of Section 4.1) and the integers 2..8 (Section 3).  Other values
- *     return EDEN_ERR_UNSUPPORTED_BITS.
+ *     sparsification of Section 4.1), the integers 2..8 (Section 3) and non-integer
+ *     1 < b < 8 (Section 4.1: each coordinate is coded with 2^(floor(b)+1) values if its
+ *     shared coin is set, with 2^floor(b) otherwise; coins are Philox stream 2, call t
+ *     giving eight 16-bit numbers for coordinates 8t..8t+7, set iff the number is below
+ *     round((b - floor(b)) * 65536)).  Other values return EDEN_ERR_UNSUPPORTED_BITS.
  *   - Rotation (Section 5): R = (1/sqrt D) H_D Diag(s), H_D the Sylvester-ordered
  *     Walsh-Hadamard matrix, D = 2^ceil(log2 d') with d' = d for b >= 1 and d' = the
  *     kept count k for b < 1; shorter vectors are zero-padded, all D coordinates are
@@ -35,6 +38,11 @@
  *     first; stream bit b is bit b%32 of 32-bit word b/32.  A code is the rank of its
  *     quantisation value in ascending order.  A packet is 1024 consecutive rotated
  *     coordinates = 128*W bytes.  The scale S travels beside the codes as one fp32.
+ *     Non-integer b: groups of 32 coordinates of W = floor(b)+1 words each: first the bit
+ *     stream of floor(b)-bit fields (an unset coordinate's code, or the upper bits of a
+ *     set coordinate's code), then one word with the lowest code bit of the set
+ *     coordinates packed in order from bit 0.  Only floor(b)*32 + (coins set) bits of a
+ *     group carry information; the padding keeps packets at 128*W bytes.
  */
 #ifndef EDEN_H_
 #define EDEN_H_
@@ -79,7 +87,8 @@ typedef struct eden_client_stat {
 uint64_t eden_kept_count(uint64_t d, double bits);
 /* D = smallest power of two >= (bits >= 1 ? d : k)  (Section 5; zero padding). */
 uint64_t eden_rot_dim(uint64_t d, double bits);
-/* W = 1 for bits <= 1, else (int)bits; 0 if the budget is unsupported (Section 3). */
+/* Widest code of a client: 1 for bits <= 1, bits for integer bits, floor(bits)+1 for
+ * non-integer bits > 1; 0 if the budget is unsupported (Sections 3, 4.1). */
 uint32_t eden_code_width(double bits);
 /* bytes of one client's packed codes: ceil(D*W/32) words rounded up to a multiple of 16 bytes
  * (Section 2.2.1: ceil(log2 |I|) * d bits). */

@@ -46,15 +46,26 @@ extern "C" uint32_t eden_code_width(double bits)
 {
     if (!(bits > 0.0)) return 0;
     if (bits <= 1.0) return 1;
-    if (bits > 8.0 || bits != std::floor(bits)) return 0;
-    return (uint32_t)bits;
+    if (bits > 8.0) return 0;
+    if (bits == std::floor(bits)) return (uint32_t)bits;
+    return (uint32_t)std::floor(bits) + 1;     // non-integer: the wider of the two tables
+}
+
+// 0 for integer and sub-bit budgets, else round(frac(b) * 65536) clamped to [1, 65535]
+static uint32_t coin_threshold(double bits)
+{
+    if (bits <= 1.0 || bits == std::floor(bits)) return 0;
+    uint32_t t = (uint32_t)std::floor((bits - std::floor(bits)) * 65536.0 + 0.5);
+    return std::min(std::max(t, 1u), 65535u);
 }
 
 extern "C" uint64_t eden_code_bytes(uint64_t d, double bits)
 {
     const uint64_t D = eden_rot_dim(d, bits);
-    const uint64_t bytes = ((D * eden_code_width(bits) + 31) / 32) * 4;
-    return (bytes + 15) / 16 * 16;
+    const uint64_t W = eden_code_width(bits);
+    // integer budgets: one bit stream; non-integer: groups of 32 coordinates padded to W words
+    const uint64_t words = coin_threshold(bits) ? ((D + 31) / 32) * W : (D * W + 31) / 32;
+    return (words * 4 + 15) / 16 * 16;
 }
 
 extern "C" uint64_t eden_num_packets(uint64_t d, double bits)
@@ -361,6 +372,7 @@ struct ClientPlan {
     int L, W;
     bool subbit;
     bool needs_work;
+    uint32_t coin_thr;   // non-integer b > 1
 };
 
 // A set of clients of one rotation dimension launched together.
@@ -368,6 +380,7 @@ struct Group {
     std::vector<uint32_t> members;   // indices into the plan array
     int L;
     bool subbit;
+    bool fractional;                 // non-integer budgets b > 1 (shape-generic kernels only)
 };
 
 struct CallLayout {
@@ -389,6 +402,7 @@ int plan_clients(uint64_t d, uint32_t n, const double* bits, std::vector<ClientP
         p.L = ceil_log2(p.D);
         p.W = (int)W;
         p.subbit = bits[c] < 1.0;
+        p.coin_thr = coin_threshold(bits[c]);
         p.needs_work = p.subbit || p.L > kGenericTileLog;
     }
     return EDEN_OK;
@@ -428,6 +442,7 @@ int make_groups(const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_b
     std::stable_sort(idx.begin(), idx.end(), [&](uint32_t a, uint32_t b) {
         if (plan[a].subbit != plan[b].subbit) return !plan[a].subbit;
         if (plan[a].L != plan[b].L) return plan[a].L > plan[b].L;
+        if ((plan[a].coin_thr != 0) != (plan[b].coin_thr != 0)) return plan[a].coin_thr == 0;
         return plan[a].W < plan[b].W;
     });
     size_t i = 0;
@@ -435,11 +450,13 @@ int make_groups(const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_b
         Group g;
         g.L = plan[idx[i]].L;
         g.subbit = plan[idx[i]].subbit;
+        g.fractional = plan[idx[i]].coin_thr != 0;
         const uint64_t need = (plan[idx[i]].needs_work ? work_buffer_bytes(plan[idx[i]].D) : 0) +
                               (g.subbit ? sel_scratch_bytes(d) : 0);
         if (need > work_bytes) return EDEN_ERR_WORKSPACE;
         uint64_t used = 0;
         while (i < idx.size() && plan[idx[i]].L == g.L && plan[idx[i]].subbit == g.subbit &&
+               (plan[idx[i]].coin_thr != 0) == g.fractional &&
                used + need <= work_bytes && g.members.size() < 32768) {
             g.members.push_back(idx[i]);
             used += need;
@@ -688,7 +705,7 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
 
 bool fast_eligible(const eden_ctx* ctx, const Group& g)
 {
-    return !ctx->force_generic && g.L > kFastTileLog && g.L <= 40;
+    return !ctx->force_generic && !g.fractional && g.L > kFastTileLog && g.L <= 40;
 }
 
 // Exact-size mask selection for one client (Section 4.1): fills the MaskSelect and the
@@ -805,6 +822,7 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
             cd.L = (uint32_t)p.L;
             cd.subbit = p.subbit;
             cd.index = p.index;
+            cd.coin_thr = p.coin_thr;
             cd.extra_scale = p.subbit ? (double)d / (double)p.k : 1.0;
             cd.mean_scale = 1.0;
             descs.push_back(cd);
@@ -918,6 +936,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             cd.L = (uint32_t)p.L;
             cd.subbit = p.subbit;
             cd.index = p.index;
+            cd.coin_thr = p.coin_thr;
             cd.extra_scale = 1.0;
             cd.mean_scale = mean ? 1.0 / (double)n : 1.0;
             descs.push_back(cd);

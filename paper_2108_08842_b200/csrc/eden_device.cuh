@@ -20,6 +20,8 @@ struct ClientDesc {
     uint32_t L;              // log2 of the rotation dimension D
     uint32_t subbit;         // 1 if b < 1
     uint32_t index;          // position of this client in the caller's arrays
+    uint32_t coin_thr;       // non-integer b > 1: coin threshold round(frac * 65536); else 0
+    uint32_t pad_;
     double extra_scale;      // encode: d/k for b < 1 (folded into S), else 1
     double mean_scale;       // decode: 1/n for the mean, 1 for accumulate
 };
@@ -73,6 +75,19 @@ __device__ __forceinline__ uint32_t sign_word(uint64_t seed, uint64_t g)
     const uint4 r = philox_stream(seed, 0u, g >> 2);
     const uint32_t w = (uint32_t)g & 3u;
     return w == 0 ? r.x : w == 1 ? r.y : w == 2 ? r.z : r.w;
+}
+
+// Coin of rotated coordinate i for a non-integer budget b > 1 (Section 4.1: the
+// coordinates that get the extra bit are picked by shared randomness): Philox stream 2,
+// call i/8 yields eight 16-bit numbers, coordinate i takes number i%8 (low half of word
+// 0, high half of word 0, ...); the coin is set iff the number is below the threshold.
+__device__ __forceinline__ bool coin_bit(uint64_t seed, uint64_t i, uint32_t threshold)
+{
+    const uint4 r = philox_stream(seed, 2u, i >> 3);
+    const uint32_t w = ((uint32_t)i >> 1) & 3u;
+    const uint32_t word = w == 0 ? r.x : w == 1 ? r.y : w == 2 ? r.z : r.w;
+    const uint32_t half = (i & 1u) ? word >> 16 : word & 0xFFFFu;
+    return half < threshold;
 }
 
 // The four 32-bit mask keys of input coordinates 4t .. 4t+3.

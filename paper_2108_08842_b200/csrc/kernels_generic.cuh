@@ -147,14 +147,22 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     extern __shared__ float s[];
     __shared__ double red[32];
     __shared__ double s_norm2;
-    __shared__ float s_tb[128], s_tv[128];
+    __shared__ float s_tb[128], s_tv[128];     // table of width W
+    __shared__ float s_tb0[64], s_tv0[64];     // table of width W - 1 (non-integer budgets)
     const ClientDesc cd = descs[blockIdx.y];
     const int T = 1 << g.lt;
     const int W = (int)cd.W, half = 1 << (W - 1);
+    const bool frac = cd.coin_thr != 0u;       // then W = floor(b) + 1
+    const int Wf = frac ? W - 1 : W;           // width of the fixed fields
     for (int j = threadIdx.x; j < half; j += blockDim.x) {
         s_tb[j] = c_pos_boundary[table_offset(W) + j];
         s_tv[j] = c_pos_value[table_offset(W) + j];
     }
+    if (frac)
+        for (int j = threadIdx.x; j < (half >> 1); j += blockDim.x) {
+            s_tb0[j] = c_pos_boundary[table_offset(W - 1) + j];
+            s_tv0[j] = c_pos_value[table_offset(W - 1) + j];
+        }
     const uint64_t base = (uint64_t)blockIdx.x << g.lt;
     if (SINGLE) {
         float local = 0.f;
@@ -180,25 +188,40 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     const int lane = threadIdx.x & 31;
     float dot = 0.f;
     const int Tr = (T + 31) & ~31;                     // whole warps take part in the reductions
-    const uint64_t total_words = (((uint64_t)1 << cd.L) * W + 31) >> 5;
+    const uint64_t D = (uint64_t)1 << cd.L;
+    const uint64_t total_words = frac ? ((D + 31) >> 5) * W : (D * W + 31) >> 5;
     for (int e = threadIdx.x; e < Tr; e += blockDim.x) {
         const float h = e < T ? s[e] : 0.f;
         const float z = h * inv_norm;
-        const int m = magnitude_index(fabsf(z), s_tb, half);
+        // non-integer budget: this coordinate uses the wider table iff its coin is set
+        const bool coin = frac && e < T && coin_bit(cd.seed, base + e, cd.coin_thr);
+        const bool wide = !frac || coin;
+        const int hw = wide ? half : half >> 1;
+        const float* tb = wide ? s_tb : s_tb0;
+        const float* tv = wide ? s_tv : s_tv0;
+        const int m = magnitude_index(fabsf(z), tb, hw);
         const bool neg = z < 0.f;
-        uint32_t code = neg ? (uint32_t)(half - 1 - m) : (uint32_t)(half + m);
-        const float q = neg ? -s_tv[m] : s_tv[m];
+        uint32_t code = neg ? (uint32_t)(hw - 1 - m) : (uint32_t)(hw + m);
+        const float q = neg ? -tv[m] : tv[m];
         if (e < T) dot = fmaf(h, q, dot); else code = 0u;
         if (!live) code = 0u;
-        // the 32 lanes hold 32 consecutive W-bit fields = W words of the bit stream:
-        // lane l's field starts at bit l*W of the group
+        // the 32 lanes hold 32 consecutive Wf-bit fields = Wf words of the bit stream:
+        // lane l's field starts at bit l*Wf of the group
+        const uint32_t field = coin ? code >> 1 : code;
         uint32_t mine = 0u;
-        for (int j = 0; j < W; ++j) {
-            const int sh = lane * W - 32 * j;
+        for (int j = 0; j < Wf; ++j) {
+            const int sh = lane * Wf - 32 * j;
             uint32_t part = 0u;
-            if (sh > -W && sh < 32) part = sh >= 0 ? code << sh : code >> (-sh);
+            if (sh > -Wf && sh < 32) part = sh >= 0 ? field << sh : field >> (-sh);
             const uint32_t word = __reduce_or_sync(0xffffffffu, part);
             if (lane == j) mine = word;
+        }
+        if (frac) {
+            // the lowest code bit of the coordinates whose coin is set, packed in order
+            const uint32_t coins = __ballot_sync(0xffffffffu, coin);
+            const int rank = __popc(coins & ((1u << lane) - 1u));
+            const uint32_t word = __reduce_or_sync(0xffffffffu, coin ? (code & 1u) << rank : 0u);
+            if (lane == Wf) mine = word;
         }
         const uint64_t widx = ((base + e) >> 5) * W + lane;
         if (lane < W && widx < total_words) cd.codes[widx] = mine;
@@ -271,20 +294,47 @@ k_dec_prep(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
 }
 
 // Value of coordinate i of the received message: centroid of its code, 0 if its packet
-// was lost (Section 4.2).  `tv` holds the 2^(W-1) positive values.
-__device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i, const float* tv)
+// was lost (Section 4.2).  Called by all 32 lanes of a warp with 32 consecutive
+// coordinates (lane = i % 32); `valid` is false for lanes beyond the vector.  `tv` holds
+// the positive values of width W, `tv0` those of width W - 1 (non-integer budgets only).
+__device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i, bool valid,
+                                                const float* tv, const float* tv0)
 {
+    const int W = (int)cd.W;
+    const bool frac = cd.coin_thr != 0u;
+    const bool coin = frac && valid && coin_bit(cd.seed, i, cd.coin_thr);
+    const uint32_t coins = frac ? __ballot_sync(0xffffffffu, coin) : 0u;
+    if (!valid) return 0.f;
     if (cd.recv) {
         const uint64_t pkt = i >> 10;
         if (!((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u)) return 0.f;
     }
-    const int W = (int)cd.W, half = 1 << (W - 1);
-    const uint64_t bit = i * W;                        // field i of the bit stream
-    const uint32_t off = (uint32_t)(bit & 31);
-    uint32_t code = cd.codes[bit >> 5] >> off;
-    if (off + W > 32) code |= cd.codes[(bit >> 5) + 1] << (32 - off);
-    code &= (1u << W) - 1u;
-    return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
+    if (!frac) {
+        const int half = 1 << (W - 1);
+        const uint64_t bit = i * W;                        // field i of the bit stream
+        const uint32_t off = (uint32_t)(bit & 31);
+        uint32_t code = cd.codes[bit >> 5] >> off;
+        if (off + W > 32) code |= cd.codes[(bit >> 5) + 1] << (32 - off);
+        code &= (1u << W) - 1u;
+        return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
+    }
+    // non-integer budget: groups of 32 coordinates, W words each: (W-1)-bit fields, then the
+    // extra bits of the coordinates whose coin is set
+    const int W0 = W - 1;
+    const uint32_t l = (uint32_t)(i & 31);
+    const uint32_t* grp = cd.codes + (i >> 5) * W;
+    const uint32_t bit = l * W0, off = bit & 31;
+    uint32_t field = grp[bit >> 5] >> off;
+    if (off + W0 > 32) field |= grp[(bit >> 5) + 1] << (32 - off);
+    field &= (1u << W0) - 1u;
+    if (coin) {
+        const int rank = __popc(coins & ((1u << l) - 1u));
+        const uint32_t code = (field << 1) | ((grp[W0] >> rank) & 1u);
+        const int half = 1 << (W - 1);
+        return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
+    }
+    const int half0 = 1 << (W0 - 1);
+    return field >= (uint32_t)half0 ? tv0[field - half0] : -tv0[half0 - 1 - field];
 }
 
 enum OutMode { OUT_WRITE = 0, OUT_ACC = 1, OUT_YHAT = 2 };
@@ -295,14 +345,18 @@ __global__ void __launch_bounds__(kGenericThreads)
 k_dec_first(const ClientDesc* __restrict__ descs, PassGeom g)
 {
     extern __shared__ float s[];
-    __shared__ float s_tv[128];
+    __shared__ float s_tv[128], s_tv0[64];
     const ClientDesc cd = descs[blockIdx.y];
     const int T = 1 << g.lt;
     const int half = 1 << (cd.W - 1);
     for (int j = threadIdx.x; j < half; j += blockDim.x) s_tv[j] = c_pos_value[table_offset(cd.W) + j];
+    if (cd.coin_thr)
+        for (int j = threadIdx.x; j < (half >> 1); j += blockDim.x)
+            s_tv0[j] = c_pos_value[table_offset(cd.W - 1) + j];
     __syncthreads();
     const uint64_t base = (uint64_t)blockIdx.x << g.lt;
-    for (int e = threadIdx.x; e < T; e += blockDim.x) s[e] = received_value(cd, base + e, s_tv);
+    // T is a multiple of 32 here (multi-pass vectors), so whole warps call received_value
+    for (int e = threadIdx.x; e < T; e += blockDim.x) s[e] = received_value(cd, base + e, true, s_tv, s_tv0);
     __syncthreads();
     tile_fwht(s, g.lt, 0, g.lt);
     for (int e = threadIdx.x; e < T; e += blockDim.x) cd.work[base + e] = s[e];
@@ -323,7 +377,7 @@ k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restric
     const ClientDesc* __restrict__ descs = descs_in + (mode == OUT_YHAT ? blockIdx.y : 0);
     const ClientState* __restrict__ states = states_in + (mode == OUT_YHAT ? blockIdx.y : 0);
     extern __shared__ float s[];
-    __shared__ float s_tv[128];
+    __shared__ float s_tv[128], s_tv0[64];
     const int T = 1 << g.lt;
     float acc[kGenericPerThread];
 #pragma unroll
@@ -336,9 +390,16 @@ k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restric
             __syncthreads();
             for (int j = threadIdx.x; j < half; j += blockDim.x)
                 s_tv[j] = c_pos_value[table_offset(cd.W) + j];
+            if (cd.coin_thr)
+                for (int j = threadIdx.x; j < (half >> 1); j += blockDim.x)
+                    s_tv0[j] = c_pos_value[table_offset(cd.W - 1) + j];
             __syncthreads();
-            for (int e = threadIdx.x; e < T; e += blockDim.x)
-                s[e] = received_value(cd, tile_coord(g, blockIdx.x, e), s_tv);
+            const int Tr = (T + 31) & ~31;               // whole warps call received_value
+            for (int e = threadIdx.x; e < Tr; e += blockDim.x) {
+                // FROM_CODES tiles are contiguous: coordinate = tile * T + e
+                const float v = received_value(cd, ((uint64_t)blockIdx.x << g.lt) + e, e < T, s_tv, s_tv0);
+                if (e < T) s[e] = v;
+            }
         } else {
             for (int e = threadIdx.x; e < T; e += blockDim.x)
                 s[e] = cd.work[tile_coord(g, blockIdx.x, e)];

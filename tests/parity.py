@@ -14,6 +14,26 @@ def unpack_codes(words: np.ndarray, D: int, W: int) -> np.ndarray:
     return (bits.reshape(D, W).astype(np.uint32) * weights).sum(axis=1).astype(np.uint32)
 
 
+def unpack_fractional(words: np.ndarray, D: int, W0: int, coins: np.ndarray) -> np.ndarray:
+    """Codes of a non-integer-budget message: groups of 32 coordinates, W0+1 words each."""
+    codes = np.zeros(D, dtype=np.int64)
+    for g in range((D + 31) // 32):
+        grp = words[g * (W0 + 1):(g + 1) * (W0 + 1)]
+        pos = 0
+        for l in range(min(32, D - 32 * g)):
+            i = 32 * g + l
+            field = 0
+            for j in range(W0):
+                b = l * W0 + j
+                field |= ((int(grp[b // 32]) >> (b % 32)) & 1) << j
+            if coins[i]:
+                codes[i] = (field << 1) | ((int(grp[W0]) >> pos) & 1)
+                pos += 1
+            else:
+                codes[i] = field
+    return codes
+
+
 def near_boundary(z: np.ndarray, W: int) -> np.ndarray:
     """|z - t| <= 1e-6 * max(1, |t|) for some interval boundary t of the 2^W-value table."""
     _, b = O.table(W)
@@ -37,6 +57,18 @@ def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, 
     ok = True
     if diff.size:
         z = O.encode(x, bits, seed, want_z=True)["z"]
+        thr = O.coin_threshold(bits)
+        if thr:
+            # non-integer budget: per-coordinate width; a boundary of either table counts
+            coins = np.array([O.coin(seed, i, thr) for i in range(D)])
+            g = unpack_fractional(gpu_words, D, W - 1, coins)
+            o = unpack_fractional(enc["codes"], D, W - 1, coins)
+            bad = np.nonzero(g != o)[0]
+            mism = int(bad.size)
+            ok = bool(np.all(near_boundary(z[bad], W) | near_boundary(z[bad], W - 1)))
+            ok = ok and bool(np.all(np.abs(g[bad] - o[bad]) == 1))
+            rel = abs(gpu_scale - enc["scale"]) / abs(enc["scale"]) if enc["scale"] != 0 else abs(gpu_scale)
+            return mism, ok, rel, enc
         g = unpack_codes(gpu_words, D, W)
         o = unpack_codes(enc["codes"], D, W)
         bad = np.nonzero(g != o)[0]

@@ -196,11 +196,23 @@ def test_sub_bit_budgets_and_mask(E, bits, d):
     run_workload(E, work)
 
 
+@pytest.mark.parametrize("bits,d", [(1.5, 100), (1.5, 40000), (2.25, 5000), (7.5, 3000), (3.75, 300000)])
+def test_non_integer_budgets(E, bits, d):
+    # Section 4.1: a shared coin per coordinate picks 2^floor(b) or 2^(floor(b)+1) values
+    n = 3
+    rng = np.random.default_rng(int(bits * 100) + d)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(d + 7, n), 0.1,
+                          lambda c: xs[c], d + 7)
+    mism, _, mean = run_workload(E, work)
+    assert mism <= 10
+
+
 def test_mixed_budgets_in_one_call(E):
     d, n = 50000, 7
     rng = np.random.default_rng(5)
     xs = rng.standard_normal((n, d)).astype(np.float32)
-    bits = np.array([0.3, 1.0, 2.0, 0.1, 4.0, 8.0, 1.0])
+    bits = np.array([0.3, 1.0, 2.0, 0.1, 4.0, 8.0, 1.5])
     work = synth.Workload("adhoc", n, d, bits, synth.client_seeds(9, n), 0.2, lambda c: xs[c], 9)
     run_workload(E, work)
 
@@ -291,7 +303,7 @@ def test_bad_arguments(E):
     ctx = _ctx(E, 1024, 2)
     x = torch.zeros(2, 1024, device="cuda")
     with pytest.raises(E.EdenError) as e:
-        ctx.encode(x, [1.5, 1.0], [1, 2])
+        ctx.encode(x, [8.5, 1.0], [1, 2])
     assert e.value.code == -2
     with pytest.raises(E.EdenError) as e:
         ctx.encode(x, [0.0, 1.0], [1, 2])

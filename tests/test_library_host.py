@@ -42,7 +42,7 @@ def test_size_rules_match_oracle(lib):
         f.argtypes = [ctypes.c_uint64, ctypes.c_double]
     lib.eden_code_width.argtypes = [ctypes.c_double]
     for d in (1, 2, 31, 32, 33, 1000, 1024, 1025, 10 ** 6, 2 ** 23, 10 ** 8):
-        for bits in (0.001, 0.1, 0.5, 0.999, 1.0, 2.0, 3.0, 4.0, 8.0):
+        for bits in (0.001, 0.1, 0.5, 0.999, 1.0, 1.5, 2.0, 2.25, 3.0, 4.0, 7.75, 8.0):
             assert lib.eden_kept_count(d, bits) == O.kept_count(d, bits)
             D = O.rot_dim(d, bits)
             assert lib.eden_rot_dim(d, bits) == D
@@ -51,7 +51,7 @@ def test_size_rules_match_oracle(lib):
             words = O.code_words(d, bits)
             cb = lib.eden_code_bytes(d, bits)
             assert cb % 16 == 0 and 4 * words <= cb < 4 * words + 16
-    for bad in (0.0, -1.0, 1.5, 2.5, 9.0, float("nan")):
+    for bad in (0.0, -1.0, 8.5, 9.0, float("nan")):
         assert lib.eden_code_width(bad) == 0
 
 
