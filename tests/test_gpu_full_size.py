@@ -97,3 +97,16 @@ def test_cfg5_full_size_sampled_clients(E):
     expect = (1 / (0.99 * eq2) - 1) * d / (1 << 27) / n
     assert abs(_nmse(mean_all.astype(np.float64), xs) - expect) < 0.05 * expect
     ctx.close()
+
+
+def test_largest_tested_dimension_2_pow_28(E):
+    # 2^28 coordinates (1 GiB of fp32): four sweeps' worth of index bits above the row pass
+    # are split 7 + 8; the oracle checks the single client coordinate by coordinate
+    d = 1 << 28
+    rng = np.random.default_rng(28)
+    x = rng.standard_normal(d, dtype=np.float32)
+    x[::4097] *= 30.0                                  # a few heavy coordinates
+    work = synth.Workload("adhoc", 1, d, np.array([1.0]), synth.client_seeds(28, 1), 0.02,
+                          lambda c: x, 28)
+    mism, _, _ = run_workload(E, work, threads=1)
+    assert mism <= 120
