@@ -422,11 +422,13 @@ int carve(const eden_ctx* ctx, uint64_t d, uint32_t n, CallLayout& lay)
 // One client's intermediate vector in the workspace; what follows it stays 256-byte aligned.
 uint64_t work_buffer_bytes(uint64_t D) { return align_up(D * sizeof(float), 256); }
 
+constexpr uint64_t kBatchHistBytes = 3ull * kSelBins * sizeof(uint32_t);
+
 // Scratch of the exact-size mask selection for one client with b < 1.
 uint64_t sel_scratch_bytes(uint64_t d)
 {
     const uint64_t n_chunks = (d + kSelChunk - 1) / kSelChunk;
-    return 256 + kHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) +
+    return 256 + kBatchHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) +
            align_up(sizeof(SelJob), 256);
 }
 
@@ -748,24 +750,26 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
     const uint64_t chunk_bytes = align_up(n_chunks * sizeof(unsigned long long), 256);
     char* sel_base = region;
     char* hist_base = sel_base + 256ull * n;
-    char* chunk_base = hist_base + kHistBytes * n;
+    char* chunk_base = hist_base + kBatchHistBytes * n;
     char* job_base = chunk_base + chunk_bytes * n;
     std::vector<SelJob> jobs(partial);
     for (uint32_t j = 0; j < n; ++j) {
         jobs[j].sel = (MaskSelect*)(sel_base + 256ull * j);
-        jobs[j].hist = (uint32_t*)(hist_base + kHistBytes * j);
+        jobs[j].hist = (uint32_t*)(hist_base + kBatchHistBytes * j);
         jobs[j].chunks = (unsigned long long*)(chunk_base + chunk_bytes * j);
     }
     batch.d_jobs = (SelJob*)job_base;
     batch.n = n;
     batch.grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
+    const unsigned hist_grid = (unsigned)(((d + 3) / 4 + (uint64_t)kSelThreads * kSelCallsPerThread - 1) /
+                                          ((uint64_t)kSelThreads * kSelCallsPerThread));
     CUDA_OK(cudaMemcpyAsync(batch.d_jobs, jobs.data(), sizeof(SelJob) * n, cudaMemcpyHostToDevice, ctx->stream));
-    CUDA_OK(cudaMemsetAsync(hist_base, 0, kHistBytes * n, ctx->stream));
+    CUDA_OK(cudaMemsetAsync(hist_base, 0, kBatchHistBytes * n, ctx->stream));
     const double keys = (double)n * (double)d;
-    LAUNCH(ctx, "sel_hist", 0, k_selb_hist, dim3(batch.grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs, 0);
-    LAUNCH(ctx, "sel_find", n * 65536.0 * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, 0);
-    LAUNCH(ctx, "sel_hist", 0, k_selb_hist, dim3(batch.grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs, 1);
-    LAUNCH(ctx, "sel_find", n * 65536.0 * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, 1);
+    for (int round = 0; round < 3; ++round) {
+        LAUNCH(ctx, "sel_hist", 0, k_selb_hist, dim3(hist_grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs, round);
+        LAUNCH(ctx, "sel_find", n * (double)kSelBins * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, round);
+    }
     LAUNCH(ctx, "sel_chunk_count", keys / 128.0, k_selb_chunk_count, dim3(batch.grid, n), kSelThreads, 0,
            (const SelJob*)batch.d_jobs);
     LAUNCH(ctx, "sel_chunk_scan", keys / 64.0, k_selb_chunk_scan, n, 1024, 0, (const SelJob*)batch.d_jobs,

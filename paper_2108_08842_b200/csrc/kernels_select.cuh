@@ -210,35 +210,126 @@ k_sel_apply(uint64_t seed, uint64_t d, const MaskSelect* __restrict__ sel,
 struct SelJob {
     uint64_t seed, d, k;
     MaskSelect* sel;
-    uint32_t* hist;                  // 2 x 65536 bins
+    uint32_t* hist;                  // three 2048-bin histograms (one per digit round)
     unsigned long long* chunks;      // one packed count per 1024 coordinates
     const float* in;                 // compact: the client's input row; scatter: its estimate of the kept coordinates
     float* out;                      // compact: the compacted vector
 };
 
+// Batched selection finds the k-th smallest key in three digit rounds of 10, 11 and 11
+// bits with histograms of up to 2048 bins (job.hist holds three of them).  Round 0 sees every key,
+// so each block counts a long run of keys in shared memory and adds its non-empty bins to
+// the global histogram once; rounds 1 and 2 only see the keys that share the digits found
+// so far (one in 1024, one in two million) and count them in global memory directly.
+// sel->bin_hi carries the digits found so far, sel->below_hi the keys below them.
+constexpr int kSelBins = 2048;
+constexpr int kSelCallsPerThread = 32;     // Philox calls (4 keys each) per thread and block in a histogram round
+
+__device__ __forceinline__ int sel_digit_shift(int round) { return round == 0 ? 22 : round == 1 ? 11 : 0; }
+__device__ __forceinline__ int sel_digit_bits(int round) { return round == 0 ? 10 : 11; }
+
 __global__ void __launch_bounds__(kSelThreads)
 k_selb_hist(const SelJob* __restrict__ jobs, int round)
 {
+    __shared__ uint32_t s_hist[kSelBins];
     const SelJob job = jobs[blockIdx.y];
-    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t * 4 >= job.d) return;
-    const uint4 k4 = mask_keys(job.seed, t);
-    const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
-    const uint32_t want = round ? job.sel->bin_hi : 0u;
-    uint32_t* hist = job.hist + (round ? 65536 : 0);
+    uint32_t* hist = job.hist + round * kSelBins;
+    const uint64_t calls = (job.d + 3) / 4;
+    const uint64_t first = (uint64_t)blockIdx.x * kSelThreads * kSelCallsPerThread;
+    if (first >= calls) return;
+    const int shift = sel_digit_shift(round);
+    const uint32_t mask = (1u << sel_digit_bits(round)) - 1u;
+    const uint32_t prefix = round ? job.sel->bin_hi : 0u;
+    const int pshift = shift + sel_digit_bits(round);         // bits above this digit
+    if (round == 0)
+        for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) s_hist[b] = 0u;
+    __syncthreads();
+    for (int it = 0; it < kSelCallsPerThread; ++it) {
+        const uint64_t t = first + (uint64_t)it * kSelThreads + threadIdx.x;
+        if (t >= calls) break;
+        const uint4 k4 = mask_keys(job.seed, t);
+        const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        if (t * 4 + j >= job.d) break;
-        if (round == 0) atomicAdd(&hist[keys[j] >> 16], 1u);
-        else if ((keys[j] >> 16) == want) atomicAdd(&hist[keys[j] & 0xFFFFu], 1u);
+        for (int j = 0; j < 4; ++j) {
+            if (t * 4 + j >= job.d) break;
+            if (round == 0) atomicAdd(&s_hist[keys[j] >> shift], 1u);
+            else if ((keys[j] >> pshift) == prefix) atomicAdd(&hist[(keys[j] >> shift) & mask], 1u);
+        }
+    }
+    if (round == 0) {
+        __syncthreads();
+        for (int b = threadIdx.x; b < kSelBins; b += kSelThreads)
+            if (s_hist[b]) atomicAdd(&hist[b], s_hist[b]);
     }
 }
 
+// One block per job: the bin of the current round's histogram that holds rank
+// k - 1 - (keys below the digits found so far); extends the digits, and after the last
+// round writes tau, below and rem.
 __global__ void __launch_bounds__(1024)
 k_selb_find(const SelJob* __restrict__ jobs, int round)
 {
+    __shared__ uint32_t warp_total[32];
+    __shared__ uint32_t warp_before[32];
     const SelJob job = jobs[blockIdx.x];
-    sel_find_body(job.hist + (round ? 65536 : 0), job.k, round, job.sel);
+    MaskSelect* sel = job.sel;
+    const uint32_t* hist = job.hist + round * kSelBins;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t below_so_far = round ? sel->below_hi : 0u;
+    const uint32_t prefix = round ? sel->bin_hi : 0u;
+    const uint32_t r = (uint32_t)(job.k - 1) - below_so_far;
+    // warp w owns bins [64 w, 64 w + 64)
+    const uint32_t* run = hist + warp * 64;
+    uint32_t v[2], mine = 0;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) { v[i] = run[i * 32 + lane]; mine += v[i]; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if (lane == 0) warp_total[warp] = mine;
+    __syncthreads();
+    if (warp == 0) {
+        const uint32_t w = warp_total[lane];
+        uint32_t inc = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += t;
+        }
+        warp_before[lane] = inc - w;
+    }
+    __syncthreads();
+    const uint32_t before = warp_before[warp];
+    if (r >= before && r < before + warp_total[warp]) {        // exactly one warp
+        uint32_t seen = before;
+        for (int i = 0; i < 2; ++i) {
+            uint32_t inc = v[i];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += t;
+            }
+            const uint32_t chunk_total = __shfl_sync(0xffffffffu, inc, 31);
+            if (r < seen + chunk_total) {
+                const uint32_t hit = __ballot_sync(0xffffffffu, r < seen + inc);
+                const int firstl = __ffs(hit) - 1;
+                if (lane == firstl) {
+                    const uint32_t bin = (uint32_t)(warp * 64 + i * 32 + lane);
+                    const uint32_t below = below_so_far + seen + inc - v[i];
+                    const uint32_t digits = (prefix << sel_digit_bits(round)) | bin;
+                    if (round < 2) {
+                        sel->bin_hi = digits;
+                        sel->below_hi = below;
+                    } else {
+                        sel->tau = digits;
+                        sel->below = below;
+                        sel->rem = (uint32_t)job.k - below;        // ties to keep, >= 1
+                    }
+                }
+                break;
+            }
+            seen += chunk_total;
+        }
+    }
 }
 
 __global__ void __launch_bounds__(kSelThreads)
