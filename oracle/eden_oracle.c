@@ -241,7 +241,12 @@ static int g_have[9];
 static void table_for_width(uint32_t W, const double **cent, const double **bound)
 {
     if (!g_have[W]) {
-        eden_oracle_lloyd_max(1u << W, g_cent[W], g_bound[W]);
+        /* solve into locals and publish afterwards: two threads that both find the cache
+           empty then store identical tables instead of one reading a half-built one */
+        double c[256], b[255];
+        eden_oracle_lloyd_max(1u << W, c, b);
+        memcpy(g_cent[W], c, sizeof(double) * (1u << W));
+        memcpy(g_bound[W], b, sizeof(double) * ((1u << W) - 1u));
         g_have[W] = 1;
     }
     *cent = g_cent[W];
