@@ -19,8 +19,8 @@
  *   - Section 5:     the rotation is the randomized Hadamard transform
  *                    R = (1/sqrt D) H_D Diag(s).
  *
- * Conventions the paper leaves open (all are this build's reading, stated in the
- * design notes; the ones marked [unpinned] are pinned only by oracle == GPU):
+ * Conventions the paper leaves open (all are this build's reading; the ones marked
+ * [unpinned] are pinned only by oracle == GPU):
  *   - H is the Sylvester matrix H[i][j] = (-1)^popcount(i & j); one transform.
  *   - d that is not a power of two is zero-padded to D = 2^ceil(log2 d'); all D
  *     rotated coordinates are coded; the estimate is truncated back.

@@ -6,7 +6,8 @@
 // steps the tile is transposed through shared memory with 64- or 128-bit conflict-free
 // accesses; global loads and stores are 64- or 128-bit and fully coalesced.
 //
-//  * column pass (k_f_enc_first, k_f_mid, k_f_dec_last): the tile is 2^LR rows of
+//  * column pass (k_f_col: the sender's first pass and the in-place middle passes;
+//    k_f_dec_last: the receiver's last pass): the tile is 2^LR rows of
 //    8192/2^LR consecutive coordinates, rows 2^lo apart; the LR row bits are transformed.
 //    Values travel as float4 (four neighbouring columns), so every stage is two packed
 //    instructions per float4 pair.
@@ -18,8 +19,10 @@
 //    tiles that differ in the LC index bits just above the block's own; those stages are
 //    done by one exchange through distributed shared memory: every block fetches its
 //    1/2^LC slice of all tiles of the cluster, does the LC stages in registers and writes
-//    the results where they belong.  This is what lets 2^24 .. 2^27 coordinates be
-//    transformed in two sweeps over HBM instead of three.
+//    the results where they belong.  That transforms 2^24 .. 2^27 coordinates in two
+//    sweeps over HBM instead of three, but on B200 the two cluster barriers per tile cost
+//    more than the sweep they save, so the default plan launches every kernel with LC = 0
+//    and the cluster forms are a tuning option.
 #pragma once
 #include "eden_device.cuh"
 #include "kernels_generic.cuh"
