@@ -459,8 +459,9 @@ k_f_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restr
 //   B: u = (t >> 4) << 8 | k << 4 | (t & 15)      registers hold u bits 7..4 (e bits 8..5)
 //   C: u = t << 4 | k            registers hold u bits 3..0  (e bits 4..1): the thread
 //                                owns the 32 consecutive coordinates 32 t .. 32 t + 31
-// Shared memory holds unit u at u + (u >> 4) (one pad per 16), conflict-free for the
-// 64-bit accesses of all three arrangements.
+// Shared memory holds unit u at u + 2 (u >> 4) (two pads per 16): conflict-free for the
+// 64-bit accesses of arrangements A and B, and arrangement C's 16 consecutive units stay
+// 16-byte aligned, so C moves them with eight 128-bit accesses.
 // With a cluster (LC > 0) the 2^LC tiles of the cluster are consecutive in memory and the
 // LC index bits above the tile are exchanged in the "slice" arrangement: register k holds
 // unit rank * (4096 >> LC) + t + 256 * (k mod (16 >> LC)) of the tile of rank k / (16 >> LC).
@@ -472,8 +473,8 @@ __device__ __forceinline__ int row_u(int t, int k)
     if (ARR == 1) return ((t >> 4) << 8) | (k << 4) | (t & 15);
     return (t << 4) | k;
 }
-__device__ __forceinline__ int row_pad(int u) { return u + (u >> 4); }
-constexpr int kRowSmemUnits = 4096 + 256;
+__device__ __forceinline__ int row_pad(int u) { return u + 2 * (u >> 4); }
+constexpr int kRowSmemUnits = 4096 + 512;
 
 template <int LC>
 __device__ __forceinline__ int slice_u(int rank, int t, int k)
@@ -485,11 +486,27 @@ template <int FROM, int TO>
 __device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
 {
     const int t = threadIdx.x;
+    if (FROM == 2) {
+        ulonglong2* p = reinterpret_cast<ulonglong2*>(s + row_pad(row_u<2>(t, 0)));
 #pragma unroll
-    for (int k = 0; k < 16; ++k) s[row_pad(row_u<FROM>(t, k))] = v[k];
+        for (int k = 0; k < 8; ++k) p[k] = make_ulonglong2(v[2 * k], v[2 * k + 1]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) s[row_pad(row_u<FROM>(t, k))] = v[k];
+    }
     __syncthreads();
+    if (TO == 2) {
+        const ulonglong2* p = reinterpret_cast<const ulonglong2*>(s + row_pad(row_u<2>(t, 0)));
 #pragma unroll
-    for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<TO>(t, k))];
+        for (int k = 0; k < 8; ++k) {
+            const ulonglong2 w = p[k];
+            v[2 * k] = w.x;
+            v[2 * k + 1] = w.y;
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<TO>(t, k))];
+    }
 }
 
 // butterflies over register index bits [B0, 4) of 16 packed units
@@ -552,6 +569,22 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
                                                  uint32_t (&words)[W], float& dot)
 {
     constexpr uint32_t half = 1u << (W - 1);
+    if constexpr (W == 1) {
+        // one bit per coordinate: the code is "not negative" and Q(|z|) is the same value
+        // for every coordinate, so shift the sign bits in (coordinate 31 first) and sum |h|
+        uint32_t negs = 0u;
+        float sum = 0.f;
+#pragma unroll
+        for (int k = 15; k >= 0; --k) {
+            float h0, h1;
+            unpack2(v[k], h0, h1);
+            negs = __funnelshift_l(__float_as_uint(h1), negs, 1);
+            negs = __funnelshift_l(__float_as_uint(h0), negs, 1);
+            sum += fabsf(h0) + fabsf(h1);
+        }
+        dot = sum * c_pos_value[0];
+        words[0] = live ? ~negs : 0u;
+    } else {
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = 0u;
 #pragma unroll
@@ -575,13 +608,14 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
 #pragma unroll
         for (int j = 0; j < W; ++j) words[j] = 0u;
     }
+    }   // W > 1
 }
 
 template <int W, int LC>
 __global__ void __launch_bounds__(kFastThreads, 4)
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
 {
-    __shared__ u64 s[kRowSmemUnits];
+    __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ double red[32];
     __shared__ float s_tb[128], s_tv[128];
     const ClientDesc cd = descs[blockIdx.y];
@@ -648,7 +682,7 @@ template <int W, int LC>
 __global__ void __launch_bounds__(kFastThreads, 4)
 k_f_dec_first(const ClientDesc* __restrict__ descs)
 {
-    __shared__ u64 s[kRowSmemUnits];
+    __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ float s_val[2 << W];                    // the 2^W values by code, then 2^W zeros
     const ClientDesc cd = descs[blockIdx.y];
     const int t = threadIdx.x;
@@ -671,18 +705,29 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = src[j];
     u64 v[16];
+    if (W == 1) {
+        // one bit per coordinate: +-c (or +-0 for a lost packet) by moving the bit into the sign
+        const uint32_t minus_c = __float_as_uint(tbl[0]) | 0x80000000u;
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
-        float q[2];
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int l = 2 * k + e;
-            const int a = (l * W) >> 5, off = (l * W) & 31;
-            uint32_t code = words[a] >> off;
-            if (off + W > 32) code |= words[a + 1] << (32 - off);
-            q[e] = tbl[code & ((1u << W) - 1u)];
+        for (int k = 0; k < 16; ++k) {
+            const uint32_t b0 = (words[0] << (31 - 2 * k)) & 0x80000000u;
+            const uint32_t b1 = (words[0] << (30 - 2 * k)) & 0x80000000u;
+            v[k] = pack2(__uint_as_float(minus_c ^ b0), __uint_as_float(minus_c ^ b1));
         }
-        v[k] = pack2(q[0], q[1]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            float q[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int l = 2 * k + e;
+                const int a = (l * W) >> 5, off = (l * W) & 31;
+                uint32_t code = words[a] >> off;
+                if (off + W > 32) code |= words[a + 1] << (32 - off);
+                q[e] = tbl[code & ((1u << W) - 1u)];
+            }
+            v[k] = pack2(q[0], q[1]);
+        }
     }
     row_step_inner(v);              // e bit 0
     row_step<0>(v);                 // e bits 4..1
