@@ -613,6 +613,9 @@ cudaError_t launch_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, int 
         default: return EDEN_ERR_INVALID_ARG;     \
     }
 
+#define EDEN_DISPATCH_FRAC(frac, CALL)            \
+    if (frac) { constexpr bool FRAC_ = true; CALL; } else { constexpr bool FRAC_ = false; CALL; }
+
 #define EDEN_DISPATCH_W(w, CALL)                  \
     switch (w) {                                  \
         case 1: { constexpr int W_ = 1; CALL; } break; \
@@ -662,10 +665,10 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
-        EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
-            LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_>),
+        EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
+            LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_, FRAC_>),
                       dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
-                      (const ClientDesc*)(d_descs + r.first), d_states + r.first)));
+                      (const ClientDesc*)(d_descs + r.first), d_states + r.first))));
     }
     return EDEN_OK;
 }
@@ -681,10 +684,10 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
-        EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
-            LAUNCH_CL(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, (k_f_dec_first<W_, LC_>),
+        EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
+            LAUNCH_CL(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, (k_f_dec_first<W_, LC_, FRAC_>),
                       dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
-                      (const ClientDesc*)(d_descs + r.first))));
+                      (const ClientDesc*)(d_descs + r.first)))));
     }
     // the receiver walks the column ranges bottom-up so that the top range comes last
     for (size_t pi = pl.cols.size(); pi-- > 0;) {
@@ -707,7 +710,7 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
 
 bool fast_eligible(const eden_ctx* ctx, const Group& g)
 {
-    return !ctx->force_generic && !g.fractional && g.L > kFastTileLog && g.L <= 40;
+    return !ctx->force_generic && g.L > kFastTileLog && g.L <= 40;
 }
 
 // Exact-size mask selection for one client (Section 4.1): fills the MaskSelect and the

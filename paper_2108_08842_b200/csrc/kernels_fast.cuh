@@ -611,13 +611,84 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
     }   // W > 1
 }
 
-template <int W, int LC>
+// ---------------------------------------------------------------------------------
+// Non-integer budgets b > 1 (Section 4.1) on the row pass: the thread owns one group of 32
+// coordinates; W = floor(b) + 1 words per group: (W-1)-bit fields, then the lowest code
+// bit of the coordinates whose coin is set, packed in order.
+// ---------------------------------------------------------------------------------
+// coins of the 32 coordinates of group g: four Philox calls of eight 16-bit numbers each
+__device__ __forceinline__ uint32_t group_coins(uint64_t seed, uint64_t g, uint32_t threshold)
+{
+    uint32_t coins = 0u;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint4 r = philox_stream(seed, 2u, 4 * g + c);
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            coins |= ((w[j] & 0xFFFFu) < threshold ? 1u : 0u) << (8 * c + 2 * j);
+            coins |= ((w[j] >> 16) < threshold ? 1u : 0u) << (8 * c + 2 * j + 1);
+        }
+    }
+    return coins;
+}
+
+// tb_hi/tv_hi: positive boundaries and values of width W; tb_lo/tv_lo: of width W - 1
+template <int W>
+__device__ __forceinline__ void quantise_pack_frac(const u64 (&v)[16], float inv_norm, bool live, uint32_t coins,
+                                                   const float* tb_hi, const float* tv_hi,
+                                                   const float* tb_lo, const float* tv_lo,
+                                                   uint32_t (&words)[W], float& dot)
+{
+    constexpr int W0 = W - 1;
+#pragma unroll
+    for (int j = 0; j < W; ++j) words[j] = 0u;
+    uint32_t pos = 0u;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        float h[2];
+        unpack2(v[k], h[0], h[1]);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int l = 2 * k + e;
+            const bool wide = (coins >> l) & 1u;
+            const int hw = wide ? (1 << W0) : (1 << W0) >> 1;       // half the number of values
+            const float* tb = wide ? tb_hi : tb_lo;
+            const float* tv = wide ? tv_hi : tv_lo;
+            const float z = h[e] * inv_norm;
+            const float az = fabsf(z);
+            int m = 0;
+#pragma unroll
+            for (int it = 0; it < W0; ++it) {
+                const int step = (1 << (W0 - 1)) >> it;
+                if (step < hw) m += (az > tb[m + step - 1]) ? step : 0;
+            }
+            dot = fmaf(fabsf(h[e]), tv[m], dot);
+            const uint32_t code = (uint32_t)m ^ (z < 0.f ? (uint32_t)hw - 1u : (uint32_t)hw);
+            const uint32_t field = wide ? code >> 1 : code;
+            const int a = (l * W0) >> 5, off = (l * W0) & 31;
+            words[a] |= field << off;
+            if (off + W0 > 32) words[a + 1] |= field >> (32 - off);
+            if (wide) {
+                words[W0] |= (code & 1u) << pos;
+                ++pos;
+            }
+        }
+    }
+    if (!live) {
+#pragma unroll
+        for (int j = 0; j < W; ++j) words[j] = 0u;
+    }
+}
+
+template <int W, int LC, bool FRAC>
 __global__ void __launch_bounds__(kFastThreads, 4)
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ double red[32];
     __shared__ float s_tb[128], s_tv[128];
+    __shared__ float s_tb0[FRAC ? 64 : 1], s_tv0[FRAC ? 64 : 1];   // width W - 1 (non-integer budgets)
     const ClientDesc cd = descs[blockIdx.y];
     const int t = threadIdx.x;
     constexpr int half = 1 << (W - 1);
@@ -625,6 +696,11 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
         s_tb[j] = c_pos_boundary[table_offset(W) + j];
         s_tv[j] = c_pos_value[table_offset(W) + j];
     }
+    if (FRAC)
+        for (int j = t; j < (half >> 1); j += kFastThreads) {
+            s_tb0[j] = c_pos_boundary[table_offset(W > 1 ? W - 1 : 1) + j];
+            s_tv0[j] = c_pos_value[table_offset(W > 1 ? W - 1 : 1) + j];
+        }
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
     u64 v[16];
     if (LC == 0) {
@@ -667,7 +743,12 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
     const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
     uint32_t words[W];
     float dot = 0.f;
-    quantise_pack_32<W>(v, inv_norm, live, s_tb, s_tv, words, dot);
+    if constexpr (FRAC && W >= 2) {
+        const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
+        quantise_pack_frac<W>(v, inv_norm, live, coins, s_tb, s_tv, s_tb0, s_tv0, words, dot);
+    } else {
+        quantise_pack_32<W>(v, inv_norm, live, s_tb, s_tv, words, dot);
+    }
     uint32_t* dst = cd.codes + ((base >> 5) + t) * W;
 #pragma unroll
     for (int j = 0; j < W; ++j) dst[j] = words[j];
@@ -678,12 +759,13 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
 // =================================================================================
 // Receiver, first pass: codes -> centroids (lost packets -> 0) -> low stages -> work
 // =================================================================================
-template <int W, int LC>
+template <int W, int LC, bool FRAC>
 __global__ void __launch_bounds__(kFastThreads, 4)
 k_f_dec_first(const ClientDesc* __restrict__ descs)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ float s_val[2 << W];                    // the 2^W values by code, then 2^W zeros
+    __shared__ float s_val0[FRAC ? (1 << W) : 1];      // the same for width W - 1 (non-integer budgets)
     const ClientDesc cd = descs[blockIdx.y];
     const int t = threadIdx.x;
     constexpr int half = 1 << (W - 1);
@@ -693,6 +775,14 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
                                          : -c_pos_value[table_offset(W) + half - 1 - j];
         s_val[j] = c;
     }
+    if (FRAC && W >= 2)
+        for (int j = t; j < (1 << W); j += kFastThreads) {
+            constexpr int h0 = half >> 1;
+            float c = 0.f;
+            if (j < (1 << (W - 1))) c = j >= h0 ? c_pos_value[table_offset(W > 1 ? W - 1 : 1) + j - h0]
+                                                : -c_pos_value[table_offset(W > 1 ? W - 1 : 1) + h0 - 1 - j];
+            s_val0[j] = c;
+        }
     __syncthreads();
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
     // the tile is 8 packets of 1024 coordinates; this thread's 32 coordinates lie in one.
@@ -705,7 +795,30 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = src[j];
     u64 v[16];
-    if (W == 1) {
+    if constexpr (FRAC && W >= 2) {
+        // non-integer budget: (W-1)-bit fields, then the extra bits of the coordinates whose coin is set
+        constexpr int W0 = W - 1;
+        const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
+        const float* tbl0 = s_val0 + (arrived ? 0 : (1 << W0));
+        uint32_t pos = 0u;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            float q[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int l = 2 * k + e;
+                const int a = (l * W0) >> 5, off = (l * W0) & 31;
+                uint32_t field = words[a] >> off;
+                if (off + W0 > 32) field |= words[a + 1] << (32 - off);
+                field &= (1u << W0) - 1u;
+                const bool wide = (coins >> l) & 1u;
+                const uint32_t code = (field << 1) | ((words[W0] >> pos) & 1u);
+                q[e] = wide ? tbl[code] : tbl0[field];
+                pos += wide ? 1u : 0u;
+            }
+            v[k] = pack2(q[0], q[1]);
+        }
+    } else if (W == 1) {
         // one bit per coordinate: +-c (or +-0 for a lost packet) by moving the bit into the sign
         const uint32_t minus_c = __float_as_uint(tbl[0]) | 0x80000000u;
 #pragma unroll
