@@ -208,6 +208,16 @@ def test_non_integer_budgets(E, bits, d):
     assert mism <= 10
 
 
+def test_many_small_clients(E):
+    # thousands of independent senders in one call (one block per client)
+    d, n = 300, 3000
+    rng = np.random.default_rng(77)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    bits = rng.choice(np.array([1.0, 2.0, 3.0]), size=n)
+    work = synth.Workload("adhoc", n, d, bits, synth.client_seeds(77, n), 0.0, lambda c: xs[c], 77)
+    run_workload(E, work)
+
+
 def test_mixed_budgets_in_one_call(E):
     d, n = 50000, 7
     rng = np.random.default_rng(5)
