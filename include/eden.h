@@ -102,6 +102,13 @@ uint64_t eden_recv_mask_words(uint64_t d, double bits);
  * accepted as long as it holds one client: calls then run in several groups. */
 uint64_t eden_workspace_bytes(uint64_t d_max, uint32_t n_batch);
 
+/* The sweeps over HBM that one client's rotation (Section 5) takes for (d, bits) on the
+ * default kernels, sender order: pass_bits[0..*n_passes) = index bits each sweep
+ * transforms (they add up to log2 D); the last entry is the sweep that reads or writes
+ * the codes.  Host only; pass_bits holds max_passes entries. */
+int eden_pass_plan(uint64_t d, double bits, uint32_t* pass_bits, uint32_t max_passes,
+                   uint32_t* n_passes);
+
 /* The quantiser the library uses for code width W (1..8): 2^W values in ascending
  * order and the 2^W - 1 interval boundaries between them, rounded to fp32
  * (Section 3: Lloyd-Max for N(0,1), centre-of-mass values).  Host arrays, host only. */

@@ -782,6 +782,27 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
 
 }  // namespace
 
+// How one client's transform is split into sweeps over HBM (host only).
+extern "C" int eden_pass_plan(uint64_t d, double bits, uint32_t* pass_bits, uint32_t max_passes,
+                              uint32_t* n_passes)
+{
+    if (!pass_bits || !n_passes || d == 0 || d > EDEN_MAX_DIM || eden_code_width(bits) == 0)
+        return EDEN_ERR_INVALID_ARG;
+    const int L = ceil_log2(eden_rot_dim(d, bits));
+    std::vector<uint32_t> out;
+    if (L <= kGenericTileLog) {
+        out.push_back((uint32_t)L);                       // one block per client
+    } else {
+        const FastPlan pl = fast_plan(L, 0);
+        for (const FastPass& ps : pl.cols) out.push_back((uint32_t)(ps.lr + ps.lc));
+        out.push_back((uint32_t)(kFastTileLog + pl.row_lc));
+    }
+    if (out.size() > max_passes) return EDEN_ERR_INVALID_ARG;
+    std::copy(out.begin(), out.end(), pass_bits);
+    *n_passes = (uint32_t)out.size();
+    return EDEN_OK;
+}
+
 // ------------------------------------------------------------------------------------
 // sender
 // ------------------------------------------------------------------------------------

@@ -47,6 +47,7 @@ _sig("eden_recv_mask_words", _u64, [_u64, _f64])
 _sig("eden_workspace_bytes", _u64, [_u64, _u32])
 _sig("eden_host_workspace_bytes", _u64, [_u64, _u32])
 _sig("eden_table", _int, [_u32, _vp, _vp])
+_sig("eden_pass_plan", _int, [_u64, _f64, _vp, _u32, ctypes.POINTER(_u32)])
 _sig("eden_create", _int, [ctypes.POINTER(_vp), _int, _vp, _vp, _u64])
 _sig("eden_destroy", _int, [_vp])
 _sig("eden_encode", _int, [_vp, _vp, _u64, _u64, _u32, _vp, _vp, _vp, _vp])
@@ -112,6 +113,14 @@ def workspace_bytes(d_max: int, n_batch: int) -> int:
 
 def host_workspace_bytes(d: int, n: int) -> int:
     return int(_lib.eden_host_workspace_bytes(d, n))
+
+
+def pass_plan(d: int, bits: float):
+    """Index bits transformed by each sweep over HBM for one client (sender order)."""
+    buf = (_u32 * 8)()
+    n = _u32(0)
+    _check(_lib.eden_pass_plan(d, bits, buf, 8, ctypes.byref(n)))
+    return list(buf[: n.value])
 
 
 def table(W: int):

@@ -105,3 +105,30 @@ def test_binding_refuses_to_run_without_cuda():
     from paper_2108_08842_b200 import eden
     with pytest.raises(RuntimeError):
         eden.Context(0)
+
+
+def test_pass_plan_covers_every_index_bit(lib):
+    lib.eden_pass_plan.argtypes = [ctypes.c_uint64, ctypes.c_double, ctypes.c_void_p, ctypes.c_uint32,
+                                   ctypes.POINTER(ctypes.c_uint32)]
+    buf = (ctypes.c_uint32 * 8)()
+    n = ctypes.c_uint32(0)
+    for L in range(0, 31):
+        d = 1 << L
+        assert lib.eden_pass_plan(d, 1.0, buf, 8, ctypes.byref(n)) == 0
+        passes = list(buf[: n.value])
+        assert sum(passes) == L
+        if L <= 13:
+            assert passes == [L]
+        else:
+            assert passes[-1] == 13 and all(1 <= p <= 8 for p in passes[:-1])
+            assert len(passes) == 1 + -(-(L - 13) // 8)            # fewest sweeps with 8-bit column passes
+            assert passes[0] == min(passes[:-1])                   # the sweep over the fp32 vectors is the narrowest
+            assert all(p == 8 for p in passes[1:-1])
+    # the benchmark configurations
+    for d, bits, want in ((1 << 24, 1.0, [3, 8, 13]), (10 ** 8, 4.0, [6, 8, 13]), (1 << 20, 2.0, [7, 13]),
+                          (1 << 23, 0.1, [7, 13]), (1024, 1.0, [10])):
+        assert lib.eden_pass_plan(d, bits, buf, 8, ctypes.byref(n)) == 0
+        assert list(buf[: n.value]) == want
+    assert lib.eden_pass_plan(0, 1.0, buf, 8, ctypes.byref(n)) == -1
+    assert lib.eden_pass_plan(1 << 20, 9.0, buf, 8, ctypes.byref(n)) == -1
+    assert lib.eden_pass_plan(1 << 30, 1.0, buf, 2, ctypes.byref(n)) == -1
