@@ -194,7 +194,10 @@ int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stream, uint64_
 
 /* x, codes (array of n host pointers), scales are HOST buffers (pinned memory makes the
  * copies asynchronous).  Copies x to the device, encodes, copies codes and scales back
- * and synchronises the stream.  Needs eden_host_workspace_bytes() of workspace. */
+ * and synchronises the stream.  Needs eden_host_workspace_bytes() of workspace.  Inputs
+ * of 64 MiB and more are processed in chunks of clients on two internal side streams so
+ * that uploads, kernels and downloads overlap; eden_client_stats then describes the last
+ * chunk only. */
 int eden_encode_host(eden_ctx* ctx, const float* x_host, uint64_t ld_x, uint64_t d, uint32_t n,
                      const double* bits, const uint64_t* seeds,
                      uint8_t* const* codes_host, float* scales_host);

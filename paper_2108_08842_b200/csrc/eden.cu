@@ -196,6 +196,9 @@ struct eden_ctx {
     std::vector<ProfileRecord> records;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
     std::vector<ProfileSummary> summary;
+    // host-buffer entry points: side streams and events for overlapping copies with kernels
+    cudaStream_t copy_in, copy_out;
+    std::vector<cudaEvent_t> sync_events;
 };
 
 static void profile_begin(eden_ctx* ctx, const char* name, double bytes)
@@ -251,6 +254,8 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->launches = 0;
     ctx->states_off = 0;
     ctx->profiling = false;
+    ctx->copy_in = nullptr;
+    ctx->copy_out = nullptr;
     ctx->force_generic = false;
     ctx->plan_variant = 0;
     if (const char* pv = std::getenv("EDEN_PLAN_VARIANT")) ctx->plan_variant = std::atoi(pv);
@@ -273,6 +278,9 @@ extern "C" int eden_destroy(eden_ctx* ctx)
         cudaEventDestroy(e.first);
         cudaEventDestroy(e.second);
     }
+    for (cudaEvent_t e : ctx->sync_events) cudaEventDestroy(e);
+    if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+    if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     delete ctx;
     return EDEN_OK;
 }
@@ -1129,9 +1137,60 @@ extern "C" int eden_encode_host(eden_ctx* ctx, const float* x_host, uint64_t ld_
         codes_dev[c] = (uint8_t*)st.take(eden_code_bytes(d, bits[c]));
         if (!codes_dev[c]) return EDEN_ERR_WORKSPACE;
     }
+    const uint64_t saved = ctx->ws_bytes;
+    // Large inputs go through in chunks of clients: the upload of the next chunk, the
+    // kernels of this one and the download of the previous chunk's codes overlap.
+    const uint64_t row_bytes = d * sizeof(float);
+    const uint32_t chunk = (uint32_t)std::max<uint64_t>(1, (32ull << 20) / row_bytes);
+    if (n > chunk && (uint64_t)n * row_bytes >= (64ull << 20)) {
+        if (!ctx->copy_in) {
+            CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking));
+            CUDA_OK(cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking));
+        }
+        const uint32_t n_chunks = (n + chunk - 1) / chunk;
+        while (ctx->sync_events.size() < 2ull * n_chunks + 2) {
+            cudaEvent_t e;
+            CUDA_OK(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+            ctx->sync_events.push_back(e);
+        }
+        cudaEvent_t ev_start = ctx->sync_events[0], ev_tail = ctx->sync_events[1];
+        // the staging area may still be in use by earlier work on the main stream
+        CUDA_OK(cudaEventRecord(ev_start, ctx->stream));
+        CUDA_OK(cudaStreamWaitEvent(ctx->copy_in, ev_start, 0));
+        CUDA_OK(cudaStreamWaitEvent(ctx->copy_out, ev_start, 0));
+        for (uint32_t j = 0; j < n_chunks; ++j) {
+            const uint32_t a = j * chunk, m = std::min(chunk, n - a);
+            CUDA_OK(cudaMemcpy2DAsync(x_dev + (uint64_t)a * row, row * sizeof(float), x_host + (uint64_t)a * ld_x,
+                                      ld_x * sizeof(float), row_bytes, m, cudaMemcpyHostToDevice, ctx->copy_in));
+            CUDA_OK(cudaEventRecord(ctx->sync_events[2 + 2 * j], ctx->copy_in));
+        }
+        ctx->ws_bytes = st.left;
+        int rc = EDEN_OK;
+        for (uint32_t j = 0; j < n_chunks && rc == EDEN_OK; ++j) {
+            const uint32_t a = j * chunk, m = std::min(chunk, n - a);
+            if (cudaStreamWaitEvent(ctx->stream, ctx->sync_events[2 + 2 * j], 0) != cudaSuccess) { rc = EDEN_ERR_CUDA; break; }
+            rc = eden_encode(ctx, x_dev + (uint64_t)a * row, row, d, m, bits + a, seeds + a,
+                             codes_dev.data() + a, scales_dev + a);
+            if (rc) break;
+            if (cudaEventRecord(ctx->sync_events[3 + 2 * j], ctx->stream) != cudaSuccess ||
+                cudaStreamWaitEvent(ctx->copy_out, ctx->sync_events[3 + 2 * j], 0) != cudaSuccess) { rc = EDEN_ERR_CUDA; break; }
+            for (uint32_t c = a; c < a + m; ++c)
+                if (cudaMemcpyAsync(codes_host[c], codes_dev[c], eden_code_bytes(d, bits[c]),
+                                    cudaMemcpyDeviceToHost, ctx->copy_out) != cudaSuccess) { rc = EDEN_ERR_CUDA; break; }
+        }
+        ctx->ws_bytes = saved;
+        // join the side streams back into the main stream whatever happened
+        cudaEventRecord(ev_tail, ctx->copy_out);
+        cudaStreamWaitEvent(ctx->stream, ev_tail, 0);
+        cudaEventRecord(ev_start, ctx->copy_in);
+        cudaStreamWaitEvent(ctx->stream, ev_start, 0);
+        if (rc) { cudaStreamSynchronize(ctx->stream); return rc; }
+        CUDA_OK(cudaMemcpyAsync(scales_host, scales_dev, n * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+        CUDA_OK(cudaStreamSynchronize(ctx->stream));
+        return EDEN_OK;
+    }
     CUDA_OK(cudaMemcpy2DAsync(x_dev, row * sizeof(float), x_host, ld_x * sizeof(float),
                               d * sizeof(float), n, cudaMemcpyHostToDevice, ctx->stream));
-    const uint64_t saved = ctx->ws_bytes;
     ctx->ws_bytes = st.left;
     const int rc = eden_encode(ctx, x_dev, row, d, n, bits, seeds, codes_dev.data(), scales_dev);
     ctx->ws_bytes = saved;

@@ -340,8 +340,9 @@ def test_small_workspace_runs_in_several_groups(E):
         eden_mod.workspace_bytes = orig
 
 
-def test_host_buffer_entry_points(E):
-    work = synth.make("cfg4", d=1 << 16, n=5)
+@pytest.mark.parametrize("d,n", [(1 << 16, 5), (1 << 22, 7)])     # the second shape takes the chunked, overlapped path
+def test_host_buffer_entry_points(E, d, n):
+    work = synth.make("cfg4", d=d, n=n)
     n, d = work.n, work.d
     xs = work.vectors()
     ctx = E.Context(0, d_max=d, n_batch=n, host_staging=True)
