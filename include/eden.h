@@ -64,6 +64,7 @@ extern "C" {
 #define EDEN_STATUS_ZERO_VECTOR  0x1u  /* some client had ||x|| = 0: scale 0, codes 0   */
 #define EDEN_STATUS_NONFINITE    0x2u  /* some client's norm was inf/nan: its output is unspecified */
 #define EDEN_STATUS_NO_DATA      0x4u  /* some client had no packet received: it was skipped */
+#define EDEN_STATUS_TIMEOUT      0x8u  /* a bounded wait inside a kernel ran out: the call's output is unspecified */
 
 #define EDEN_PACKET_COORDS 1024u
 #define EDEN_MAX_DIM       (1ull << 30)

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -15,6 +16,8 @@
 #include "kernels_fast.cuh"
 #include "kernels_select.cuh"
 #include "lloyd_max.h"
+
+static_assert(eden::kStatusTimeout == EDEN_STATUS_TIMEOUT, "status bit of the bounded waits");
 
 using namespace eden;
 
@@ -193,6 +196,8 @@ struct eden_ctx {
     bool profiling;
     bool force_generic;
     int plan_variant;
+    int row_staging;                 // 1: the sender's row pass runs in its persistent, bulk-copy-staged form
+    int sm_count;
     std::vector<ProfileRecord> records;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
     std::vector<ProfileSummary> summary;
@@ -259,6 +264,14 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->force_generic = false;
     ctx->plan_variant = 0;
     if (const char* pv = std::getenv("EDEN_PLAN_VARIANT")) ctx->plan_variant = std::atoi(pv);
+    ctx->row_staging = 0;
+    if (const char* rs = std::getenv("EDEN_ROW_STAGING")) ctx->row_staging = std::atoi(rs);
+    ctx->sm_count = 0;
+    if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cuda_device) != cudaSuccess ||
+        ctx->sm_count <= 0) {
+        delete ctx;
+        return EDEN_ERR_CUDA;
+    }
     const Tables& t = tables();
     if (cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_pos_value, t.pos_value, sizeof(t.pos_value)) != cudaSuccess ||
@@ -649,9 +662,28 @@ void width_runs(const std::vector<ClientPlan>& plan, const Group& g, std::vector
     }
 }
 
+// Blocks of `kernel` that fit on the device at once (cached per kernel and device).
+template <typename K>
+int resident_blocks(const eden_ctx* ctx, K kernel, uint32_t dynamic_smem)
+{
+    static std::mutex mu;
+    static std::map<std::pair<const void*, int>, int> cache;
+    std::lock_guard<std::mutex> lock(mu);
+    const auto key = std::make_pair((const void*)kernel, ctx->device);
+    auto it = cache.find(key);
+    if (it != cache.end()) return it->second;
+    int per_sm = 0;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dynamic_smem) != cudaSuccess)
+        return -1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kFastThreads, dynamic_smem) != cudaSuccess ||
+        per_sm < 1)
+        return -1;
+    return cache[key] = per_sm * ctx->sm_count;
+}
+
 // Sender passes of one group on the register-blocked path.
 int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g,
-                      ClientDesc* d_descs, ClientState* d_states, uint64_t d)
+                      ClientDesc* d_descs, ClientState* d_states, uint64_t d, uint32_t* d_status)
 {
     const uint32_t gn = (uint32_t)g.members.size();
     const double D = (double)(1ull << g.L);
@@ -673,6 +705,19 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
+        if (ctx->row_staging && pl.row_lc == 0) {
+            const int tiles_log = g.L - kFastTileLog;
+            const uint32_t total = r.count << tiles_log;
+            EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_W(r.W, {
+                const int resident = resident_blocks(ctx, k_f_enc_last_staged<W_, FRAC_>, kStagedDynamicBytes);
+                if (resident < 1) return EDEN_ERR_CUDA;
+                const uint32_t blocks = std::min<uint32_t>(total, (uint32_t)resident);
+                LAUNCH(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last_staged<W_, FRAC_>),
+                       blocks, kFastThreads, kStagedDynamicBytes, (const ClientDesc*)(d_descs + r.first), d_states + r.first,
+                       total, tiles_log, d_status);
+            }));
+            continue;
+        }
         EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
             LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_, FRAC_>),
                       dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
@@ -897,7 +942,7 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
                    dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
         }
         if (fast_eligible(ctx, g) && (x_aligned || g.subbit)) {
-            rc = fast_encode_group(ctx, plan, g, d_descs + first, d_states + first, d);
+            rc = fast_encode_group(ctx, plan, g, d_descs + first, d_states + first, d, d_status);
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);

@@ -681,26 +681,82 @@ __device__ __forceinline__ void quantise_pack_frac(const u64 (&v)[16], float inv
     }
 }
 
+// Shared-memory tables of the row pass of the sender: positive boundaries and values of
+// width W, and of width W - 1 for non-integer budgets.
+template <int W, bool FRAC>
+struct EncTables {
+    float tb[128], tv[128];
+    float tb0[FRAC ? 64 : 1], tv0[FRAC ? 64 : 1];
+    __device__ __forceinline__ void fill(int t)
+    {
+        constexpr int half = 1 << (W - 1);
+        for (int j = t; j < half; j += kFastThreads) {
+            tb[j] = c_pos_boundary[table_offset(W) + j];
+            tv[j] = c_pos_value[table_offset(W) + j];
+        }
+        if (FRAC)
+            for (int j = t; j < (half >> 1); j += kFastThreads) {
+                tb0[j] = c_pos_boundary[table_offset(W > 1 ? W - 1 : 1) + j];
+                tv0[j] = c_pos_value[table_offset(W > 1 ? W - 1 : 1) + j];
+            }
+    }
+};
+
+// The W code words of the thread's 32 coordinates, as one or two 128-bit stores where the
+// width allows (code buffers are 16-byte aligned on this path).
+template <int W>
+__device__ __forceinline__ void store_words(uint32_t* dst, const uint32_t (&words)[W])
+{
+    if constexpr (W == 2) {
+        *reinterpret_cast<uint2*>(dst) = make_uint2(words[0], words[1]);
+    } else if constexpr (W == 4 || W == 8) {
+#pragma unroll
+        for (int j = 0; j < W; j += 4)
+            *reinterpret_cast<uint4*>(dst + j) = make_uint4(words[j], words[j + 1], words[j + 2], words[j + 3]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < W; ++j) dst[j] = words[j];
+    }
+}
+
+// The 13 stages of one tile held in arrangement A, then quantise, pack and store the tile's
+// code words; returns the thread's part of sum |h| Q(|z|).
+template <int W, bool FRAC>
+__device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& cd, double n2, uint64_t base,
+                                               u64* s, const EncTables<W, FRAC>& tab)
+{
+    const int t = threadIdx.x;
+    row_step<0>(v);                 // e bits 12..9
+    row_exchange<0, 1>(v, s);
+    row_step<0>(v);                 // e bits 8..5
+    __syncthreads();
+    row_exchange<1, 2>(v, s);
+    row_step<0>(v);                 // e bits 4..1
+    row_step_inner(v);              // e bit 0
+    const bool live = n2 > 0.0 && n2 < INFINITY;
+    const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
+    uint32_t words[W];
+    float dot = 0.f;
+    if constexpr (FRAC && W >= 2) {
+        const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
+        quantise_pack_frac<W>(v, inv_norm, live, coins, tab.tb, tab.tv, tab.tb0, tab.tv0, words, dot);
+    } else {
+        quantise_pack_32<W>(v, inv_norm, live, tab.tb, tab.tv, words, dot);
+    }
+    store_words<W>(cd.codes + ((base >> 5) + t) * W, words);
+    return dot;
+}
+
 template <int W, int LC, bool FRAC>
 __global__ void __launch_bounds__(kFastThreads, 4)
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ double red[32];
-    __shared__ float s_tb[128], s_tv[128];
-    __shared__ float s_tb0[FRAC ? 64 : 1], s_tv0[FRAC ? 64 : 1];   // width W - 1 (non-integer budgets)
+    __shared__ EncTables<W, FRAC> tab;
     const ClientDesc cd = descs[blockIdx.y];
     const int t = threadIdx.x;
-    constexpr int half = 1 << (W - 1);
-    for (int j = t; j < half; j += kFastThreads) {
-        s_tb[j] = c_pos_boundary[table_offset(W) + j];
-        s_tv[j] = c_pos_value[table_offset(W) + j];
-    }
-    if (FRAC)
-        for (int j = t; j < (half >> 1); j += kFastThreads) {
-            s_tb0[j] = c_pos_boundary[table_offset(W > 1 ? W - 1 : 1) + j];
-            s_tv0[j] = c_pos_value[table_offset(W > 1 ? W - 1 : 1) + j];
-        }
+    tab.fill(t);
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
     u64 v[16];
     if (LC == 0) {
@@ -731,29 +787,119 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
         for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<0>(t, k))];
         __syncthreads();                               // s is rewritten by the next exchange
     }
-    row_step<0>(v);                 // e bits 12..9
-    row_exchange<0, 1>(v, s);
-    row_step<0>(v);                 // e bits 8..5
-    __syncthreads();
-    row_exchange<1, 2>(v, s);
-    row_step<0>(v);                 // e bits 4..1
-    row_step_inner(v);              // e bit 0
-    const double n2 = states[blockIdx.y].norm2;
-    const bool live = n2 > 0.0 && n2 < INFINITY;
-    const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
-    uint32_t words[W];
-    float dot = 0.f;
-    if constexpr (FRAC && W >= 2) {
-        const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
-        quantise_pack_frac<W>(v, inv_norm, live, coins, s_tb, s_tv, s_tb0, s_tv0, words, dot);
-    } else {
-        quantise_pack_32<W>(v, inv_norm, live, s_tb, s_tv, words, dot);
-    }
-    uint32_t* dst = cd.codes + ((base >> 5) + t) * W;
-#pragma unroll
-    for (int j = 0; j < W; ++j) dst[j] = words[j];
+    const float dot = enc_last_tile<W, FRAC>(v, cd, states[blockIdx.y].norm2, base, s, tab);
     const double tot = block_sum((double)dot, red);
     if (t == 0) atomicAdd(&states[blockIdx.y].dot, tot);
+}
+
+// ---------------------------------------------------------------------------------
+// Sender, last pass, persistent form: a resident set of blocks walks all tiles of all
+// clients of the launch (tile g belongs to client g >> tiles_log).  The next tile of a block
+// is brought into a staging buffer in shared memory by one bulk asynchronous copy
+// (cp.async.bulk, completion on an mbarrier) while the block works on the tile it holds in
+// registers, so the global-memory latency of a tile is hidden behind the arithmetic of the
+// one before it.  Every wait on the mbarrier is bounded; a wait that runs out raises
+// EDEN_STATUS_TIMEOUT and the block returns.
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// one arrival that announces `bytes` of asynchronous copies, then the copy itself
+__device__ __forceinline__ void bulk_load_tile(void* dst_smem, const void* src_global, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst_smem)), "l"(src_global), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+// waits for the phase of the given parity; false if about two seconds pass first
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\t"
+                     "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                     "selp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+        if (done) return true;
+        if (clock64() - t0 > 4000000000ll) return false;
+    }
+}
+
+constexpr uint32_t kStatusTimeout = 0x8u;   // EDEN_STATUS_TIMEOUT
+constexpr uint32_t kStagedDynamicBytes = 4u << kFastTileLog;   // one tile
+
+template <int W, bool FRAC>
+__global__ void __launch_bounds__(kFastThreads, 3)
+k_f_enc_last_staged(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states,
+                    uint32_t total_tiles, int tiles_log, uint32_t* __restrict__ status)
+{
+    extern __shared__ __align__(128) unsigned char staged_dyn[];   // kStagedDynamicBytes: the staging buffer
+    u64* stage = reinterpret_cast<u64*>(staged_dyn);
+    __shared__ __align__(16) u64 s[kRowSmemUnits];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ double red[32];
+    __shared__ int s_fail;
+    __shared__ EncTables<W, FRAC> tab;
+    const int t = threadIdx.x;
+    constexpr uint32_t kTileBytes = 4u << kFastTileLog;
+    tab.fill(t);
+    if (t == 0) {
+        s_fail = 0;
+        mbar_init(&bar, 1);
+    }
+    __syncthreads();
+    uint32_t g = blockIdx.x;
+    if (t == 0 && g < total_tiles) {
+        const ClientDesc& c0 = descs[g >> tiles_log];
+        bulk_load_tile(stage, c0.work + ((uint64_t)(g & ((1u << tiles_log) - 1u)) << kFastTileLog), kTileBytes, &bar);
+    }
+    uint32_t parity = 0;
+    uint32_t cur = 0xFFFFFFFFu;          // client whose partial sum `acc` holds
+    double acc = 0.0;
+    for (; g < total_tiles; g += gridDim.x) {
+        if (!mbar_wait_bounded(&bar, parity)) s_fail = 1;
+        parity ^= 1u;
+        u64 v[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) v[k] = stage[row_u<0>(t, k)];
+        __syncthreads();                               // the staging buffer is free again
+        if (s_fail) break;
+        const uint32_t gn = g + gridDim.x;
+        if (t == 0 && gn < total_tiles) {
+            const ClientDesc& cn = descs[gn >> tiles_log];
+            bulk_load_tile(stage, cn.work + ((uint64_t)(gn & ((1u << tiles_log) - 1u)) << kFastTileLog), kTileBytes, &bar);
+        }
+        const uint32_t client = g >> tiles_log;
+        if (client != cur) {
+            if (cur != 0xFFFFFFFFu) {
+                const double tot = block_sum(acc, red);
+                if (t == 0) atomicAdd(&states[cur].dot, tot);
+            }
+            cur = client;
+            acc = 0.0;
+        }
+        const ClientDesc cd = descs[client];
+        const uint64_t base = (uint64_t)(g & ((1u << tiles_log) - 1u)) << kFastTileLog;
+        acc += (double)enc_last_tile<W, FRAC>(v, cd, states[client].norm2, base, s, tab);
+        // the barrier after the next tile's staging read orders this tile's last exchange
+        // reads before the next tile's first exchange writes
+    }
+    if (s_fail) {
+        if (t == 0) atomicOr(status, kStatusTimeout);
+        return;
+    }
+    if (cur != 0xFFFFFFFFu) {
+        const double tot = block_sum(acc, red);
+        if (t == 0) atomicAdd(&states[cur].dot, tot);
+    }
 }
 
 // =================================================================================

@@ -67,7 +67,7 @@ _sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
 _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(_u64),
                                 ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
 
-STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA = 1, 2, 4
+STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA, STATUS_TIMEOUT = 1, 2, 4, 8
 PACKET_COORDS = 1024
 
 

@@ -166,6 +166,20 @@ def test_pass_plans_at_2_pow_24_and_25(E, variant, monkeypatch):
         run_workload(E, work)
 
 
+@pytest.mark.parametrize("bits", [1.0, 2.0, 4.0, 8.0, 2.5])
+def test_sender_row_pass_staged_by_bulk_copies(E, bits, monkeypatch):
+    # the persistent form of the sender's last pass (tiles staged in shared memory by bulk
+    # asynchronous copies) must give the same messages as the default form; three clients of
+    # 2^20 rotated coordinates are 384 tiles, several per resident block with a ragged split
+    monkeypatch.setenv("EDEN_ROW_STAGING", "1")
+    d, n = (1 << 20) - 5, 3
+    rng = np.random.default_rng(int(bits * 10))
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(17, n), 0.0,
+                          lambda c: xs[c], 17)
+    run_workload(E, work)
+
+
 @pytest.mark.parametrize("W", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_every_code_width(E, W):
     d, n = 40000, 2
