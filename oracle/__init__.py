@@ -84,6 +84,18 @@ def _L():
         lib.eden_oracle_encode.restype = ctypes.c_int
         lib.eden_oracle_decode.argtypes = [vp, f64, f64, u64, vp, u64, vp]
         lib.eden_oracle_decode.restype = ctypes.c_int
+        for name in ("eden_oracle_uniform_entropy", "eden_oracle_uniform_delta",
+                     "eden_oracle_uniform_second_moment"):
+            getattr(lib, name).argtypes = [f64]
+            getattr(lib, name).restype = f64
+        lib.eden_oracle_uniform_value.argtypes = [f64, u32]
+        lib.eden_oracle_uniform_value.restype = f64
+        lib.eden_oracle_uniform_index.argtypes = [f64, f64]
+        lib.eden_oracle_uniform_index.restype = ctypes.c_int32
+        lib.eden_oracle_encode_uniform.argtypes = [vp, u64, f64, u64, vp, vp, vp]
+        lib.eden_oracle_encode_uniform.restype = ctypes.c_int
+        lib.eden_oracle_decode_uniform.argtypes = [vp, f64, f64, u64, vp, u64, vp]
+        lib.eden_oracle_decode_uniform.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -271,4 +283,89 @@ def mean(codes, scales, bits, seeds, d: int, recv_masks=None, threads: int = 1):
                 if not nodata:
                     acc += xh
                     used += 1
+    return acc / n, used
+
+
+# --------------------------------------------------------------------------- Section 4.3
+UNIFORM_MAX_INDEX = 127
+
+
+def uniform_entropy(delta: float) -> float:
+    """H of the uniform-interval family I_Delta under N(0,1), bits per coordinate."""
+    return float(_L().eden_oracle_uniform_entropy(float(delta)))
+
+
+def uniform_delta(bits: float) -> float:
+    """Delta_b: the smallest Delta with H(I_Delta) <= bits (0.0 if out of range)."""
+    return float(_L().eden_oracle_uniform_delta(float(bits)))
+
+
+def uniform_value(delta: float, m: int) -> float:
+    """Centre of mass of the interval of magnitude index m (the outermost one is open)."""
+    return float(_L().eden_oracle_uniform_value(float(delta), int(m)))
+
+
+def uniform_second_moment(delta: float) -> float:
+    return float(_L().eden_oracle_uniform_second_moment(float(delta)))
+
+
+def uniform_index(z: float, delta: float) -> int:
+    return int(_L().eden_oracle_uniform_index(float(z), float(delta)))
+
+
+def encode_uniform(x: np.ndarray, delta: float, seed: int, want_z: bool = False):
+    """One sender over I_Delta.  Returns dict(index int8[D], scale float64, z)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    d = x.shape[0]
+    D = rot_dim(d, 1.0)
+    index = np.zeros(D, dtype=np.int8)
+    scale = np.zeros(1, dtype=np.float64)
+    z = np.zeros(D, dtype=np.float64) if want_z else None
+    rc = _L().eden_oracle_encode_uniform(_ptr(x), d, float(delta), int(seed), _ptr(index), _ptr(scale),
+                                         _ptr(z) if want_z else None)
+    if rc:
+        raise MemoryError("oracle encode_uniform")
+    return {"index": index, "scale": float(scale[0]), "z": z}
+
+
+def decode_uniform(index: np.ndarray, scale: float, delta: float, seed: int, d: int, recv_mask=None):
+    index = np.ascontiguousarray(index, dtype=np.int8)
+    xhat = np.zeros(d, dtype=np.float64)
+    rm = None
+    if recv_mask is not None:
+        rm = np.ascontiguousarray(recv_mask, dtype=np.uint32)
+    rc = _L().eden_oracle_decode_uniform(_ptr(index), float(scale), float(delta), int(seed),
+                                         _ptr(rm) if rm is not None else None, int(d), _ptr(xhat))
+    if rc < 0:
+        raise MemoryError("oracle decode_uniform")
+    return xhat, rc == 1
+
+
+def encode_uniform_all(xs, deltas, seeds, threads: int = 1, want_z: bool = False):
+    n = len(seeds)
+
+    def one(c):
+        return encode_uniform(xs[c], deltas[c], seeds[c], want_z)
+
+    if threads <= 1:
+        return [one(c) for c in range(n)]
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        return list(ex.map(one, range(n)))
+
+
+def mean_uniform(indices, scales, deltas, seeds, d: int, recv_masks=None, threads: int = 1):
+    """Receiver over I_Delta: (1/n) * sum_c x_hat_c; returns (mean float64[d], n_used)."""
+    n = len(seeds)
+
+    def one(c):
+        return decode_uniform(indices[c], scales[c], deltas[c], seeds[c], d,
+                              None if recv_masks is None else recv_masks[c])
+
+    acc = np.zeros(d, dtype=np.float64)
+    used = 0
+    with ThreadPoolExecutor(max_workers=max(1, threads)) as ex:
+        for xh, nodata in ex.map(one, range(n)):
+            if not nodata:
+                acc += xh
+                used += 1
     return acc / n, used

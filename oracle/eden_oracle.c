@@ -48,6 +48,13 @@
  *     upper floor(b) bits of a set coordinate's code), then one word holding the lowest
  *     code bit of the set coordinates, packed in coordinate order from bit 0.
  *     Only floor(b)*32 + (number of coins) bits of a group are meaningful.  [layout unpinned]
+ *   - Section 4.3's uniform-interval family I_Delta (functions *_uniform_* at the end):
+ *     index n = round(z / Delta), an endpoint going to the interval nearer zero like
+ *     everywhere else; indices are clamped to +-127, i.e. the family is made finite by
+ *     letting the two outermost intervals run to infinity; the message is one signed
+ *     byte per rotated coordinate (what an entropy coder would consume; the coder itself
+ *     is not part of this build) plus S.  Boundary k is fl32(fl32(Delta) * (k - 1/2)).
+ *                                                       [clamp, byte layout unpinned]
  *   - The interval decision is taken after rounding z and the boundary to fp32,
  *     the precision the GPU kernels decide in; everything else is double.
  *   - ||x|| = 0: scale 0, all codes 0.  A client with no received packet
@@ -509,6 +516,145 @@ int eden_oracle_decode(const uint32_t *codes, double S, double bits, uint64_t se
     } else {
         for (uint64_t i = 0; i < d; ++i) xhat[i] = q[i];
     }
+    free(q);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Section 4.3: the uniform-interval family                                    */
+/*   I_Delta = { [Delta (n - 1/2), Delta (n + 1/2)] : n integer },             */
+/* its entropy H = -sum_n p_n log2 p_n under N(0,1), Delta_b = the smallest    */
+/* Delta with H <= b, and EDEN with Q = centre of mass of the interval.        */
+/* ------------------------------------------------------------------------- */
+#define EDEN_ORACLE_UNIFORM_MAX_INDEX 127
+
+double eden_oracle_uniform_entropy(double delta)
+{
+    double p0 = std_normal_mass(-0.5 * delta, 0.5 * delta);
+    double h = p0 > 0.0 ? -p0 * log2(p0) : 0.0;
+    for (uint64_t n = 1;; ++n) {
+        double a = delta * ((double)n - 0.5);
+        double p = std_normal_mass(a, a + delta);
+        if (!(p > 0.0)) break;                 /* the tail mass has underflowed */
+        h -= 2.0 * p * log2(p);                /* intervals n and -n */
+    }
+    return h;
+}
+
+/* H falls as Delta grows, so "the smallest Delta with H <= b" is the root of H = b. */
+double eden_oracle_uniform_delta(double bits)
+{
+    double lo = 1e-4, hi = 64.0;               /* H(lo) ~ 15.3 bits, H(hi) ~ 0 */
+    if (!(bits > eden_oracle_uniform_entropy(hi)) || !(bits < eden_oracle_uniform_entropy(lo))) return 0.0;
+    for (int it = 0; it < 200; ++it) {
+        double mid = 0.5 * (lo + hi);
+        if (eden_oracle_uniform_entropy(mid) <= bits) hi = mid; else lo = mid;
+    }
+    return hi;
+}
+
+/* centre of mass of the interval of magnitude index m (0 <= m <= 127); the index's sign
+   is the value's sign                                     [underflow rule unpinned] */
+double eden_oracle_uniform_value(double delta, uint32_t m)
+{
+    if (m == 0) return 0.0;
+    double a = delta * ((double)m - 0.5);
+    double b = m == EDEN_ORACLE_UNIFORM_MAX_INDEX ? INFINITY : a + delta;
+    /* beyond ~38 standard deviations the mass underflows in double precision; such an
+       interval (never reached by data) takes its inner endpoint as its value */
+    if (!(std_normal_mass(a, b) > 0.0)) return a;
+    return eden_oracle_centre_of_mass(a, b);
+}
+
+/* E[Q(z)^2] of the clamped family; vNMSE = 1/E[Q^2] - 1 (Corollary 2.4) */
+double eden_oracle_uniform_second_moment(double delta)
+{
+    double acc = 0.0;
+    for (uint32_t m = 1; m <= EDEN_ORACLE_UNIFORM_MAX_INDEX; ++m) {
+        double a = delta * ((double)m - 0.5);
+        double b = m == EDEN_ORACLE_UNIFORM_MAX_INDEX ? INFINITY : a + delta;
+        double q = eden_oracle_uniform_value(delta, m);
+        acc += 2.0 * std_normal_mass(a, b) * q * q;
+    }
+    return acc;
+}
+
+/* index of z: the number of positive boundaries Delta (k - 1/2), k = 1..127, strictly
+   below |z|, with z's sign; compared in fp32 like eden_oracle_quantise */
+int32_t eden_oracle_uniform_index(double z, double delta)
+{
+    float az = (float)fabs(z);
+    float df = (float)delta;
+    int32_t m = 0;
+    for (int32_t k = 1; k <= EDEN_ORACLE_UNIFORM_MAX_INDEX; ++k) {
+        float t = df * ((float)k - 0.5f);
+        if (az > t) m = k; else break;
+    }
+    return z < 0.0 ? -m : m;
+}
+
+/* Sender with Q over I_Delta (b >= 1 shape: no sparsification).  index[D] signed bytes. */
+int eden_oracle_encode_uniform(const float *x, uint64_t d, double delta, uint64_t seed,
+                               int8_t *index, double *scale_out, double *z_out)
+{
+    uint64_t D = eden_oracle_rot_dim(d, 1.0);
+    double *y = (double *)calloc(D, sizeof(double));
+    if (!y) return -1;
+    for (uint64_t i = 0; i < d; ++i) y[i] = (double)x[i];
+    double N2 = 0.0;
+    for (uint64_t i = 0; i < D; ++i) N2 += y[i] * y[i];
+    memset(index, 0, D);
+    if (N2 == 0.0) {
+        *scale_out = 0.0;
+        if (z_out) memset(z_out, 0, sizeof(double) * D);
+        free(y);
+        return 0;
+    }
+    for (uint64_t i = 0; i < D; ++i) y[i] *= eden_oracle_sign(seed, i);
+    eden_oracle_fwht(y, D);
+    double inv_sqrt_D = 1.0 / sqrt((double)D);
+    for (uint64_t i = 0; i < D; ++i) y[i] *= inv_sqrt_D;             /* r = R(y) */
+    double eta = sqrt((double)D) / sqrt(N2);
+    double dot = 0.0;
+    for (uint64_t i = 0; i < D; ++i) {
+        double z = eta * y[i];
+        int32_t n = eden_oracle_uniform_index(z, delta);
+        double q = eden_oracle_uniform_value(delta, (uint32_t)(n < 0 ? -n : n));
+        dot += y[i] * (n < 0 ? -q : q);
+        index[i] = (int8_t)n;
+        if (z_out) z_out[i] = z;
+    }
+    *scale_out = N2 / dot;
+    free(y);
+    return 0;
+}
+
+/* Receiver for one sender of the uniform family; same contract as eden_oracle_decode.
+   An index byte of -128 never occurs in a message; it is read as -127. */
+int eden_oracle_decode_uniform(const int8_t *index, double S, double delta, uint64_t seed,
+                               const uint32_t *recv_mask, uint64_t d, double *xhat)
+{
+    uint64_t D = eden_oracle_rot_dim(d, 1.0);
+    memset(xhat, 0, sizeof(double) * d);
+    double *q = (double *)calloc(D, sizeof(double));
+    if (!q) return -1;
+    uint64_t received = 0;
+    for (uint64_t i = 0; i < D; ++i) {
+        uint64_t pkt = i / EDEN_ORACLE_PACKET;
+        int arrived = recv_mask ? (int)((recv_mask[pkt / 32u] >> (pkt % 32u)) & 1u) : 1;
+        if (!arrived) continue;
+        ++received;
+        int32_t n = index[i];
+        uint32_t m = (uint32_t)(n < 0 ? -n : n);
+        if (m > EDEN_ORACLE_UNIFORM_MAX_INDEX) m = EDEN_ORACLE_UNIFORM_MAX_INDEX;
+        double v = eden_oracle_uniform_value(delta, m);
+        q[i] = n < 0 ? -v : v;
+    }
+    if (received == 0) { free(q); return 1; }
+    double p = (double)received / (double)D;
+    eden_oracle_fwht(q, D);
+    double f = S / (p * sqrt((double)D));
+    for (uint64_t i = 0; i < d; ++i) xhat[i] = q[i] * f * eden_oracle_sign(seed, i);
     free(q);
     return 0;
 }
