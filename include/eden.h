@@ -191,6 +191,57 @@ int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bi
 int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stream, uint64_t seed,
                                      uint64_t d, double bits, uint32_t* mask_bits);
 
+/* ---- Section 4.3: the uniform-interval family --------------------------------------- */
+
+/* Section 4.3 replaces the 2^b Lloyd-Max intervals by
+ *     I_Delta = { [Delta (n - 1/2), Delta (n + 1/2)] : n integer },
+ * Delta_b = the smallest Delta whose entropy under N(0,1) is at most b bits, so that an
+ * entropy coder (not part of this library) can send the indices in about b bits per
+ * coordinate.  The interval of a coordinate is n = round(z / Delta) (an endpoint goes to
+ * the interval nearer zero), its value the interval's centre of mass.  This library
+ * clamps n to +-EDEN_UNIFORM_MAX_INDEX (the two outermost intervals run to infinity) and
+ * writes one signed byte per rotated coordinate: byte i of a client's message is the
+ * index of rotated coordinate i; a packet is still 1024 coordinates.  Supported widths:
+ * EDEN_UNIFORM_MIN_DELTA <= Delta < 2 (Section 4.3 requires Delta in (0, 2)); other
+ * values return EDEN_ERR_UNSUPPORTED_BITS.  No sparsification: budgets below
+ * eden_uniform_entropy(2) ~ 1.24 bits are not reachable with this family. */
+#define EDEN_UNIFORM_MAX_INDEX 127
+#define EDEN_UNIFORM_MIN_DELTA 0.0625
+
+/* Host only.  Entropy in bits per coordinate of I_Delta under N(0,1); 0 for delta <= 0. */
+double eden_uniform_entropy(double delta);
+/* Host only.  Delta_b for a budget of `bits` per coordinate; 0 if it falls outside the
+ * supported widths. */
+double eden_uniform_delta(double bits);
+/* Host only.  values[m], m = 0..127: centre of mass of the interval of magnitude index m,
+ * rounded to fp32 (what the kernels use); the value of index -m is -values[m]. */
+int eden_uniform_values(double delta, float* values);
+/* Bytes of one client's index message: the rotation dimension, rounded up to 16. */
+uint64_t eden_uniform_index_bytes(uint64_t d);
+
+/* eden_encode with Q over I_Delta.  delta: host, n interval widths.  index: host array
+ * of n dev pointers, each to eden_uniform_index_bytes(d) bytes, 16-byte aligned.
+ * scales as for eden_encode.  Same error and status behaviour. */
+int eden_encode_uniform(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                        const double* delta, const uint64_t* seeds,
+                        int8_t* const* index, float* scales);
+/* eden_decode_accumulate / eden_mean for such messages (index pointers 4-byte aligned). */
+int eden_decode_accumulate_uniform(eden_ctx* ctx, const int8_t* const* index, const float* scales,
+                                   const double* delta, const uint64_t* seeds,
+                                   const uint32_t* const* recv_masks,
+                                   uint64_t d, uint32_t n, float* acc, uint32_t* n_used);
+int eden_mean_uniform(eden_ctx* ctx, const int8_t* const* index, const float* scales,
+                      const double* delta, const uint64_t* seeds,
+                      const uint32_t* const* recv_masks,
+                      uint64_t d, uint32_t n, float* mean);
+/* Occurrences of each index value in each client's message: hist (dev, n * 256 words,
+ * overwritten), hist[c * 256 + v + 128] = number of rotated coordinates of client c with
+ * index v.  The empirical entropy of these counts estimates the entropy-coded length
+ * (Section 4.3 and its appendix on representation length).  index pointers 16-byte
+ * aligned. */
+int eden_index_histogram(eden_ctx* ctx, const int8_t* const* index, uint64_t d, uint32_t n,
+                         uint32_t* hist);
+
 /* ---- the same two steps on host memory (copies included) --------------------------- */
 
 /* x, codes (array of n host pointers), scales are HOST buffers (pinned memory makes the

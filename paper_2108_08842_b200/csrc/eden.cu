@@ -16,6 +16,7 @@
 #include "kernels_fast.cuh"
 #include "kernels_select.cuh"
 #include "lloyd_max.h"
+#include "uniform_family.h"
 
 static_assert(eden::kStatusTimeout == EDEN_STATUS_TIMEOUT, "status bit of the bounded waits");
 
@@ -145,7 +146,7 @@ extern "C" uint64_t eden_workspace_bytes(uint64_t d_max, uint32_t n_batch)
     const uint64_t n_chunks = (d_max + kSelChunk - 1) / kSelChunk;
     const uint64_t sel = 256 + kHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) + 256;
     return fixed_layout(d_max).end + align_up(per_client_bytes() * n_batch, 256) + 1024 +
-           (uint64_t)n_batch * (align_up(D * sizeof(float), 256) + sel);
+           (uint64_t)n_batch * (align_up(D * sizeof(float), 256) + sel + 512 /* uniform-family values */);
 }
 
 extern "C" int eden_table(uint32_t W, float* centroids, float* boundaries)
@@ -156,6 +157,23 @@ extern "C" int eden_table(uint32_t W, float* centroids, float* boundaries)
     std::copy(t.boundaries[W].begin(), t.boundaries[W].end(), boundaries);
     return EDEN_OK;
 }
+
+extern "C" double eden_uniform_entropy(double delta)
+{
+    return delta > 0.0 ? uniform_entropy(delta) : 0.0;
+}
+
+extern "C" double eden_uniform_delta(double bits) { return uniform_delta(bits); }
+
+extern "C" int eden_uniform_values(double delta, float* values)
+{
+    if (!values) return EDEN_ERR_INVALID_ARG;
+    if (!(delta >= kUniformMinDelta) || !(delta < kUniformMaxDelta)) return EDEN_ERR_UNSUPPORTED_BITS;
+    uniform_values(delta, values);
+    return EDEN_OK;
+}
+
+extern "C" uint64_t eden_uniform_index_bytes(uint64_t d) { return (eden_rot_dim(d, 1.0) + 15) / 16 * 16; }
 
 extern "C" const char* eden_strerror(int code)
 {
@@ -394,6 +412,7 @@ struct ClientPlan {
     bool subbit;
     bool needs_work;
     uint32_t coin_thr;   // non-integer b > 1
+    double delta;        // uniform-interval family (Section 4.3): interval width; else 0
 };
 
 // A set of clients of one rotation dimension launched together.
@@ -401,19 +420,37 @@ struct Group {
     std::vector<uint32_t> members;   // indices into the plan array
     int L;
     bool subbit;
-    bool fractional;                 // non-integer budgets b > 1 (shape-generic kernels only)
+    bool fractional;                 // non-integer budgets b > 1
+    bool uniform;                    // uniform-interval family: one signed byte per coordinate
 };
 
 struct CallLayout {
-    uint64_t descs_off, states_off, work_off, work_bytes;
+    uint64_t descs_off, states_off, utab_off, work_off, work_bytes;
 };
 
-int plan_clients(uint64_t d, uint32_t n, const double* bits, std::vector<ClientPlan>& plan)
+constexpr uint64_t kUniformTableBytes = kUniformValues * sizeof(float);
+
+// `delta` non-null: every client uses the uniform-interval family of that width (then
+// `bits` is not read): one byte per rotated coordinate, no sparsification.
+int plan_clients(uint64_t d, uint32_t n, const double* bits, const double* delta, std::vector<ClientPlan>& plan)
 {
-    if (d == 0 || n == 0 || !bits) return EDEN_ERR_INVALID_ARG;
+    if (d == 0 || n == 0 || (!bits && !delta)) return EDEN_ERR_INVALID_ARG;
     if (d > EDEN_MAX_DIM) return EDEN_ERR_TOO_LARGE;
     plan.resize(n);
-    for (uint32_t c = 0; c < n; ++c) {
+    for (uint32_t c = 0; c < n && delta; ++c) {
+        if (!(delta[c] >= kUniformMinDelta) || !(delta[c] < kUniformMaxDelta)) return EDEN_ERR_UNSUPPORTED_BITS;
+        ClientPlan& p = plan[c];
+        p.index = c;
+        p.k = d;
+        p.D = eden_rot_dim(d, 1.0);
+        p.L = ceil_log2(p.D);
+        p.W = 8;
+        p.subbit = false;
+        p.coin_thr = 0;
+        p.delta = delta[c];
+        p.needs_work = p.L > kGenericTileLog;
+    }
+    for (uint32_t c = 0; c < n && !delta; ++c) {
         const uint32_t W = eden_code_width(bits[c]);
         if (W == 0) return EDEN_ERR_UNSUPPORTED_BITS;
         ClientPlan& p = plan[c];
@@ -424,17 +461,19 @@ int plan_clients(uint64_t d, uint32_t n, const double* bits, std::vector<ClientP
         p.W = (int)W;
         p.subbit = bits[c] < 1.0;
         p.coin_thr = coin_threshold(bits[c]);
+        p.delta = 0.0;
         p.needs_work = p.subbit || p.L > kGenericTileLog;
     }
     return EDEN_OK;
 }
 
-int carve(const eden_ctx* ctx, uint64_t d, uint32_t n, CallLayout& lay)
+int carve(const eden_ctx* ctx, uint64_t d, uint32_t n, bool uniform, CallLayout& lay)
 {
     const FixedLayout f = fixed_layout(d);
     lay.descs_off = f.end;
     lay.states_off = lay.descs_off + align_up(sizeof(ClientDesc) * (uint64_t)n, 256);
-    lay.work_off = lay.states_off + align_up(sizeof(ClientState) * (uint64_t)n, 256);
+    lay.utab_off = lay.states_off + align_up(sizeof(ClientState) * (uint64_t)n, 256);
+    lay.work_off = lay.utab_off + (uniform ? kUniformTableBytes * (uint64_t)n : 0);
     if (lay.work_off > ctx->ws_bytes) return EDEN_ERR_WORKSPACE;
     lay.work_bytes = ctx->ws_bytes - lay.work_off;
     return EDEN_OK;
@@ -474,6 +513,7 @@ int make_groups(const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_b
         g.L = plan[idx[i]].L;
         g.subbit = plan[idx[i]].subbit;
         g.fractional = plan[idx[i]].coin_thr != 0;
+        g.uniform = plan[idx[i]].delta > 0.0;
         const uint64_t need = (plan[idx[i]].needs_work ? work_buffer_bytes(plan[idx[i]].D) : 0) +
                               (g.subbit ? sel_scratch_bytes(d) : 0);
         if (need > work_bytes) return EDEN_ERR_WORKSPACE;
@@ -688,7 +728,8 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     const uint32_t gn = (uint32_t)g.members.size();
     const double D = (double)(1ull << g.L);
     const unsigned tiles = (unsigned)((1ull << g.L) >> kFastTileLog);
-    const FastPlan pl = fast_plan(g.L, ctx->plan_variant);
+    // the uniform-interval family has no cluster form of the row pass
+    const FastPlan pl = fast_plan(g.L, g.uniform ? 0 : ctx->plan_variant);
     for (size_t pi = 0; pi < pl.cols.size(); ++pi) {
         const FastPass& ps = pl.cols[pi];
         if (pi == 0) {
@@ -705,6 +746,11 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
+        if (g.uniform) {
+            LAUNCH(ctx, "f_enc_last", r.count * 5.0 * D, (k_f_enc_last<8, 0, false, true>), dim3(tiles, r.count),
+                   kFastThreads, 0, (const ClientDesc*)(d_descs + r.first), d_states + r.first);
+            continue;
+        }
         if (ctx->row_staging && pl.row_lc == 0) {
             const int tiles_log = g.L - kFastTileLog;
             const uint32_t total = r.count << tiles_log;
@@ -859,19 +905,46 @@ extern "C" int eden_pass_plan(uint64_t d, double bits, uint32_t* pass_bits, uint
 // ------------------------------------------------------------------------------------
 // sender
 // ------------------------------------------------------------------------------------
-extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
-                           const double* bits, const uint64_t* seeds,
-                           uint8_t* const* codes, float* scales)
+namespace {
+
+// Values of the uniform-interval family for the clients in processing order, uploaded
+// behind the descriptors; sets each descriptor's table pointer and interval width.
+int upload_uniform_tables(eden_ctx* ctx, const CallLayout& lay, const std::vector<ClientPlan>& plan,
+                          const std::vector<uint32_t>& order, std::vector<ClientDesc>& descs)
+{
+    std::vector<float> tabs((size_t)kUniformValues * descs.size());
+    std::map<double, size_t> seen;                 // clients usually share one width
+    float* d_tabs = (float*)(ctx->ws + lay.utab_off);
+    for (size_t j = 0; j < descs.size(); ++j) {
+        const double delta = plan[order[j]].delta;
+        auto it = seen.find(delta);
+        if (it == seen.end()) {
+            uniform_values(delta, &tabs[j * kUniformValues]);
+            seen[delta] = j;
+        } else {
+            std::copy(&tabs[it->second * kUniformValues], &tabs[(it->second + 1) * kUniformValues],
+                      &tabs[j * kUniformValues]);
+        }
+        descs[j].utable = d_tabs + j * kUniformValues;
+        descs[j].delta = (float)delta;
+    }
+    CUDA_OK(cudaMemcpyAsync(d_tabs, tabs.data(), tabs.size() * sizeof(float), cudaMemcpyHostToDevice, ctx->stream));
+    return EDEN_OK;
+}
+
+int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                  const double* bits, const double* delta, const uint64_t* seeds,
+                  uint8_t* const* codes, float* scales)
 {
     if (!ctx || !x || !seeds || !codes || !scales || ld_x < d) return EDEN_ERR_INVALID_ARG;
     std::vector<ClientPlan> plan;
-    int rc = plan_clients(d, n, bits, plan);
+    int rc = plan_clients(d, n, bits, delta, plan);
     if (rc) return rc;
     for (uint32_t c = 0; c < n; ++c)
         if (!codes[c] || ((uintptr_t)codes[c] & 15u)) return EDEN_ERR_INVALID_ARG;
     CUDA_OK(cudaSetDevice(ctx->device));
     CallLayout lay;
-    rc = carve(ctx, d, n, lay);
+    rc = carve(ctx, d, n, delta != nullptr, lay);
     if (rc) return rc;
     std::vector<Group> groups;
     rc = make_groups(plan, d, lay.work_bytes, groups);
@@ -914,6 +987,10 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
     ClientState* d_states = (ClientState*)(ctx->ws + lay.states_off);
     uint32_t* d_status = (uint32_t*)(ctx->ws + f.status);
     ctx->states_off = lay.states_off;
+    if (delta) {
+        rc = upload_uniform_tables(ctx, lay, plan, ctx->order, descs);
+        if (rc) return rc;
+    }
     CUDA_OK(cudaMemcpyAsync(d_descs, descs.data(), sizeof(ClientDesc) * n, cudaMemcpyHostToDevice, ctx->stream));
     CUDA_OK(cudaMemsetAsync(d_states, 0, sizeof(ClientState) * n, ctx->stream));
 
@@ -971,23 +1048,41 @@ extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_
     return EDEN_OK;
 }
 
+}  // namespace
+
+extern "C" int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                           const double* bits, const uint64_t* seeds,
+                           uint8_t* const* codes, float* scales)
+{
+    if (!bits) return EDEN_ERR_INVALID_ARG;
+    return encode_common(ctx, x, ld_x, d, n, bits, nullptr, seeds, codes, scales);
+}
+
+extern "C" int eden_encode_uniform(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                                   const double* delta, const uint64_t* seeds,
+                                   int8_t* const* index, float* scales)
+{
+    if (!delta) return EDEN_ERR_INVALID_ARG;
+    return encode_common(ctx, x, ld_x, d, n, nullptr, delta, seeds, (uint8_t* const*)index, scales);
+}
+
 // ------------------------------------------------------------------------------------
 // receiver
 // ------------------------------------------------------------------------------------
 static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
-                         const double* bits, const uint64_t* seeds,
+                         const double* bits, const double* delta, const uint64_t* seeds,
                          const uint32_t* const* recv_masks, uint64_t d, uint32_t n,
                          float* out, bool mean)
 {
     if (!ctx || !codes || !scales || !seeds || !out) return EDEN_ERR_INVALID_ARG;
     std::vector<ClientPlan> plan;
-    int rc = plan_clients(d, n, bits, plan);
+    int rc = plan_clients(d, n, bits, delta, plan);
     if (rc) return rc;
     for (uint32_t c = 0; c < n; ++c)
         if (!codes[c] || ((uintptr_t)codes[c] & 3u)) return EDEN_ERR_INVALID_ARG;
     CUDA_OK(cudaSetDevice(ctx->device));
     CallLayout lay;
-    rc = carve(ctx, d, n, lay);
+    rc = carve(ctx, d, n, delta != nullptr, lay);
     if (rc) return rc;
     std::vector<Group> groups;
     rc = make_groups(plan, d, lay.work_bytes, groups);
@@ -1028,6 +1123,10 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
     ClientState* d_states = (ClientState*)(ctx->ws + lay.states_off);
     uint32_t* d_status = (uint32_t*)(ctx->ws + f.status);
     ctx->states_off = lay.states_off;
+    if (delta) {
+        rc = upload_uniform_tables(ctx, lay, plan, ctx->order, descs);
+        if (rc) return rc;
+    }
     CUDA_OK(cudaMemcpyAsync(d_descs, descs.data(), sizeof(ClientDesc) * n, cudaMemcpyHostToDevice, ctx->stream));
     CUDA_OK(cudaMemsetAsync(d_states, 0, sizeof(ClientState) * n, ctx->stream));
     LAUNCH(ctx, "dec_prep", n * 8.0, k_dec_prep, n, 256, 0, d_descs, d_states, scales, d_status);
@@ -1105,9 +1204,56 @@ extern "C" int eden_decode_accumulate(eden_ctx* ctx, const uint8_t* const* codes
                                       const uint32_t* const* recv_masks,
                                       uint64_t d, uint32_t n, float* acc, uint32_t* n_used)
 {
-    const int rc = decode_common(ctx, codes, scales, bits, seeds, recv_masks, d, n, acc, false);
+    if (!bits) return EDEN_ERR_INVALID_ARG;
+    const int rc = decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, acc, false);
     if (rc == EDEN_OK && n_used) *n_used = n;
     return rc;
+}
+
+extern "C" int eden_decode_accumulate_uniform(eden_ctx* ctx, const int8_t* const* index, const float* scales,
+                                              const double* delta, const uint64_t* seeds,
+                                              const uint32_t* const* recv_masks,
+                                              uint64_t d, uint32_t n, float* acc, uint32_t* n_used)
+{
+    if (!delta) return EDEN_ERR_INVALID_ARG;
+    const int rc = decode_common(ctx, (const uint8_t* const*)index, scales, nullptr, delta, seeds, recv_masks,
+                                 d, n, acc, false);
+    if (rc == EDEN_OK && n_used) *n_used = n;
+    return rc;
+}
+
+extern "C" int eden_mean_uniform(eden_ctx* ctx, const int8_t* const* index, const float* scales,
+                                 const double* delta, const uint64_t* seeds,
+                                 const uint32_t* const* recv_masks,
+                                 uint64_t d, uint32_t n, float* mean)
+{
+    if (!delta) return EDEN_ERR_INVALID_ARG;
+    return decode_common(ctx, (const uint8_t* const*)index, scales, nullptr, delta, seeds, recv_masks, d, n,
+                         mean, true);
+}
+
+// How often each index value occurs in each client's message (Section 4.3: what an entropy
+// coder's model, and the estimate of the coded length, are built from).
+extern "C" int eden_index_histogram(eden_ctx* ctx, const int8_t* const* index, uint64_t d, uint32_t n,
+                                    uint32_t* hist)
+{
+    if (!ctx || !index || !hist || d == 0 || n == 0) return EDEN_ERR_INVALID_ARG;
+    if (d > EDEN_MAX_DIM) return EDEN_ERR_TOO_LARGE;
+    for (uint32_t c = 0; c < n; ++c)
+        if (!index[c] || ((uintptr_t)index[c] & 15u)) return EDEN_ERR_INVALID_ARG;
+    CUDA_OK(cudaSetDevice(ctx->device));
+    const uint64_t D = eden_rot_dim(d, 1.0);
+    const uint64_t ptr_bytes = align_up(sizeof(const int8_t*) * (uint64_t)n, 256);
+    const FixedLayout f = fixed_layout(d);
+    if (f.end + ptr_bytes > ctx->ws_bytes) return EDEN_ERR_WORKSPACE;
+    const int8_t** d_ptrs = (const int8_t**)(ctx->ws + f.end);
+    CUDA_OK(cudaMemcpyAsync(d_ptrs, index, sizeof(const int8_t*) * (uint64_t)n, cudaMemcpyHostToDevice, ctx->stream));
+    CUDA_OK(cudaMemsetAsync(hist, 0, 256ull * sizeof(uint32_t) * n, ctx->stream));
+    const uint64_t per_block = (uint64_t)kHistThreads * kHistBytesPerThread;
+    const unsigned blocks = (unsigned)std::min<uint64_t>((D + per_block - 1) / per_block, 4ull * ctx->sm_count);
+    LAUNCH(ctx, "index_hist", (double)n * (double)D, k_index_hist, dim3(blocks, n), kHistThreads, 0,
+           (const int8_t* const*)d_ptrs, D, hist);
+    return EDEN_OK;
 }
 
 extern "C" int eden_mean(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
@@ -1115,7 +1261,8 @@ extern "C" int eden_mean(eden_ctx* ctx, const uint8_t* const* codes, const float
                          const uint32_t* const* recv_masks,
                          uint64_t d, uint32_t n, float* mean)
 {
-    return decode_common(ctx, codes, scales, bits, seeds, recv_masks, d, n, mean, true);
+    if (!bits) return EDEN_ERR_INVALID_ARG;
+    return decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, mean, true);
 }
 
 extern "C" int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bits,

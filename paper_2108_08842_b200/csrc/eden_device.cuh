@@ -21,9 +21,10 @@ struct ClientDesc {
     uint32_t subbit;         // 1 if b < 1
     uint32_t index;          // position of this client in the caller's arrays
     uint32_t coin_thr;       // non-integer b > 1: coin threshold round(frac * 65536); else 0
-    uint32_t pad_;
+    float delta;             // uniform-interval family (Section 4.3): interval width; else 0
     double extra_scale;      // encode: d/k for b < 1 (folded into S), else 1
     double mean_scale;       // decode: 1/n for the mean, 1 for accumulate
+    const float* utable;     // uniform-interval family: values of magnitude index 0..127; else nullptr
 };
 
 // Per-client values produced on the device.
@@ -88,6 +89,27 @@ __device__ __forceinline__ bool coin_bit(uint64_t seed, uint64_t i, uint32_t thr
     const uint32_t word = w == 0 ? r.x : w == 1 ? r.y : w == 2 ? r.z : r.w;
     const uint32_t half = (i & 1u) ? word >> 16 : word & 0xFFFFu;
     return half < threshold;
+}
+
+// Uniform-interval family I_Delta (Section 4.3): magnitude index of |z| = the number of
+// boundaries fl(delta * (k - 1/2)), k = 1..127, strictly below |z| (an endpoint belongs to
+// the interval nearer zero; indices beyond 127 fall into the open outermost interval).
+// The candidate floor(|z|/delta + 1/2) is at most one off; the two neighbouring boundaries,
+// formed exactly as defined, settle it.
+constexpr int kUniformMaxIndex = 127;
+__device__ __forceinline__ int uniform_magnitude(float az, float delta, float inv_delta)
+{
+    int c = (int)fminf(fmaf(az, inv_delta, 0.5f), (float)kUniformMaxIndex);
+    if (c >= 1 && !(az > __fmul_rn(delta, (float)c - 0.5f))) --c;
+    else if (c < kUniformMaxIndex && az > __fmul_rn(delta, (float)c + 0.5f)) ++c;
+    return c;
+}
+// value of a message byte: the byte is the signed index n, |n| <= 127 (-128 reads as -127)
+__device__ __forceinline__ float uniform_byte_value(uint32_t byte, const float* values)
+{
+    const int n = (int)(int8_t)byte;
+    const int m = min(n < 0 ? -n : n, kUniformMaxIndex);
+    return n < 0 ? -values[m] : values[m];
 }
 
 // The four 32-bit mask keys of input coordinates 4t .. 4t+3.

@@ -681,12 +681,45 @@ __device__ __forceinline__ void quantise_pack_frac(const u64 (&v)[16], float inv
     }
 }
 
+// Uniform-interval family (Section 4.3) on the row pass: one signed byte per coordinate
+// (the index n = round(z / delta), clamped to +-127), eight words per thread.
+__device__ __forceinline__ void quantise_pack_uniform(const u64 (&v)[16], float inv_norm, bool live, float delta,
+                                                      const float* s_tv, uint32_t (&words)[8], float& dot)
+{
+    const float inv_delta = __frcp_rn(delta);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) words[j] = 0u;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        float h[2];
+        unpack2(v[k], h[0], h[1]);
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int l = 2 * k + e;
+            const float z = h[e] * inv_norm;
+            const int m = uniform_magnitude(fabsf(z), delta, inv_delta);
+            dot = fmaf(fabsf(h[e]), s_tv[m], dot);
+            const uint32_t byte = (uint32_t)(z < 0.f ? -m : m) & 0xFFu;
+            words[l >> 2] |= byte << (8 * (l & 3));
+        }
+    }
+    if (!live) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) words[j] = 0u;
+    }
+}
+
 // Shared-memory tables of the row pass of the sender: positive boundaries and values of
 // width W, and of width W - 1 for non-integer budgets.
 template <int W, bool FRAC>
 struct EncTables {
     float tb[128], tv[128];
     float tb0[FRAC ? 64 : 1], tv0[FRAC ? 64 : 1];
+    // uniform-interval family (W = 8): the 128 values of this client by magnitude index
+    __device__ __forceinline__ void fill_uniform(int t, const float* __restrict__ values)
+    {
+        for (int j = t; j < 128; j += kFastThreads) tv[j] = values[j];
+    }
     __device__ __forceinline__ void fill(int t)
     {
         constexpr int half = 1 << (W - 1);
@@ -721,7 +754,7 @@ __device__ __forceinline__ void store_words(uint32_t* dst, const uint32_t (&word
 
 // The 13 stages of one tile held in arrangement A, then quantise, pack and store the tile's
 // code words; returns the thread's part of sum |h| Q(|z|).
-template <int W, bool FRAC>
+template <int W, bool FRAC, bool UNI = false>
 __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& cd, double n2, uint64_t base,
                                                u64* s, const EncTables<W, FRAC>& tab)
 {
@@ -737,7 +770,10 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
     const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
     uint32_t words[W];
     float dot = 0.f;
-    if constexpr (FRAC && W >= 2) {
+    if constexpr (UNI) {
+        static_assert(W == 8 && !FRAC, "the uniform-interval family sends one byte per coordinate");
+        quantise_pack_uniform(v, inv_norm, live, cd.delta, tab.tv, words, dot);
+    } else if constexpr (FRAC && W >= 2) {
         const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
         quantise_pack_frac<W>(v, inv_norm, live, coins, tab.tb, tab.tv, tab.tb0, tab.tv0, words, dot);
     } else {
@@ -747,7 +783,7 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
     return dot;
 }
 
-template <int W, int LC, bool FRAC>
+template <int W, int LC, bool FRAC, bool UNI = false>
 __global__ void __launch_bounds__(kFastThreads, 4)
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
 {
@@ -756,7 +792,8 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
     __shared__ EncTables<W, FRAC> tab;
     const ClientDesc cd = descs[blockIdx.y];
     const int t = threadIdx.x;
-    tab.fill(t);
+    if (UNI) tab.fill_uniform(t, cd.utable);
+    else tab.fill(t);
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
     u64 v[16];
     if (LC == 0) {
@@ -787,7 +824,7 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
         for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<0>(t, k))];
         __syncthreads();                               // s is rewritten by the next exchange
     }
-    const float dot = enc_last_tile<W, FRAC>(v, cd, states[blockIdx.y].norm2, base, s, tab);
+    const float dot = enc_last_tile<W, FRAC, UNI>(v, cd, states[blockIdx.y].norm2, base, s, tab);
     const double tot = block_sum((double)dot, red);
     if (t == 0) atomicAdd(&states[blockIdx.y].dot, tot);
 }
@@ -917,8 +954,11 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
     constexpr int half = 1 << (W - 1);
     for (int j = t; j < (2 << W); j += kFastThreads) {
         float c = 0.f;
-        if (j < (1 << W)) c = j >= half ? c_pos_value[table_offset(W) + j - half]
-                                         : -c_pos_value[table_offset(W) + half - 1 - j];
+        if (j < (1 << W)) {
+            if (W == 8 && cd.utable) c = uniform_byte_value((uint32_t)j, cd.utable);   // Section 4.3: the byte is the signed index
+            else c = j >= half ? c_pos_value[table_offset(W) + j - half]
+                               : -c_pos_value[table_offset(W) + half - 1 - j];
+        }
         s_val[j] = c;
     }
     if (FRAC && W >= 2)

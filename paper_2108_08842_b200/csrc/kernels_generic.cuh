@@ -154,9 +154,10 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     const int W = (int)cd.W, half = 1 << (W - 1);
     const bool frac = cd.coin_thr != 0u;       // then W = floor(b) + 1
     const int Wf = frac ? W - 1 : W;           // width of the fixed fields
+    const bool uniform = cd.utable != nullptr;  // Section 4.3: W = 8, the byte is the signed index
     for (int j = threadIdx.x; j < half; j += blockDim.x) {
         s_tb[j] = c_pos_boundary[table_offset(W) + j];
-        s_tv[j] = c_pos_value[table_offset(W) + j];
+        s_tv[j] = uniform ? cd.utable[j] : c_pos_value[table_offset(W) + j];
     }
     if (frac)
         for (int j = threadIdx.x; j < (half >> 1); j += blockDim.x) {
@@ -187,6 +188,7 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
     const int lane = threadIdx.x & 31;
     float dot = 0.f;
+    const float inv_delta = uniform ? __frcp_rn(cd.delta) : 0.f;
     const int Tr = (T + 31) & ~31;                     // whole warps take part in the reductions
     const uint64_t D = (uint64_t)1 << cd.L;
     const uint64_t total_words = frac ? ((D + 31) >> 5) * W : (D * W + 31) >> 5;
@@ -199,9 +201,10 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
         const int hw = wide ? half : half >> 1;
         const float* tb = wide ? s_tb : s_tb0;
         const float* tv = wide ? s_tv : s_tv0;
-        const int m = magnitude_index(fabsf(z), tb, hw);
+        const int m = uniform ? uniform_magnitude(fabsf(z), cd.delta, inv_delta) : magnitude_index(fabsf(z), tb, hw);
         const bool neg = z < 0.f;
         uint32_t code = neg ? (uint32_t)(hw - 1 - m) : (uint32_t)(hw + m);
+        if (uniform) code = (uint32_t)(neg ? -m : m) & 0xFFu;
         const float q = neg ? -tv[m] : tv[m];
         if (e < T) dot = fmaf(h, q, dot); else code = 0u;
         if (!live) code = 0u;
@@ -316,6 +319,7 @@ __device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i
         uint32_t code = cd.codes[bit >> 5] >> off;
         if (off + W > 32) code |= cd.codes[(bit >> 5) + 1] << (32 - off);
         code &= (1u << W) - 1u;
+        if (cd.utable) return uniform_byte_value(code, tv);
         return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
     }
     // non-integer budget: groups of 32 coordinates, W words each: (W-1)-bit fields, then the
@@ -349,7 +353,8 @@ k_dec_first(const ClientDesc* __restrict__ descs, PassGeom g)
     const ClientDesc cd = descs[blockIdx.y];
     const int T = 1 << g.lt;
     const int half = 1 << (cd.W - 1);
-    for (int j = threadIdx.x; j < half; j += blockDim.x) s_tv[j] = c_pos_value[table_offset(cd.W) + j];
+    for (int j = threadIdx.x; j < half; j += blockDim.x)
+        s_tv[j] = cd.utable ? cd.utable[j] : c_pos_value[table_offset(cd.W) + j];
     if (cd.coin_thr)
         for (int j = threadIdx.x; j < (half >> 1); j += blockDim.x)
             s_tv0[j] = c_pos_value[table_offset(cd.W - 1) + j];
@@ -389,7 +394,7 @@ k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restric
             const int half = 1 << (cd.W - 1);
             __syncthreads();
             for (int j = threadIdx.x; j < half; j += blockDim.x)
-                s_tv[j] = c_pos_value[table_offset(cd.W) + j];
+                s_tv[j] = cd.utable ? cd.utable[j] : c_pos_value[table_offset(cd.W) + j];
             if (cd.coin_thr)
                 for (int j = threadIdx.x; j < (half >> 1); j += blockDim.x)
                     s_tv0[j] = c_pos_value[table_offset(cd.W - 1) + j];
@@ -432,6 +437,48 @@ k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restric
             }
         }
     }
+}
+
+// =================================================================================
+// Uniform-interval family (Section 4.3): occurrences of each index value in a client's
+// message (D signed bytes), for the entropy coder's model and the coded-length estimate.
+// hist[client][n + 128] counts index n.  Per-warp histograms in shared memory, flushed once.
+// =================================================================================
+constexpr int kHistThreads = 256;
+constexpr int kHistBytesPerThread = 64;
+
+__global__ void __launch_bounds__(kHistThreads)
+k_index_hist(const int8_t* const* __restrict__ index, uint64_t D, uint32_t* __restrict__ hist)
+{
+    __shared__ uint32_t s_h[kHistThreads / 32][256];
+    const int t = threadIdx.x, warp = t >> 5;
+    for (int j = t; j < (kHistThreads / 32) * 256; j += kHistThreads) (&s_h[0][0])[j] = 0u;
+    __syncthreads();
+    const int8_t* __restrict__ src = index[blockIdx.y];
+    const uint64_t units = D >> 4;                              // 16-byte units
+    const uint64_t per_block = (uint64_t)kHistThreads * (kHistBytesPerThread / 16);
+    for (uint64_t u0 = (uint64_t)blockIdx.x * per_block; u0 < units; u0 += (uint64_t)gridDim.x * per_block) {
+#pragma unroll
+        for (int r = 0; r < kHistBytesPerThread / 16; ++r) {
+            const uint64_t u = u0 + (uint64_t)r * kHistThreads + t;
+            if (u < units) {
+                const uint4 w = reinterpret_cast<const uint4*>(src)[u];
+                const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 4; ++b)
+                        atomicAdd(&s_h[warp][(((words[a] >> (8 * b)) & 0xFFu) + 128u) & 0xFFu], 1u);
+            }
+        }
+    }
+    if (blockIdx.x == 0 && t < (int)(D & 15u))                  // D < 16: a few single bytes
+        atomicAdd(&s_h[0][((uint32_t)(uint8_t)src[(units << 4) + t] + 128u) & 0xFFu], 1u);
+    __syncthreads();
+    uint32_t total = 0u;
+#pragma unroll
+    for (int w = 0; w < kHistThreads / 32; ++w) total += s_h[w][t];
+    if (total) atomicAdd(&hist[(uint64_t)blockIdx.y * 256u + t], total);
 }
 
 }  // namespace eden

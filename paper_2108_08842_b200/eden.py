@@ -61,6 +61,14 @@ _sig("eden_client_stats", _int, [_vp, _u32, _vp])
 _sig("eden_launch_count", _u64, [_vp])
 _sig("eden_sparsification_mask_noalloc", _int, [_int, _vp, _u64, _u64, _f64, _vp])
 _sig("eden_strerror", ctypes.c_char_p, [_int])
+_sig("eden_uniform_entropy", _f64, [_f64])
+_sig("eden_uniform_delta", _f64, [_f64])
+_sig("eden_uniform_values", _int, [_f64, _vp])
+_sig("eden_uniform_index_bytes", _u64, [_u64])
+_sig("eden_encode_uniform", _int, [_vp, _vp, _u64, _u64, _u32, _vp, _vp, _vp, _vp])
+_sig("eden_decode_accumulate_uniform", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp, _vp])
+_sig("eden_mean_uniform", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp])
+_sig("eden_index_histogram", _int, [_vp, _vp, _u64, _u32, _vp])
 _sig("eden_profile_enable", _int, [_vp, _int])
 _sig("eden_force_generic_kernels", _int, [_vp, _int])
 _sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
@@ -69,6 +77,8 @@ _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctyp
 
 STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA, STATUS_TIMEOUT = 1, 2, 4, 8
 PACKET_COORDS = 1024
+UNIFORM_MAX_INDEX = 127
+UNIFORM_MIN_DELTA = 0.0625
 
 
 class EdenError(RuntimeError):
@@ -129,6 +139,26 @@ def table(W: int):
     b = np.zeros(max((1 << W) - 1, 1), dtype=np.float32)
     _check(_lib.eden_table(W, c.ctypes.data, b.ctypes.data))
     return c, b[: (1 << W) - 1]
+
+
+def uniform_entropy(delta: float) -> float:
+    return float(_lib.eden_uniform_entropy(float(delta)))
+
+
+def uniform_delta(bits: float) -> float:
+    """Delta_b of Section 4.3 (0.0 if outside the supported widths)."""
+    return float(_lib.eden_uniform_delta(float(bits)))
+
+
+def uniform_values(delta: float) -> np.ndarray:
+    """float32[128]: the value of each magnitude index, as the kernels use it."""
+    v = np.zeros(128, dtype=np.float32)
+    _check(_lib.eden_uniform_values(float(delta), v.ctypes.data))
+    return v
+
+
+def uniform_index_bytes(d: int) -> int:
+    return int(_lib.eden_uniform_index_bytes(d))
 
 
 def _f64s(v) -> np.ndarray:
@@ -198,6 +228,41 @@ class Context:
         _check(_lib.eden_encode(self._h, x.data_ptr(), x.stride(0), d, n, bits.ctypes.data,
                                 seeds.ctypes.data, tab, scales.data_ptr()))
         return codes, scales
+
+    def encode_uniform(self, x: torch.Tensor, delta, seeds, index: Optional[List[torch.Tensor]] = None,
+                       scales: Optional[torch.Tensor] = None):
+        """eden_encode_uniform: one int8 index per rotated coordinate.  Returns (index, scales)."""
+        assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1
+        n, d = x.shape
+        delta, seeds = _f64s(delta), _u64s(seeds)
+        assert len(delta) == n and len(seeds) == n
+        if index is None:
+            index = [torch.empty(uniform_index_bytes(d), dtype=torch.int8, device=x.device) for _ in range(n)]
+        if scales is None:
+            scales = torch.empty(n, dtype=torch.float32, device=x.device)
+        _check(_lib.eden_encode_uniform(self._h, x.data_ptr(), x.stride(0), d, n, delta.ctypes.data,
+                                        seeds.ctypes.data, _ptr_table(index), scales.data_ptr()))
+        return index, scales
+
+    def mean_uniform(self, index, scales, delta, seeds, d: int, recv_masks=None,
+                     out: Optional[torch.Tensor] = None):
+        if out is None:
+            out = torch.empty(d, dtype=torch.float32, device=scales.device)
+        return self._decode(_lib.eden_mean_uniform, index, scales, delta, seeds, recv_masks, d, out)
+
+    def decode_accumulate_uniform(self, index, scales, delta, seeds, d: int, acc: torch.Tensor, recv_masks=None):
+        used = _u32(0)
+        self._decode(_lib.eden_decode_accumulate_uniform, index, scales, delta, seeds, recv_masks, d, acc,
+                     extra=(ctypes.byref(used),))
+        return int(used.value)
+
+    def index_histogram(self, index, d: int, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """eden_index_histogram: int32 [n, 256], column v + 128 counts index v."""
+        n = len(index)
+        if out is None:
+            out = torch.empty((n, 256), dtype=torch.int32, device=index[0].device)
+        _check(_lib.eden_index_histogram(self._h, _ptr_table(index), d, n, out.data_ptr()))
+        return out
 
     # ------------------------------------------------------------------ receiver
     def _decode(self, fn, codes, scales, bits, seeds, recv_masks, d, out, extra=()):
@@ -311,3 +376,19 @@ def eden_mean(ctx: Context, codes, scales, bits, seeds, d, recv_masks=None, out=
 
 def eden_decode_accumulate(ctx: Context, codes, scales, bits, seeds, d, acc, recv_masks=None):
     return ctx.decode_accumulate(codes, scales, bits, seeds, d, acc, recv_masks)
+
+
+def eden_encode_uniform(ctx: Context, x, delta, seeds, index=None, scales=None):
+    return ctx.encode_uniform(x, delta, seeds, index, scales)
+
+
+def eden_mean_uniform(ctx: Context, index, scales, delta, seeds, d, recv_masks=None, out=None):
+    return ctx.mean_uniform(index, scales, delta, seeds, d, recv_masks, out)
+
+
+def eden_decode_accumulate_uniform(ctx: Context, index, scales, delta, seeds, d, acc, recv_masks=None):
+    return ctx.decode_accumulate_uniform(index, scales, delta, seeds, d, acc, recv_masks)
+
+
+def eden_index_histogram(ctx: Context, index, d, out=None):
+    return ctx.index_histogram(index, d, out)

@@ -132,3 +132,37 @@ def test_pass_plan_covers_every_index_bit(lib):
     assert lib.eden_pass_plan(0, 1.0, buf, 8, ctypes.byref(n)) == -1
     assert lib.eden_pass_plan(1 << 20, 9.0, buf, 8, ctypes.byref(n)) == -1
     assert lib.eden_pass_plan(1 << 30, 1.0, buf, 2, ctypes.byref(n)) == -1
+
+
+def test_uniform_family_host_figures_match_the_oracle(lib):
+    # Section 4.3: entropy of I_Delta, Delta_b and the interval values, host-only calls
+    lib.eden_uniform_entropy.restype = ctypes.c_double
+    lib.eden_uniform_entropy.argtypes = [ctypes.c_double]
+    lib.eden_uniform_delta.restype = ctypes.c_double
+    lib.eden_uniform_delta.argtypes = [ctypes.c_double]
+    lib.eden_uniform_values.argtypes = [ctypes.c_double, ctypes.c_void_p]
+    lib.eden_uniform_index_bytes.restype = ctypes.c_uint64
+    lib.eden_uniform_index_bytes.argtypes = [ctypes.c_uint64]
+    for delta in (0.0625, 0.3, 0.5224, 1.0, 1.99):
+        assert abs(lib.eden_uniform_entropy(delta) - O.uniform_entropy(delta)) < 1e-12
+        vals = np.zeros(128, dtype=np.float32)
+        assert lib.eden_uniform_values(delta, vals.ctypes.data) == 0
+        ref = np.array([O.uniform_value(delta, m) for m in range(128)]).astype(np.float32)
+        assert np.array_equal(vals, ref)
+    for bits in (1.3, 2.0, 3.0, 4.5, 6.0):
+        got, ref = lib.eden_uniform_delta(bits), O.uniform_delta(bits)
+        assert abs(got - ref) <= 1e-12 * ref
+    # outside the supported widths [1/16, 2)
+    assert lib.eden_uniform_delta(1.2) == 0.0 and lib.eden_uniform_delta(6.1) == 0.0
+    assert lib.eden_uniform_delta(float("nan")) == 0.0
+    vals = np.zeros(128, dtype=np.float32)
+    for bad in (0.0, 0.06, 2.0, float("nan")):
+        assert lib.eden_uniform_values(bad, vals.ctypes.data) == -2
+    assert lib.eden_uniform_values(0.5, None) == -1
+    for d in (1, 15, 16, 17, 1000, 10 ** 6):
+        D = O.rot_dim(d, 1.0)
+        assert lib.eden_uniform_index_bytes(d) == (D + 15) // 16 * 16
+    # entry points reject missing arguments before touching a device
+    assert lib.eden_encode_uniform(None, None, 0, 8, 1, None, None, None, None) == -1
+    assert lib.eden_mean_uniform(None, None, None, None, None, None, 8, 1, None) == -1
+    assert lib.eden_index_histogram(None, None, 8, 1, None) == -1
