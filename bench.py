@@ -59,6 +59,9 @@ def config_of(work, extra=None):
     cfg = {"workload": work.name, "n_clients": int(work.n), "d": int(work.d), "bits": bits,
            "packet_drop_prob": work.drop_prob, "value_law": work.description,
            "l2_policy": "inputs larger than L2 (no flush)"}
+    if getattr(work, "quantiser", None):
+        cfg["quantiser"] = work.quantiser
+        cfg.pop("bits")
     if extra:
         cfg.update(extra)
     return cfg
@@ -206,14 +209,39 @@ def run_gpu(args):
         masks_np = [work.recv_mask(c, eden.num_packets(d, float(bits[c]))) for c in range(n)]
         masks_gpu = [torch.from_numpy(m.view(np.int32)).to(dev) for m in masks_np]
     ctx = eden.Context(local_rank, d_max=d, n_batch=n, host_staging=True)
-    codes = ctx.alloc_codes(d, bits)
     scales = torch.empty(n, dtype=torch.float32, device=dev)
     mean = torch.empty(d, dtype=torch.float32, device=dev)
+    uniform = args.uniform_bits is not None
+    if uniform:
+        # Section 4.3's uniform-interval family: one index byte per rotated coordinate, and
+        # the histogram an entropy coder would be built from
+        delta = eden.uniform_delta(args.uniform_bits)
+        if delta == 0.0:
+            raise SystemExit("--uniform-bits: no supported interval width for this budget")
+        deltas = np.full(n, delta)
+        codes = [torch.empty(eden.uniform_index_bytes(d), dtype=torch.int8, device=dev) for _ in range(n)]
+        hist = torch.empty((n, 256), dtype=torch.int32, device=dev)
+        work.quantiser = "uniform intervals, b=%g, delta=%.6f" % (args.uniform_bits, delta)
+
+        def encode_step():
+            ctx.encode_uniform(x_gpu, deltas, seeds, codes, scales)
+            ctx.index_histogram(codes, d, hist)
+
+        def mean_step():
+            ctx.mean_uniform(codes, scales, deltas, seeds, d, masks_gpu, mean)
+    else:
+        codes = ctx.alloc_codes(d, bits)
+
+        def encode_step():
+            ctx.encode(x_gpu, bits, seeds, codes, scales)
+
+        def mean_step():
+            ctx.mean(codes, scales, bits, seeds, d, masks_gpu, mean)
     torch.cuda.synchronize()
 
     def step():
-        ctx.encode(x_gpu, bits, seeds, codes, scales)
-        ctx.mean(codes, scales, bits, seeds, d, masks_gpu, mean)
+        encode_step()
+        mean_step()
 
     def barrier():
         torch.cuda.synchronize()
@@ -238,9 +266,9 @@ def run_gpu(args):
     for _ in range(args.steps):
         a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
         a.record()
-        ctx.encode(x_gpu, bits, seeds, codes, scales)
+        encode_step()
         b.record()
-        ctx.mean(codes, scales, bits, seeds, d, masks_gpu, mean)
+        mean_step()
         c.record()
         t_events.append((a, b, c))
     barrier()
@@ -282,7 +310,7 @@ def run_gpu(args):
     # ---- end to end: same step through the host-buffer entry points (pinned memory),
     #      host->device and device->host copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not uniform:
         codes_h = [torch.empty(eden.code_bytes(d, float(b)), dtype=torch.uint8, pin_memory=True).numpy()
                    for b in bits]
         scales_h = torch.empty(n, dtype=torch.float32, pin_memory=True).numpy()
@@ -314,7 +342,7 @@ def run_gpu(args):
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not uniform:
         threads = min(cores, n, 8)
         d_s = min(d, 1 << 26)       # about 10-30 s of CPU work
         sample = synth.make(args.workload, d=d_s, n=threads, seed=rank)
@@ -352,6 +380,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (small profiling runs)")
     ap.add_argument("--d", type=int, default=None, help="override the dimension (sweeps)")
     ap.add_argument("--bits", type=float, default=None, help="override every client's bit budget (sweeps)")
+    ap.add_argument("--uniform-bits", type=float, default=None,
+                    help="use the uniform-interval family (Section 4.3) at this entropy budget instead of the "
+                         "Lloyd-Max tables; device-resident timing only (no end-to-end or CPU leg)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

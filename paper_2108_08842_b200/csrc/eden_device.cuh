@@ -94,15 +94,18 @@ __device__ __forceinline__ bool coin_bit(uint64_t seed, uint64_t i, uint32_t thr
 // Uniform-interval family I_Delta (Section 4.3): magnitude index of |z| = the number of
 // boundaries fl(delta * (k - 1/2)), k = 1..127, strictly below |z| (an endpoint belongs to
 // the interval nearer zero; indices beyond 127 fall into the open outermost interval).
-// The candidate floor(|z|/delta + 1/2) is at most one off; the two neighbouring boundaries,
-// formed exactly as defined, settle it.
+// The candidate floor(|z|/delta + 1/2 - 2^-10) is the index or one below it (the 2^-10
+// outweighs every rounding error of the candidate's arithmetic, which stays below 4e-5 for
+// quotients up to 127), so one comparison with the next boundary, formed exactly as
+// defined, settles it.  The floor is taken by adding 2^23 with rounding towards minus
+// infinity, which leaves the integer in the low mantissa bits and, as a float, in t - 2^23.
 constexpr int kUniformMaxIndex = 127;
 __device__ __forceinline__ int uniform_magnitude(float az, float delta, float inv_delta)
 {
-    int c = (int)fminf(fmaf(az, inv_delta, 0.5f), (float)kUniformMaxIndex);
-    if (c >= 1 && !(az > __fmul_rn(delta, (float)c - 0.5f))) --c;
-    else if (c < kUniformMaxIndex && az > __fmul_rn(delta, (float)c + 0.5f)) ++c;
-    return c;
+    const float u = fminf(fmaf(az, inv_delta, 0.5f - 0.0009765625f), (float)kUniformMaxIndex - 0.5f);
+    const float t = __fadd_rd(u, 8388608.f);                   // 2^23 + floor(u), floor(u) in 0..126
+    const float next = __fmul_rn(delta, t - 8388607.5f);       // boundary floor(u) + 1: delta * (floor(u) + 1/2)
+    return (int)(__float_as_uint(t) & 0xFFu) + (az > next ? 1 : 0);
 }
 // value of a message byte: the byte is the signed index n, |n| <= 127 (-128 reads as -127)
 __device__ __forceinline__ float uniform_byte_value(uint32_t byte, const float* values)

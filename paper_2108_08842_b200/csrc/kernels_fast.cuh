@@ -699,8 +699,12 @@ __device__ __forceinline__ void quantise_pack_uniform(const u64 (&v)[16], float 
             const float z = h[e] * inv_norm;
             const int m = uniform_magnitude(fabsf(z), delta, inv_delta);
             dot = fmaf(fabsf(h[e]), s_tv[m], dot);
-            const uint32_t byte = (uint32_t)(z < 0.f ? -m : m) & 0xFFu;
-            words[l >> 2] |= byte << (8 * (l & 3));
+            // two's complement of +-m by the sign bit of z (m = 0 gives 0 for either sign),
+            // its low byte moved into byte l % 4 of the word
+            const int sgn = (int)__float_as_uint(z) >> 31;
+            const uint32_t n = (uint32_t)((m ^ sgn) - sgn);
+            const uint32_t sel = (l & 3) == 0 ? 0x3214u : (l & 3) == 1 ? 0x3240u : (l & 3) == 2 ? 0x3410u : 0x4210u;
+            words[l >> 2] = __byte_perm(words[l >> 2], n, sel);
         }
     }
     if (!live) {
