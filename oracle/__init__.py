@@ -6,7 +6,7 @@ from the paper.  It shares nothing with the CUDA library and must not be importe
 the product package; only the tests, the smoke check and the benchmark's CPU-baseline
 leg may use it.
 
-Parity unpinned (conventions of this build, fixed only by oracle == GPU): the wire
+Parity unpinned (conventions of this implementation, fixed only by oracle == GPU): the wire
 layout of the packed codes, the Philox stream layout, and the tie-breaks at interval
 endpoints and at zero.  Everything else is pinned by ``tests/test_oracle_*.py``.
 """

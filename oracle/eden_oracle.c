@@ -19,7 +19,7 @@
  *   - Section 5:     the rotation is the randomized Hadamard transform
  *                    R = (1/sqrt D) H_D Diag(s).
  *
- * Conventions the paper leaves open (all are this build's reading; the ones marked
+ * Conventions the paper leaves open (all are readings chosen by this implementation; the ones marked
  * [unpinned] are pinned only by oracle == GPU):
  *   - H is the Sylvester matrix H[i][j] = (-1)^popcount(i & j); one transform.
  *   - d that is not a power of two is zero-padded to D = 2^ceil(log2 d'); all D
@@ -53,7 +53,7 @@
  *     everywhere else; indices are clamped to +-127, i.e. the family is made finite by
  *     letting the two outermost intervals run to infinity; the message is one signed
  *     byte per rotated coordinate (what an entropy coder would consume; the coder itself
- *     is not part of this build) plus S.  Boundary k is fl32(fl32(Delta) * (k - 1/2)).
+ *     is not implemented here) plus S.  Boundary k is fl32(fl32(Delta) * (k - 1/2)).
  *                                                       [clamp, byte layout unpinned]
  *   - The interval decision is taken after rounding z and the boundary to fp32,
  *     the precision the GPU kernels decide in; everything else is double.

@@ -180,7 +180,7 @@ extern "C" const char* eden_strerror(int code)
     switch (code) {
         case EDEN_OK: return "ok";
         case EDEN_ERR_INVALID_ARG: return "invalid argument";
-        case EDEN_ERR_UNSUPPORTED_BITS: return "unsupported bit budget (use 0 < b <= 1 or an integer 2..8)";
+        case EDEN_ERR_UNSUPPORTED_BITS: return "unsupported bit budget (0 < b <= 8) or interval width (1/16 <= Delta < 2)";
         case EDEN_ERR_CUDA: return "CUDA error";
         case EDEN_ERR_WORKSPACE: return "workspace too small";
         case EDEN_ERR_TOO_LARGE: return "dimension too large";
@@ -212,6 +212,7 @@ struct eden_ctx {
     std::vector<uint32_t> order;     // processing order of the last call: order[j] = client
     uint64_t states_off;             // where the last call put its ClientState array
     bool profiling;
+    bool profile_open;               // profile_begin recorded a start event that profile_end must close
     bool force_generic;
     int plan_variant;
     int row_staging;                 // 1: the sender's row pass runs in its persistent, bulk-copy-staged form
@@ -226,6 +227,7 @@ struct eden_ctx {
 
 static void profile_begin(eden_ctx* ctx, const char* name, double bytes)
 {
+    ctx->profile_open = false;
     if (!ctx->profiling) return;
     ProfileRecord r;
     r.name = name;
@@ -234,17 +236,23 @@ static void profile_begin(eden_ctx* ctx, const char* name, double bytes)
         r.start = ctx->event_pool[ctx->records.size()].first;
         r.stop = ctx->event_pool[ctx->records.size()].second;
     } else {
-        if (cudaEventCreate(&r.start) != cudaSuccess || cudaEventCreate(&r.stop) != cudaSuccess) return;
+        if (cudaEventCreate(&r.start) != cudaSuccess) return;
+        if (cudaEventCreate(&r.stop) != cudaSuccess) {
+            cudaEventDestroy(r.start);
+            return;
+        }
         ctx->event_pool.push_back({r.start, r.stop});
     }
     cudaEventRecord(r.start, ctx->stream);
     ctx->records.push_back(r);
+    ctx->profile_open = true;
 }
 
 static void profile_end(eden_ctx* ctx)
 {
-    if (!ctx->profiling || ctx->records.empty()) return;
+    if (!ctx->profile_open) return;
     cudaEventRecord(ctx->records.back().stop, ctx->stream);
+    ctx->profile_open = false;
 }
 
 #define CUDA_OK(expr)                                 \
@@ -277,6 +285,7 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->launches = 0;
     ctx->states_off = 0;
     ctx->profiling = false;
+    ctx->profile_open = false;
     ctx->copy_in = nullptr;
     ctx->copy_out = nullptr;
     ctx->force_generic = false;

@@ -1,7 +1,7 @@
 """Parity of the CUDA library against the CPU oracle, through the C ABI (via the thin
 binding), on seeded synthetic inputs.
 
-Tolerances (the ones the task fixes):
+Tolerances:
   * packed codes and sparsification masks bit-exact, except coordinates whose normalised
     value lies within 1e-6 * max(1, |t|) of an interval boundary t; those are counted and
     may only land in the neighbouring interval;
