@@ -587,21 +587,29 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
     } else {
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = 0u;
+    // coordinates in descending order, so that widths that divide 32 can shift the word up
+    // by one field and drop the code into the low bits
 #pragma unroll
-    for (int k = 0; k < 16; ++k) {
+    for (int k = 15; k >= 0; --k) {
         float h[2];
         unpack2(v[k], h[0], h[1]);
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
+        for (int e = 1; e >= 0; --e) {
             const int l = 2 * k + e;
             const float z = h[e] * inv_norm;
             const int m = fast_magnitude<W>(fabsf(z), s_tb);
             dot = fmaf(fabsf(h[e]), W <= 2 ? (m ? c_pos_value[half] : c_pos_value[half - 1]) : s_tv[m], dot);
-            // code = half + m for z >= 0 and half - 1 - m otherwise
-            const uint32_t code = (uint32_t)m ^ (z < 0.f ? half - 1u : half);
+            // code = half + m for z >= 0 and half - 1 - m otherwise: set the top bit, then
+            // flip all W bits where the sign bit of z is set
+            const uint32_t flip = (uint32_t)((int)__float_as_uint(z) >> 31) & (2u * half - 1u);
+            const uint32_t code = ((uint32_t)m | half) ^ flip;
             const int a = (l * W) >> 5, off = (l * W) & 31;
-            words[a] |= code << off;
-            if (off + W > 32) words[a + 1] |= code >> (32 - off);
+            if constexpr (32 % W == 0) {
+                words[a] = (words[a] << W) | code;
+            } else {
+                words[a] |= code << off;
+                if (off + W > 32) words[a + 1] |= code >> (32 - off);
+            }
         }
     }
     if (!live) {
