@@ -192,9 +192,16 @@ def run_gpu(args):
     __graft_entry__.build()
     from paper_2108_08842_b200 import eden, synth
 
-    work = synth.make(args.workload, d=args.d, n=args.n, seed=rank)
+    # replicas (default): every rank has a round of its own.  --sharded: one round, its
+    # senders split over the ranks, the mean finished by one all-reduce of d floats.
+    work = synth.make(args.workload, d=args.d, n=args.n, seed=0 if args.sharded else rank)
     if args.bits is not None:
         work.bits = np.full(work.n, float(args.bits))
+    n_total = work.n
+    if args.sharded:
+        if n_total < world:
+            raise SystemExit("--sharded needs at least one sender per rank")
+        work = work.share(replicas.shard_clients(n_total, rank, world))
     n, d = work.n, work.d
     cores = host_cores()
     dev = torch.device("cuda", local_rank)
@@ -235,8 +242,12 @@ def run_gpu(args):
         def encode_step():
             ctx.encode(x_gpu, bits, seeds, codes, scales)
 
-        def mean_step():
-            ctx.mean(codes, scales, bits, seeds, d, masks_gpu, mean)
+        if args.sharded:
+            def mean_step():
+                replicas.sharded_mean(ctx, codes, scales, bits, seeds, d, n_total, masks_gpu, mean)
+        else:
+            def mean_step():
+                ctx.mean(codes, scales, bits, seeds, d, masks_gpu, mean)
     torch.cuda.synchronize()
 
     def step():
@@ -282,7 +293,10 @@ def run_gpu(args):
     total_ms, enc_ms, dec_ms = replicas.max_over_ranks([total_ms, enc_ms, dec_ms], dev)
     ms_per_step = total_ms / args.steps
     in_bytes = n * d * 4
-    value = replicas.whole_job_gbs(world, in_bytes, ms_per_step)
+    if args.sharded:
+        value = n_total * d * 4 / (ms_per_step * 1e-3) / 1e9
+    else:
+        value = replicas.whole_job_gbs(world, in_bytes, ms_per_step)
 
     # ---- roofline of the dominant kernel (by event time inside the timed region)
     peak, peak_kind = measured_hbm_peak()
@@ -302,15 +316,19 @@ def run_gpu(args):
                     for k, v in sorted(kernels.items(), key=lambda kv: -kv[1]["ms"])}
 
     # ---- accuracy of the GPU estimate against the true mean (untimed)
-    true_mean = x_gpu.double().mean(dim=0)
-    nmse = float(((mean.double() - true_mean) ** 2).sum() / ((x_gpu.double() ** 2).sum() / n))
+    true_mean = x_gpu.double().sum(dim=0) / n_total
+    energy = (x_gpu.double() ** 2).sum() / n_total
+    if args.sharded and world > 1:
+        dist.all_reduce(true_mean)
+        dist.all_reduce(energy)
+    nmse = float(((mean.double() - true_mean) ** 2).sum() / energy)
     del true_mean
     status = ctx.status()
 
     # ---- end to end: same step through the host-buffer entry points (pinned memory),
     #      host->device and device->host copies inside the timed region
     e2e = None
-    if not args.no_e2e and not uniform:
+    if not args.no_e2e and not uniform and not args.sharded:
         codes_h = [torch.empty(eden.code_bytes(d, float(b)), dtype=torch.uint8, pin_memory=True).numpy()
                    for b in bits]
         scales_h = torch.empty(n, dtype=torch.float32, pin_memory=True).numpy()
@@ -342,7 +360,7 @@ def run_gpu(args):
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not uniform:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not uniform and not args.sharded:
         threads = min(cores, n, 8)
         d_s = min(d, 1 << 26)       # about 10-30 s of CPU work
         sample = synth.make(args.workload, d=d_s, n=threads, seed=rank)
@@ -354,8 +372,10 @@ def run_gpu(args):
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": config_of(work, {"parallelism": "replicas x%d" % world}),
+                "scaling": "strong" if args.sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": config_of(work, {"parallelism": ("senders split over %d ranks, one all-reduce" % world)
+                                           if args.sharded else "replicas x%d" % world,
+                                           "n_clients_total": int(n_total) * (1 if args.sharded else world)}),
                 "encode_gbs": in_bytes / (enc_ms * 1e-3) / 1e9, "decode_mean_gbs": in_bytes / (dec_ms * 1e-3) / 1e9,
                 "encode_ms": enc_ms, "decode_mean_ms": dec_ms,
                 "roofline": roofline, "kernels": kernel_table, "cpu_baseline": cpu, "e2e": e2e,
@@ -380,6 +400,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (small profiling runs)")
     ap.add_argument("--d", type=int, default=None, help="override the dimension (sweeps)")
     ap.add_argument("--bits", type=float, default=None, help="override every client's bit budget (sweeps)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="one round with its senders split over the ranks and the mean finished by an "
+                         "all-reduce (strong scaling) instead of independent replicas; device-resident timing only")
     ap.add_argument("--uniform-bits", type=float, default=None,
                     help="use the uniform-interval family (Section 4.3) at this entropy budget instead of the "
                          "Lloyd-Max tables; device-resident timing only (no end-to-end or CPU leg)")

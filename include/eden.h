@@ -163,6 +163,16 @@ int eden_mean(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
               const uint32_t* const* recv_masks,
               uint64_t d, uint32_t n, float* mean);
 
+/* This GPU's share of the mean when the n_total senders of a round are split over several
+ * GPUs (the senders are independent until the final sum, Section 2.2.2):
+ *     partial[i] = (1/n_total) sum over the n given clients of x_hat_c[i]     (overwritten)
+ * so that the element-wise sum of the partial vectors of all GPUs (one all-reduce of d
+ * floats, done by the caller) is the mean over all n_total senders.  n <= n_total. */
+int eden_mean_partial(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                      const double* bits, const uint64_t* seeds,
+                      const uint32_t* const* recv_masks,
+                      uint64_t d, uint32_t n, uint64_t n_total, float* partial);
+
 /* The sparsification mask of Section 4.1 for (seed, d, bits < 1) as a bitmap:
  * mask_bits dev, ceil(d/32) words, bit i of word i/32 = coordinate i is kept. */
 int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bits,

@@ -1081,9 +1081,10 @@ extern "C" int eden_encode_uniform(eden_ctx* ctx, const float* x, uint64_t ld_x,
 static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
                          const double* bits, const double* delta, const uint64_t* seeds,
                          const uint32_t* const* recv_masks, uint64_t d, uint32_t n,
-                         float* out, bool mean)
+                         float* out, uint64_t divisor /* 0: accumulate into out; else overwrite out with the sum / divisor */)
 {
     if (!ctx || !codes || !scales || !seeds || !out) return EDEN_ERR_INVALID_ARG;
+    const bool mean = divisor != 0;
     std::vector<ClientPlan> plan;
     int rc = plan_clients(d, n, bits, delta, plan);
     if (rc) return rc;
@@ -1123,7 +1124,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             cd.index = p.index;
             cd.coin_thr = p.coin_thr;
             cd.extra_scale = 1.0;
-            cd.mean_scale = mean ? 1.0 / (double)n : 1.0;
+            cd.mean_scale = mean ? 1.0 / (double)divisor : 1.0;
             descs.push_back(cd);
             ctx->order.push_back(p.index);
         }
@@ -1214,7 +1215,7 @@ extern "C" int eden_decode_accumulate(eden_ctx* ctx, const uint8_t* const* codes
                                       uint64_t d, uint32_t n, float* acc, uint32_t* n_used)
 {
     if (!bits) return EDEN_ERR_INVALID_ARG;
-    const int rc = decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, acc, false);
+    const int rc = decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, acc, 0);
     if (rc == EDEN_OK && n_used) *n_used = n;
     return rc;
 }
@@ -1226,7 +1227,7 @@ extern "C" int eden_decode_accumulate_uniform(eden_ctx* ctx, const int8_t* const
 {
     if (!delta) return EDEN_ERR_INVALID_ARG;
     const int rc = decode_common(ctx, (const uint8_t* const*)index, scales, nullptr, delta, seeds, recv_masks,
-                                 d, n, acc, false);
+                                 d, n, acc, 0);
     if (rc == EDEN_OK && n_used) *n_used = n;
     return rc;
 }
@@ -1238,7 +1239,7 @@ extern "C" int eden_mean_uniform(eden_ctx* ctx, const int8_t* const* index, cons
 {
     if (!delta) return EDEN_ERR_INVALID_ARG;
     return decode_common(ctx, (const uint8_t* const*)index, scales, nullptr, delta, seeds, recv_masks, d, n,
-                         mean, true);
+                         mean, n);
 }
 
 // How often each index value occurs in each client's message (Section 4.3: what an entropy
@@ -1271,7 +1272,16 @@ extern "C" int eden_mean(eden_ctx* ctx, const uint8_t* const* codes, const float
                          uint64_t d, uint32_t n, float* mean)
 {
     if (!bits) return EDEN_ERR_INVALID_ARG;
-    return decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, mean, true);
+    return decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, mean, n);
+}
+
+extern "C" int eden_mean_partial(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                                 const double* bits, const uint64_t* seeds,
+                                 const uint32_t* const* recv_masks,
+                                 uint64_t d, uint32_t n, uint64_t n_total, float* partial)
+{
+    if (!bits || n_total < n) return EDEN_ERR_INVALID_ARG;
+    return decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, partial, n_total);
 }
 
 extern "C" int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bits,

@@ -61,6 +61,7 @@ _sig("eden_client_stats", _int, [_vp, _u32, _vp])
 _sig("eden_launch_count", _u64, [_vp])
 _sig("eden_sparsification_mask_noalloc", _int, [_int, _vp, _u64, _u64, _f64, _vp])
 _sig("eden_strerror", ctypes.c_char_p, [_int])
+_sig("eden_mean_partial", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _u64, _vp])
 _sig("eden_uniform_entropy", _f64, [_f64])
 _sig("eden_uniform_delta", _f64, [_f64])
 _sig("eden_uniform_values", _int, [_f64, _vp])
@@ -281,6 +282,21 @@ class Context:
             out = torch.empty(d, dtype=torch.float32, device=scales.device)
         return self._decode(_lib.eden_mean, codes, scales, bits, seeds, recv_masks, d, out)
 
+    def mean_partial(self, codes, scales, bits, seeds, d: int, n_total: int, recv_masks=None,
+                     out: Optional[torch.Tensor] = None):
+        """eden_mean_partial: (1/n_total) * sum over the given clients; the partial vectors of
+        all GPUs add up to the mean over all n_total senders."""
+        if out is None:
+            out = torch.empty(d, dtype=torch.float32, device=scales.device)
+        n = len(codes)
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        assert len(bits) == n and len(seeds) == n
+        tab = _ptr_table(codes)
+        mtab = None if recv_masks is None else _ptr_table(recv_masks)
+        _check(_lib.eden_mean_partial(self._h, tab, scales.data_ptr(), bits.ctypes.data, seeds.ctypes.data, mtab,
+                                      d, n, int(n_total), out.data_ptr()))
+        return out
+
     def decode_accumulate(self, codes, scales, bits, seeds, d: int, acc: torch.Tensor, recv_masks=None):
         """eden_decode_accumulate: acc += sum_c x_hat_c; returns the number of clients counted."""
         used = _u32(0)
@@ -392,3 +408,7 @@ def eden_decode_accumulate_uniform(ctx: Context, index, scales, delta, seeds, d,
 
 def eden_index_histogram(ctx: Context, index, d, out=None):
     return ctx.index_histogram(index, d, out)
+
+
+def eden_mean_partial(ctx: Context, codes, scales, bits, seeds, d, n_total, recv_masks=None, out=None):
+    return ctx.mean_partial(codes, scales, bits, seeds, d, n_total, recv_masks, out)

@@ -82,11 +82,20 @@ class Workload:
     seed: int = 0
     description: str = ""
     _masks: Optional[List[Optional[np.ndarray]]] = field(default=None, repr=False)
+    _index: Optional[List[int]] = field(default=None, repr=False)   # a share: client j is sender _index[j] of the round
 
     def recv_mask(self, client: int, n_packets: int) -> Optional[np.ndarray]:
         if self.drop_prob <= 0.0:
             return None
-        return loss_mask(self.seed, client, n_packets, self.drop_prob)
+        sender = self._index[client] if self._index is not None else client
+        return loss_mask(self.seed, sender, n_packets, self.drop_prob)
+
+    def share(self, clients) -> "Workload":
+        """The part of this round made of the given senders: same vectors, seeds, budgets and
+        losses, renumbered from 0."""
+        idx = [int(c) for c in clients]
+        return Workload(self.name, len(idx), self.d, self.bits[idx], self.seeds[idx], self.drop_prob,
+                        lambda j: self.vector(idx[j]), self.seed, self.description, None, idx)
 
     def vectors(self) -> np.ndarray:
         """All senders' vectors as one float32[n, d] array."""

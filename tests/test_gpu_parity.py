@@ -375,3 +375,42 @@ def test_host_buffer_entry_points(E, d, n):
                    [torch.from_numpy(m.view(np.int32)).cuda() for m in masks]).cpu().numpy()
     assert np.array_equal(out, dev)
     ctx.close()
+
+
+def test_partial_means_of_two_shares_add_up_to_the_mean(E):
+    # the round's senders split over two receivers (here: two calls on one GPU): each
+    # share's eden_mean_partial divides by the round's sender count, the sum is the mean
+    from paper_2108_08842_b200 import replicas
+    d, n = 70001, 5
+    rng = np.random.default_rng(21)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    bits = [2.0, 0.5, 1.0, 4.0, 2.5]
+    seeds = [int(s) for s in synth.client_seeds(21, n)]
+    encs = O.encode_all([xs[c] for c in range(n)], bits, seeds, threads=4)
+    masks_np = []
+    for c in range(n):
+        packets = O.num_packets(O.rot_dim(d, bits[c]))
+        words = np.full((packets + 31) // 32, 0xFFFFFFFF, dtype=np.uint32)
+        words[0] &= ~np.uint32(1 << (c % 7))               # one lost packet each
+        masks_np.append(words)
+    ref, used = O.mean([e["codes"] for e in encs], [e["scale"] for e in encs], bits, seeds, d, masks_np, threads=4)
+    assert used == n
+    ctx = _ctx(E, d, n)
+    total = torch.zeros(d, dtype=torch.float32, device="cuda")
+    for rank in range(2):
+        mine = list(replicas.shard_clients(n, rank, 2))
+        codes = []
+        for c in mine:
+            buf = np.zeros(E.code_bytes(d, bits[c]), dtype=np.uint8)
+            buf[: encs[c]["codes"].nbytes] = encs[c]["codes"].view(np.uint8)
+            codes.append(torch.from_numpy(buf).cuda())
+        scales = torch.tensor([np.float32(encs[c]["scale"]) for c in mine], dtype=torch.float32, device="cuda")
+        masks = [torch.from_numpy(masks_np[c].view(np.int32)).cuda() for c in mine]
+        part = ctx.mean_partial(codes, scales, [bits[c] for c in mine], [seeds[c] for c in mine], d, n, masks)
+        total += part
+    assert ctx.status() == 0
+    err = np.max(np.abs(total.cpu().numpy().astype(np.float64) - ref))
+    assert err <= MEAN_TOL * np.max(np.abs(ref))
+    with pytest.raises(E.EdenError):
+        ctx.mean_partial(codes, scales, [bits[c] for c in mine], [seeds[c] for c in mine], d, 1, masks)
+    ctx.close()
