@@ -450,6 +450,35 @@ def test_nmse_of_mean_is_vnmse_over_n():
     assert abs(tot / rounds - limit) < 0.15 * limit, (tot / rounds, limit)
 
 
+def test_nmse_of_mean_with_unequal_budgets_and_norms_follows_lemma_2_2():
+    # NMSE = sum_c vNMSE(c) ||x_c||^2 / (n sum_c ||x_c||^2): senders with different budgets
+    # (Section 4.1) and different norms; d = 4096 keeps every rotation unpadded (k = 2048 at b = 0.5)
+    d = 4096
+    budgets = [0.5, 1.0, 1.0, 2.0, 3.0, 4.0]
+    norms = [3.0, 1.0, 0.2, 2.0, 5.0, 1.0]
+    n = len(budgets)
+    rng = np.random.default_rng(33)
+    xs = np.stack([rng.standard_normal(d) * s for s in norms]).astype(np.float32)
+    energy = (xs.astype(np.float64) ** 2).sum(axis=1)
+
+    def vnmse(b):
+        if b < 1:
+            return math.pi / (2 * b) - 1                      # Corollary 4.2
+        c, _, _, p = _levels(1 << int(b))
+        return 1 / (p * c * c).sum() - 1                      # Corollary 2.4
+    limit = sum(vnmse(b) * e for b, e in zip(budgets, energy)) / (n * energy.sum())
+    true = xs.astype(np.float64).mean(axis=0)
+    denom = energy.sum() / n
+    rounds, tot = 30, 0.0
+    for r in range(rounds):
+        seeds = [9000 + r * n + c for c in range(n)]
+        enc = [O.encode(xs[c], budgets[c], seeds[c]) for c in range(n)]
+        mean, used = O.mean([e["codes"] for e in enc], [e["scale"] for e in enc], budgets, seeds, d)
+        assert used == n
+        tot += np.dot(mean - true, mean - true) / denom
+    assert abs(tot / rounds - limit) < 0.15 * limit, (tot / rounds, limit)
+
+
 # ----------------------------------------------------------------------------- non-integer budgets b > 1
 def _coins_from_raw_philox(seed, D, bits):
     thr = int(math.floor((bits - math.floor(bits)) * 65536 + 0.5))
