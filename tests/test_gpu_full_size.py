@@ -110,3 +110,19 @@ def test_largest_tested_dimension_2_pow_28(E):
                           lambda c: x, 28)
     mism, _, _ = run_workload(E, work, threads=1)
     assert mism <= 120
+
+
+def test_uniform_family_at_cfg4_size_with_packet_loss(E):
+    # Section 4.3's quantiser at configuration 4's dimension and loss rate (eight clients
+    # keep the oracle to about a minute): every index byte, scale and the mean
+    from tests.test_gpu_uniform import run_uniform
+    work = synth.make("cfg4", n=8)
+    assert work.d == 1 << 24
+    xs = work.vectors()
+    delta = O.uniform_delta(3.0)
+    mism, status, encs, hist = run_uniform(E, xs, [delta] * work.n, work.seeds, drop=0.1, threads=THREADS)
+    assert status == 0 and mism <= 40
+    # empirical entropy of every client's message meets the 3-bit budget
+    f = hist.astype(np.float64) / (1 << 24)
+    ent = -np.sum(np.where(f > 0, f * np.log2(np.where(f > 0, f, 1.0)), 0.0), axis=1)
+    assert np.all(np.abs(ent - 3.0) < 0.01)
