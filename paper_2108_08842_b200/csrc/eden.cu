@@ -916,6 +916,19 @@ extern "C" int eden_pass_plan(uint64_t d, double bits, uint32_t* pass_bits, uint
 // ------------------------------------------------------------------------------------
 namespace {
 
+// The call's descriptors and, right behind them in the workspace, its zeroed per-client
+// state, in one copy (one stream operation less than a copy and a memset, which matters
+// for small rounds).
+int upload_descs_and_clear_states(eden_ctx* ctx, const CallLayout& lay, const std::vector<ClientDesc>& descs)
+{
+    const size_t n = descs.size();
+    const size_t bytes = (size_t)(lay.states_off - lay.descs_off) + sizeof(ClientState) * n;
+    std::vector<unsigned char> image(bytes, 0);
+    std::memcpy(image.data(), descs.data(), sizeof(ClientDesc) * n);
+    CUDA_OK(cudaMemcpyAsync(ctx->ws + lay.descs_off, image.data(), bytes, cudaMemcpyHostToDevice, ctx->stream));
+    return EDEN_OK;
+}
+
 // Values of the uniform-interval family for the clients in processing order, uploaded
 // behind the descriptors; sets each descriptor's table pointer and interval width.
 int upload_uniform_tables(eden_ctx* ctx, const CallLayout& lay, const std::vector<ClientPlan>& plan,
@@ -1000,8 +1013,8 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
         rc = upload_uniform_tables(ctx, lay, plan, ctx->order, descs);
         if (rc) return rc;
     }
-    CUDA_OK(cudaMemcpyAsync(d_descs, descs.data(), sizeof(ClientDesc) * n, cudaMemcpyHostToDevice, ctx->stream));
-    CUDA_OK(cudaMemsetAsync(d_states, 0, sizeof(ClientState) * n, ctx->stream));
+    rc = upload_descs_and_clear_states(ctx, lay, descs);
+    if (rc) return rc;
 
     for (size_t gi = 0; gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
@@ -1137,8 +1150,8 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         rc = upload_uniform_tables(ctx, lay, plan, ctx->order, descs);
         if (rc) return rc;
     }
-    CUDA_OK(cudaMemcpyAsync(d_descs, descs.data(), sizeof(ClientDesc) * n, cudaMemcpyHostToDevice, ctx->stream));
-    CUDA_OK(cudaMemsetAsync(d_states, 0, sizeof(ClientState) * n, ctx->stream));
+    rc = upload_descs_and_clear_states(ctx, lay, descs);
+    if (rc) return rc;
     LAUNCH(ctx, "dec_prep", n * 8.0, k_dec_prep, n, 256, 0, d_descs, d_states, scales, d_status);
 
     // the first group with b >= 1 covers every output coordinate, so for the mean it may
