@@ -145,7 +145,12 @@ extern "C" uint64_t eden_workspace_bytes(uint64_t d_max, uint32_t n_batch)
     // per client: descriptors, one intermediate vector, and (b < 1) the mask-selection scratch
     const uint64_t n_chunks = (d_max + kSelChunk - 1) / kSelChunk;
     const uint64_t sel = 256 + kHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) + 256;
-    return fixed_layout(d_max).end + align_up(per_client_bytes() * n_batch, 256) + 1024 +
+    // partial sums of the receiver's last pass when a round has too few tiles to fill the
+    // GPU (sized for 148 SMs; a split that does not fit is simply not used)
+    const uint64_t tiles = std::max<uint64_t>(1, D >> 13);
+    const uint64_t rows = std::min<uint64_t>(std::min<uint64_t>(n_batch, 16), (296 + tiles - 1) / tiles);
+    const uint64_t partials = rows >= 2 ? rows * align_up(d_max, 64) * sizeof(float) : 0;
+    return fixed_layout(d_max).end + align_up(per_client_bytes() * n_batch, 256) + 1024 + partials +
            (uint64_t)n_batch * (align_up(D * sizeof(float), 256) + sel + 512 /* uniform-family values */);
 }
 
@@ -782,8 +787,10 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
 }
 
 // Receiver passes of one group on the register-blocked path.
+// `part`/`part_bytes`: free workspace behind the group's work buffers, for partial sums.
 int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g,
-                      ClientDesc* d_descs, ClientState* d_states, float* out, uint64_t d, int mode)
+                      ClientDesc* d_descs, ClientState* d_states, float* out, uint64_t d, int mode,
+                      float* part, uint64_t part_bytes)
 {
     const uint32_t gn = (uint32_t)g.members.size();
     const double D = (double)(1ull << g.L);
@@ -805,12 +812,36 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
                 LAUNCH_CL(ctx, "f_mid", gn * 8.0 * D, (k_f_col<LR_, LC_, false>), dim3(tiles, gn),
                           dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo)));
         } else {
-            EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
-                LAUNCH_CL(ctx, "f_dec_last",
-                          gn * 4.0 * D + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<double>((double)d, D),
-                          (k_f_dec_last<LR_, LC_>), dim3(tiles, mode == OUT_YHAT ? gn : 1u), dim3(kFastThreads), ps.lc,
-                          (const ClientDesc*)d_descs, (const ClientState*)d_states, mode == OUT_YHAT ? 1u : gn,
-                          ps.lo, out, d, mode)));
+            // A round with few tiles leaves most SMs idle if every block walks all clients:
+            // split the clients over block rows, each row summing into a partial vector of
+            // its own, and add the partial vectors up afterwards (a fixed order, so the
+            // result does not depend on scheduling).
+            const uint64_t stride = align_up(d, 64);
+            uint32_t rows = 1, per = gn;
+            if (mode != OUT_YHAT && ps.lc == 0 && gn >= 2 && tiles < 2u * (unsigned)ctx->sm_count) {
+                const uint32_t want = std::min<uint32_t>(std::min<uint32_t>(gn, 16u),
+                                                         (2u * (unsigned)ctx->sm_count + tiles - 1) / tiles);
+                per = (gn + want - 1) / want;
+                rows = (gn + per - 1) / per;
+                if (rows < 2 || (uint64_t)rows * stride * sizeof(float) > part_bytes) { rows = 1; per = gn; }
+            }
+            if (rows > 1) {
+                EDEN_DISPATCH_LR(ps.lr,
+                    LAUNCH_CL(ctx, "f_dec_last", gn * 4.0 * D + rows * 4.0 * std::min<double>((double)d, D),
+                              (k_f_dec_last<LR_, 0>), dim3(tiles, rows), dim3(kFastThreads), 0,
+                              (const ClientDesc*)d_descs, (const ClientState*)d_states, per,
+                              ps.lo, part, d, (int)OUT_PART, gn, stride));
+                LAUNCH(ctx, "dec_sum", (rows + (mode == OUT_ACC ? 2.0 : 1.0)) * 4.0 * (double)d, k_sum_partials,
+                       (unsigned)((d + 1023) / 1024), 256, 0, (const float*)part, rows, stride, d, out,
+                       mode == OUT_ACC ? 1 : 0);
+            } else {
+                EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
+                    LAUNCH_CL(ctx, "f_dec_last",
+                              gn * 4.0 * D + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<double>((double)d, D),
+                              (k_f_dec_last<LR_, LC_>), dim3(tiles, mode == OUT_YHAT ? gn : 1u), dim3(kFastThreads), ps.lc,
+                              (const ClientDesc*)d_descs, (const ClientState*)d_states, mode == OUT_YHAT ? 1u : gn,
+                              ps.lo, out, d, mode, gn, (uint64_t)0)));
+            }
         }
     }
     return EDEN_OK;
@@ -1116,8 +1147,10 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
     descs.reserve(n);
     ctx->order.clear();
     std::vector<uint32_t> group_start;
+    std::vector<uint64_t> group_work_end;       // bytes of the work region the group's buffers take
     for (const Group& g : groups) {
         group_start.push_back((uint32_t)descs.size());
+        group_work_end.push_back(0);
         uint64_t off = 0;
         for (uint32_t m : g.members) {
             const ClientPlan& p = plan[m];
@@ -1125,6 +1158,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             std::memset(&cd, 0, sizeof(cd));
             cd.work = p.needs_work ? (float*)(ctx->ws + lay.work_off + off) : nullptr;
             if (p.needs_work) off += work_buffer_bytes(p.D);
+            group_work_end.back() = off;
             cd.src = nullptr;
             cd.codes = (uint32_t*)codes[p.index];
             cd.recv = recv_masks ? recv_masks[p.index] : nullptr;
@@ -1189,7 +1223,9 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         const uint32_t loop_n = g.subbit ? 1u : gn;
         const unsigned rows = g.subbit ? gn : 1u;
         if (fast_eligible(ctx, g)) {
-            rc = fast_decode_group(ctx, plan, g, d_descs + first, d_states + first, out, d, mode);
+            rc = fast_decode_group(ctx, plan, g, d_descs + first, d_states + first, out, d, mode,
+                                   (float*)(ctx->ws + lay.work_off + group_work_end[gi]),
+                                   lay.work_bytes - group_work_end[gi]);
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);

@@ -374,17 +374,22 @@ k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, 
 // =================================================================================
 // Receiver, last pass: for every client of the group finish the inverse transform of the
 // tile, apply sign and factor, add into registers; store the sum once (Sections 2.2.2,
-// 4.2).  mode: OUT_WRITE / OUT_ACC into out[0, d), or OUT_YHAT into the client's own work
-// buffer (b < 1: one block row per client, n_group = 1).
+// 4.2).  mode: OUT_WRITE / OUT_ACC into out[0, d), OUT_YHAT into the client's own work
+// buffer (b < 1: one block row per client), or OUT_PART: block row y sums clients
+// [y * n_group, min((y + 1) * n_group, n_members)) into out + y * part_stride.
 // =================================================================================
 template <int LR, int LC>
 __global__ void __launch_bounds__(kFastThreads, 2)
 k_f_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restrict__ states_in,
-             uint32_t n_group, int lo, float* __restrict__ out, uint64_t d, int mode)
+             uint32_t n_group, int lo, float* __restrict__ out, uint64_t d, int mode,
+             uint32_t n_members, uint64_t part_stride)
 {
-    // OUT_YHAT: block row y handles member y alone (n_group = 1)
-    const ClientDesc* __restrict__ descs = descs_in + (mode == OUT_YHAT ? blockIdx.y : 0);
-    const ClientState* __restrict__ states = states_in + (mode == OUT_YHAT ? blockIdx.y : 0);
+    // OUT_YHAT: block row y handles member y alone; OUT_PART: its own run of n_group members
+    const uint32_t first = mode == OUT_YHAT ? blockIdx.y : mode == OUT_PART ? blockIdx.y * n_group : 0u;
+    if (mode == OUT_YHAT) n_group = 1u;
+    if (mode == OUT_PART) n_group = min(n_group, n_members - first);
+    const ClientDesc* __restrict__ descs = descs_in + first;
+    const ClientState* __restrict__ states = states_in + first;
     __shared__ ulonglong2 s[2048];
     __shared__ uint32_t s_sign[256];
     const ColTile ct = col_tile<LR, LC>(blockIdx.x, lo);
@@ -424,7 +429,7 @@ k_f_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restr
         }
     }
     const uint64_t limit = mode == OUT_YHAT ? (1ull << descs[0].L) : d;
-    float* dst = mode == OUT_YHAT ? descs[0].work : out;
+    float* dst = mode == OUT_YHAT ? descs[0].work : mode == OUT_PART ? out + blockIdx.y * part_stride : out;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         const uint64_t i = LC == 0

@@ -341,7 +341,9 @@ __device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i
     return field >= (uint32_t)half0 ? tv0[field - half0] : -tv0[half0 - 1 - field];
 }
 
-enum OutMode { OUT_WRITE = 0, OUT_ACC = 1, OUT_YHAT = 2 };
+// OUT_PART: block row y sums its own run of the group's clients into partial vector y (the
+// partial vectors are added up by k_sum_partials): more blocks when a round has few tiles.
+enum OutMode { OUT_WRITE = 0, OUT_ACC = 1, OUT_YHAT = 2, OUT_PART = 3 };
 
 // First pass of the decode (a row pass over the low bits): unpack, centroid lookup,
 // lost packets to zero, low stages; writes the work buffer.
@@ -435,6 +437,30 @@ k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restric
                 if (mode == OUT_ACC) dst[i] += acc[k];
                 else dst[i] = acc[k];
             }
+        }
+    }
+}
+
+// out[i] (+)= sum over the G partial vectors of part[g * stride + i], i < d.
+__global__ void __launch_bounds__(256)
+k_sum_partials(const float* __restrict__ part, uint32_t G, uint64_t stride, uint64_t d,
+               float* __restrict__ out, int accumulate)
+{
+    const uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;      // group of four coordinates
+    const uint64_t i = q * 4;
+    if (i >= d) return;
+    if (i + 3 < d && (((uintptr_t)out) & 15u) == 0) {
+        float4 a = accumulate ? *reinterpret_cast<const float4*>(out + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t g = 0; g < G; ++g) {
+            const float4 v = *reinterpret_cast<const float4*>(part + g * stride + i);
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+        }
+        *reinterpret_cast<float4*>(out + i) = a;
+    } else {
+        for (uint64_t j = i; j < d && j < i + 4; ++j) {
+            float a = accumulate ? out[j] : 0.f;
+            for (uint32_t g = 0; g < G; ++g) a += part[g * stride + j];
+            out[j] = a;
         }
     }
 }

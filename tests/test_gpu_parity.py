@@ -180,6 +180,17 @@ def test_sender_row_pass_staged_by_bulk_copies(E, bits, monkeypatch):
     run_workload(E, work)
 
 
+@pytest.mark.parametrize("n,d", [(11, (1 << 17) - 9), (37, (1 << 15) + 5)])
+def test_many_clients_of_few_tiles_split_the_last_receiver_pass(E, n, d):
+    # with fewer tiles than the GPU has room for, the receiver's last pass spreads the clients
+    # over block rows that sum into partial vectors (37 clients over 13 rows: a ragged last row)
+    rng = np.random.default_rng(n)
+    xs = (rng.standard_normal((n, d)) * np.exp(rng.standard_normal((n, 1)))).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.full(n, 2.0), synth.client_seeds(n, n), 0.05,
+                          lambda c: xs[c], n)
+    run_workload(E, work, check_clients=range(n))
+
+
 @pytest.mark.parametrize("W", [1, 2, 3, 4, 5, 6, 7, 8])
 def test_every_code_width(E, W):
     d, n = 40000, 2
