@@ -1229,8 +1229,29 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);
-            LAUNCH(ctx, "dec_single", gn * code_bits_per_coord(plan, g) / 8.0 * (double)(1ull << g.L) + 4.0 * d, k_dec_last<true>, dim3(1, rows), kGenericThreads, sizeof(float) << g.L,
-                   d_descs + first, d_states + first, loop_n, rg, out, d, mode);
+            // many small clients: spread them over block rows with partial sums (see
+            // fast_decode_group), up to about two blocks per SM
+            const uint64_t stride = align_up(d, 64);
+            float* part = (float*)(ctx->ws + lay.work_off + group_work_end[gi]);
+            const uint64_t part_bytes = lay.work_bytes - group_work_end[gi];
+            uint32_t split_rows = 1, per = gn;
+            if (!g.subbit && gn >= 4) {
+                const uint32_t want = std::min<uint32_t>(gn / 2, 2u * (unsigned)ctx->sm_count);
+                per = (gn + want - 1) / want;
+                split_rows = (gn + per - 1) / per;
+                if (split_rows < 2 || (uint64_t)split_rows * stride * sizeof(float) > part_bytes) { split_rows = 1; per = gn; }
+            }
+            if (split_rows > 1) {
+                LAUNCH(ctx, "dec_single", gn * code_bits_per_coord(plan, g) / 8.0 * (double)(1ull << g.L) + split_rows * 4.0 * d,
+                       k_dec_last<true>, dim3(1, split_rows), kGenericThreads, sizeof(float) << g.L,
+                       d_descs + first, d_states + first, per, rg, part, d, (int)OUT_PART, gn, stride);
+                LAUNCH(ctx, "dec_sum", (split_rows + (mode == OUT_ACC ? 2.0 : 1.0)) * 4.0 * (double)d, k_sum_partials,
+                       (unsigned)((d + 1023) / 1024), 256, 0, (const float*)part, split_rows, stride, d, out,
+                       mode == OUT_ACC ? 1 : 0);
+            } else {
+                LAUNCH(ctx, "dec_single", gn * code_bits_per_coord(plan, g) / 8.0 * (double)(1ull << g.L) + 4.0 * d, k_dec_last<true>, dim3(1, rows), kGenericThreads, sizeof(float) << g.L,
+                       d_descs + first, d_states + first, loop_n, rg, out, d, mode, gn, (uint64_t)0);
+            }
         } else {
             const int lc = kGenericTileLog;
             LAUNCH(ctx, "dec_first", gn * (4.0 + code_bits_per_coord(plan, g) / 8.0) * (double)(1ull << g.L), k_dec_first, dim3((unsigned)((1ull << g.L) >> lc), gn), kGenericThreads,
@@ -1245,7 +1266,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
                            d_descs + first, cg);
                 else
                     LAUNCH(ctx, "dec_last", gn * 4.0 * (double)(1ull << g.L) + (mode == OUT_ACC ? 8.0 : 4.0) * std::min<uint64_t>(d, 1ull << g.L), k_dec_last<false>, dim3(tiles, rows), kGenericThreads, sizeof(float) << cg.lt,
-                           d_descs + first, d_states + first, loop_n, cg, out, d, mode);
+                           d_descs + first, d_states + first, loop_n, cg, out, d, mode, gn, (uint64_t)0);
             }
         }
         if (g.subbit) {

@@ -378,11 +378,15 @@ k_dec_first(const ClientDesc* __restrict__ descs, PassGeom g)
 template <bool FROM_CODES>
 __global__ void __launch_bounds__(kGenericThreads)
 k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restrict__ states_in,
-           uint32_t n_group, PassGeom g, float* __restrict__ out, uint64_t d, int mode)
+           uint32_t n_group, PassGeom g, float* __restrict__ out, uint64_t d, int mode,
+           uint32_t n_members, uint64_t part_stride)
 {
-    // OUT_YHAT: block row y handles member y alone (n_group = 1)
-    const ClientDesc* __restrict__ descs = descs_in + (mode == OUT_YHAT ? blockIdx.y : 0);
-    const ClientState* __restrict__ states = states_in + (mode == OUT_YHAT ? blockIdx.y : 0);
+    // OUT_YHAT: block row y handles member y alone (n_group = 1); OUT_PART: block row y sums
+    // members [y * n_group, min((y + 1) * n_group, n_members)) into out + y * part_stride
+    const uint32_t first = mode == OUT_YHAT ? blockIdx.y : mode == OUT_PART ? blockIdx.y * n_group : 0u;
+    if (mode == OUT_PART) n_group = min(n_group, n_members - first);
+    const ClientDesc* __restrict__ descs = descs_in + first;
+    const ClientState* __restrict__ states = states_in + first;
     extern __shared__ float s[];
     __shared__ float s_tv[128], s_tv0[64];
     const int T = 1 << g.lt;
@@ -427,7 +431,7 @@ k_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restric
         __syncthreads();
     }
     const uint64_t limit = mode == OUT_YHAT ? (1ull << descs[0].L) : d;
-    float* dst = mode == OUT_YHAT ? descs[0].work : out;
+    float* dst = mode == OUT_YHAT ? descs[0].work : mode == OUT_PART ? out + blockIdx.y * part_stride : out;
 #pragma unroll
     for (int k = 0; k < kGenericPerThread; ++k) {
         const int e = threadIdx.x + k * kGenericThreads;
