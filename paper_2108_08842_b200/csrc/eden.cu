@@ -736,7 +736,8 @@ int resident_blocks(const eden_ctx* ctx, K kernel, uint32_t dynamic_smem)
 }
 
 // Sender passes of one group on the register-blocked path.
-int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g,
+// `h_descs`: the host copy of the group's descriptors (d_descs is the same array on the device).
+int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g, const ClientDesc* h_descs,
                       ClientDesc* d_descs, ClientState* d_states, uint64_t d, uint32_t* d_status)
 {
     const uint32_t gn = (uint32_t)g.members.size();
@@ -760,9 +761,13 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
+        // the row pass addresses client j of the run at work0 + j * 2^L
+        for (uint32_t j = 0; j < r.count; ++j)
+            if (h_descs[r.first + j].work != h_descs[r.first].work + ((uint64_t)j << g.L)) return EDEN_ERR_INVALID_ARG;
         if (g.uniform) {
             LAUNCH(ctx, "f_enc_last", r.count * 5.0 * D, (k_f_enc_last<8, 0, false, true>), dim3(tiles, r.count),
-                   kFastThreads, 0, (const ClientDesc*)(d_descs + r.first), d_states + r.first);
+                   kFastThreads, 0, (const ClientDesc*)(d_descs + r.first), d_states + r.first,
+                   (const float*)h_descs[r.first].work, g.L);
             continue;
         }
         if (ctx->row_staging && pl.row_lc == 0) {
@@ -781,7 +786,8 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
         EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
             LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_, FRAC_>),
                       dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
-                      (const ClientDesc*)(d_descs + r.first), d_states + r.first))));
+                      (const ClientDesc*)(d_descs + r.first), d_states + r.first,
+                      (const float*)h_descs[r.first].work, g.L))));
     }
     return EDEN_OK;
 }
@@ -1072,7 +1078,7 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
                    dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
         }
         if (fast_eligible(ctx, g) && (x_aligned || g.subbit)) {
-            rc = fast_encode_group(ctx, plan, g, d_descs + first, d_states + first, d, d_status);
+            rc = fast_encode_group(ctx, plan, g, descs.data() + first, d_descs + first, d_states + first, d, d_status);
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);

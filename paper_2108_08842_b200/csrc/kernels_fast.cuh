@@ -59,6 +59,9 @@ __device__ __forceinline__ void cluster_sync_execution()
 
 typedef unsigned long long u64;
 
+// 32-bit shared-memory address of a pointer into shared memory
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
 // ---------------------------------------------------------------------------------
 // packed fp32 pairs
 // ---------------------------------------------------------------------------------
@@ -487,6 +490,11 @@ __device__ __forceinline__ int slice_u(int rank, int t, int k)
     return rank * (4096 >> LC) + t + 256 * (k & ((16 >> LC) - 1));
 }
 
+// Between arrangements B and C a unit moves only inside a group of 16 consecutive threads
+// (unit t << 4 | k of arrangement C sits in thread (t & ~15) | k of arrangement B), so that
+// exchange is ordered by a warp barrier; A <-> B crosses warps and takes the block barrier.
+// A thread writes arrangement FROM at the addresses it read last in that arrangement, so
+// back-to-back exchanges need no barrier between them.
 template <int FROM, int TO>
 __device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
 {
@@ -499,7 +507,8 @@ __device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
 #pragma unroll
         for (int k = 0; k < 16; ++k) s[row_pad(row_u<FROM>(t, k))] = v[k];
     }
-    __syncthreads();
+    if (FROM + TO == 3) __syncwarp();
+    else __syncthreads();
     if (TO == 2) {
         const ulonglong2* p = reinterpret_cast<const ulonglong2*>(s + row_pad(row_u<2>(t, 0)));
 #pragma unroll
@@ -779,7 +788,6 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
     row_step<0>(v);                 // e bits 12..9
     row_exchange<0, 1>(v, s);
     row_step<0>(v);                 // e bits 8..5
-    __syncthreads();
     row_exchange<1, 2>(v, s);
     row_step<0>(v);                 // e bits 4..1
     row_step_inner(v);              // e bit 0
@@ -800,24 +808,28 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
     return dot;
 }
 
+// `work0`: the intermediate vector of the launch's first client; the clients' vectors follow
+// one another 2^L floats apart, so a block's tile address needs no descriptor and its loads
+// start at once.
 template <int W, int LC, bool FRAC, bool UNI = false>
 __global__ void __launch_bounds__(kFastThreads, 4)
-k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states)
+k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ double red[32];
     __shared__ EncTables<W, FRAC> tab;
-    const ClientDesc cd = descs[blockIdx.y];
     const int t = threadIdx.x;
-    if (UNI) tab.fill_uniform(t, cd.utable);
-    else tab.fill(t);
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
     u64 v[16];
     if (LC == 0) {
-        const u64* __restrict__ src = reinterpret_cast<const u64*>(cd.work + base);
+        const u64* __restrict__ src = reinterpret_cast<const u64*>(work0 + ((uint64_t)blockIdx.y << L) + base);
 #pragma unroll
         for (int k = 0; k < 16; ++k) v[k] = src[row_u<0>(t, k)];
-    } else {
+    }
+    const ClientDesc cd = descs[blockIdx.y];
+    if (UNI) tab.fill_uniform(t, cd.utable);
+    else tab.fill(t);
+    if (LC != 0) {
         // fetch this block's slice of all tiles of the cluster, do the stages across the
         // tiles, hand every result to the block that owns its tile
         cg::cluster_group cluster = cg::this_cluster();
@@ -855,8 +867,6 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
 // one before it.  Every wait on the mbarrier is bounded; a wait that runs out raises
 // EDEN_STATUS_TIMEOUT and the block returns.
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
@@ -1049,7 +1059,6 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
     row_step<0>(v);                 // e bits 4..1
     row_exchange<2, 1>(v, s);
     row_step<0>(v);                 // e bits 8..5
-    __syncthreads();
     row_exchange<1, 0>(v, s);
     row_step<0>(v);                 // e bits 12..9
     if (LC == 0) {
