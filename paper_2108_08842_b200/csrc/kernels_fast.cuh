@@ -382,7 +382,11 @@ k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, 
 // [y * n_group, min((y + 1) * n_group, n_members)) into out + y * part_stride.
 // =================================================================================
 template <int LR, int LC>
-__global__ void __launch_bounds__(kFastThreads, 2)
+// Three resident blocks per SM where the pass has an exchange (more than three row bits):
+// the extra warps cover the exchange and the per-client load latency (cfg5's shape, six
+// bits: 4990 -> 5520 GB/s at the price of a few spilled registers); two where it has none
+// and the registers matter more (cfg4's shape, three bits: 5870 GB/s against 5640).
+__global__ void __launch_bounds__(kFastThreads, (LR > 3 ? 3 : 2))
 k_f_dec_last(const ClientDesc* __restrict__ descs_in, const ClientState* __restrict__ states_in,
              uint32_t n_group, int lo, float* __restrict__ out, uint64_t d, int mode,
              uint32_t n_members, uint64_t part_stride)
@@ -739,8 +743,8 @@ __device__ __forceinline__ void quantise_pack_uniform(const u64 (&v)[16], float 
 // width W, and of width W - 1 for non-integer budgets.
 template <int W, bool FRAC>
 struct EncTables {
-    float tb[128], tv[128];
-    float tb0[FRAC ? 64 : 1], tv0[FRAC ? 64 : 1];
+    float tb[1 << (W - 1)], tv[1 << (W - 1)];
+    float tb0[FRAC && W > 1 ? 1 << (W - 2) : 1], tv0[FRAC && W > 1 ? 1 << (W - 2) : 1];
     // uniform-interval family (W = 8): the 128 values of this client by magnitude index
     __device__ __forceinline__ void fill_uniform(int t, const float* __restrict__ values)
     {
@@ -812,7 +816,11 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
 // one another 2^L floats apart, so a block's tile address needs no descriptor and its loads
 // start at once.
 template <int W, int LC, bool FRAC, bool UNI = false>
-__global__ void __launch_bounds__(kFastThreads, 4)
+// Five resident blocks per SM for integer budgets (51 registers; at most a few words
+// spilled): cfg5's shape 3240 -> 3370 GB/s, cfg4's 5000 -> 5090 GB/s.  Six fit as well but
+// run slower (2940 / 4310 GB/s): 230 KB of shared memory leave the SM almost no L1 to land
+// the tiles' loads in.  The non-integer budgets keep four (their coins cost registers).
+__global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : 5))
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
