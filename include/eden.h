@@ -65,6 +65,8 @@ extern "C" {
 #define EDEN_STATUS_NONFINITE    0x2u  /* some client's norm was inf/nan: its output is unspecified */
 #define EDEN_STATUS_NO_DATA      0x4u  /* some client had no packet received: it was skipped */
 #define EDEN_STATUS_TIMEOUT      0x8u  /* a bounded wait inside a kernel ran out: the call's output is unspecified */
+#define EDEN_STATUS_SCRATCH      0x10u /* a b < 1 mask selection outgrew its candidate list (sized for a margin of
+                                          twelve standard deviations): that client's mask, and so its output, is unspecified */
 
 #define EDEN_PACKET_COORDS 1024u
 #define EDEN_MAX_DIM       (1ull << 30)

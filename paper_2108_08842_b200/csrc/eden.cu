@@ -499,11 +499,25 @@ uint64_t work_buffer_bytes(uint64_t D) { return align_up(D * sizeof(float), 256)
 constexpr uint64_t kBatchHistBytes = 3ull * kSelBins * sizeof(uint32_t);
 
 // Scratch of the exact-size mask selection for one client with b < 1.
+constexpr uint64_t kCandBytes = (uint64_t)kSelCandCap * sizeof(uint2);
+
+// The two-pass selection holds the keys that share tau's first digit, about d / 2048 of
+// them (a binomial count): used while that, with a margin of many standard deviations,
+// fits the candidate list.
+bool two_pass_selection(uint64_t d)
+{
+    // EDEN_SEL_ROUNDS=3 keeps the three histogram rounds at every size (tuning and tests)
+    if (const char* e = std::getenv("EDEN_SEL_ROUNDS"))
+        if (std::atoi(e) == 3) return false;
+    const double mean = (double)d / (double)kSelBins;
+    return mean + 12.0 * std::sqrt(mean) + 64.0 <= (double)kSelCandCap;
+}
+
 uint64_t sel_scratch_bytes(uint64_t d)
 {
     const uint64_t n_chunks = (d + kSelChunk - 1) / kSelChunk;
     return 256 + kBatchHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) +
-           align_up(sizeof(SelJob), 256);
+           align_up(sizeof(SelJob), 256) + (two_pass_selection(d) ? kCandBytes : 0);
 }
 
 // Groups: clients of one rotation dimension (and, within it, of one kind: b >= 1 or
@@ -900,11 +914,14 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
     char* hist_base = sel_base + 256ull * n;
     char* chunk_base = hist_base + kBatchHistBytes * n;
     char* job_base = chunk_base + chunk_bytes * n;
+    char* cand_base = job_base + align_up(sizeof(SelJob), 256) * n;
+    const bool two_pass = two_pass_selection(d);
     std::vector<SelJob> jobs(partial);
     for (uint32_t j = 0; j < n; ++j) {
         jobs[j].sel = (MaskSelect*)(sel_base + 256ull * j);
         jobs[j].hist = (uint32_t*)(hist_base + kBatchHistBytes * j);
         jobs[j].chunks = (unsigned long long*)(chunk_base + chunk_bytes * j);
+        jobs[j].cand = two_pass ? (uint2*)(cand_base + kCandBytes * j) : nullptr;
     }
     batch.d_jobs = (SelJob*)job_base;
     batch.n = n;
@@ -914,6 +931,17 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
     CUDA_OK(cudaMemcpyAsync(batch.d_jobs, jobs.data(), sizeof(SelJob) * n, cudaMemcpyHostToDevice, ctx->stream));
     CUDA_OK(cudaMemsetAsync(hist_base, 0, kBatchHistBytes * n, ctx->stream));
     const double keys = (double)n * (double)d;
+    if (two_pass) {
+        uint32_t* d_status = (uint32_t*)(ctx->ws + fixed_layout(1).status);
+        LAUNCH(ctx, "sel_hist", 0, k_selc_hist, dim3(hist_grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs);
+        LAUNCH(ctx, "sel_find", n * (double)kSelBins * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, 0);
+        LAUNCH(ctx, "sel_collect", keys / 128.0, k_selc_collect, dim3(batch.grid, n), kSelThreads, 0,
+               (const SelJob*)batch.d_jobs);
+        LAUNCH(ctx, "sel_resolve", keys / 256.0, k_selc_resolve, n, 1024, 0, (const SelJob*)batch.d_jobs, d_status);
+        LAUNCH(ctx, "sel_chunk_scan", keys / 64.0, k_selb_chunk_scan, n, 1024, 0, (const SelJob*)batch.d_jobs,
+               (uint64_t)batch.grid);
+        return EDEN_OK;
+    }
     for (int round = 0; round < 3; ++round) {
         LAUNCH(ctx, "sel_hist", 0, k_selb_hist, dim3(hist_grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs, round);
         LAUNCH(ctx, "sel_find", n * (double)kSelBins * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, round);

@@ -214,6 +214,7 @@ struct SelJob {
     unsigned long long* chunks;      // one packed count per 1024 coordinates
     const float* in;                 // compact: the client's input row; scatter: its estimate of the kept coordinates
     float* out;                      // compact: the compacted vector
+    uint2* cand;                     // two-pass selection: (key, coordinate) of the keys that share tau's first digit
 };
 
 // Batched selection finds the k-th smallest key in three digit rounds of 10, 11 and 11
@@ -360,6 +361,130 @@ k_selb_chunk_scan(const SelJob* __restrict__ jobs, uint64_t n_chunks)
         const unsigned long long v = chunk_counts[j];
         chunk_counts[j] = run;
         run += v;
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// Two-pass selection (vectors short enough for the candidate list, kSelCandCap).  The
+// first digit of tau, the top 11 bits, comes from one histogram round as above.  The second
+// pass over the keys does two things at once: it counts, per chunk of 1024 coordinates, the
+// keys whose first digit is smaller (they are below tau whatever its other bits are), and it
+// appends the keys that share the digit, about one in 2048, to the job's candidate list with
+// their coordinates.  One block per job then finds tau's remaining 21 bits among the
+// candidates alone and adds each candidate below (or equal to) tau to its chunk's count.
+// The keys are generated three times per side (histogram, this pass, compaction or scatter)
+// instead of five.  job.hist[kSelBins] counts the candidates (zeroed with the histograms).
+// ---------------------------------------------------------------------------------
+constexpr int kSelFirstShift = 21;                     // first digit = key >> 21 (11 bits, kSelBins bins)
+constexpr uint32_t kSelCandCap = 61440;                // candidates a job can hold (480 KB)
+constexpr uint32_t kStatusScratch = 0x10u;             // EDEN_STATUS_SCRATCH
+
+__global__ void __launch_bounds__(kSelThreads)
+k_selc_hist(const SelJob* __restrict__ jobs)
+{
+    __shared__ uint32_t s_hist[kSelBins];
+    const SelJob job = jobs[blockIdx.y];
+    const uint64_t calls = (job.d + 3) / 4;
+    const uint64_t first = (uint64_t)blockIdx.x * kSelThreads * kSelCallsPerThread;
+    if (first >= calls) return;
+    for (int b = threadIdx.x; b < kSelBins; b += kSelThreads) s_hist[b] = 0u;
+    __syncthreads();
+    for (int it = 0; it < kSelCallsPerThread; ++it) {
+        const uint64_t t = first + (uint64_t)it * kSelThreads + threadIdx.x;
+        if (t >= calls) break;
+        const uint4 k4 = mask_keys(job.seed, t);
+        const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (t * 4 + j < job.d) atomicAdd(&s_hist[keys[j] >> kSelFirstShift], 1u);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < kSelBins; b += kSelThreads)
+        if (s_hist[b]) atomicAdd(&job.hist[b], s_hist[b]);
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+k_selc_collect(const SelJob* __restrict__ jobs)
+{
+    __shared__ unsigned long long scratch[33];
+    const SelJob job = jobs[blockIdx.y];
+    const uint32_t digit = job.sel->bin_hi;
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint4 k4 = mask_keys(job.seed, t);
+    const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
+    unsigned long long mine = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint64_t i = t * 4 + j;
+        if (i >= job.d) break;
+        const uint32_t top = keys[j] >> kSelFirstShift;
+        if (top < digit) {
+            ++mine;
+        } else if (top == digit) {
+            const uint32_t slot = atomicAdd(&job.hist[kSelBins], 1u);
+            if (slot < kSelCandCap) job.cand[slot] = make_uint2(keys[j], (uint32_t)i);
+        }
+    }
+    unsigned long long total;
+    block_exclusive_scan(mine, scratch, &total);
+    if (threadIdx.x == 0) job.chunks[blockIdx.x] = total;
+}
+
+// One block of 1024 threads per job.
+__global__ void __launch_bounds__(1024)
+k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status)
+{
+    __shared__ uint32_t s_hist[kSelBins];
+    __shared__ unsigned long long scratch[33];
+    __shared__ uint32_t s_bin, s_before;
+    const SelJob job = jobs[blockIdx.x];
+    MaskSelect* sel = job.sel;
+    const uint32_t found = job.hist[kSelBins];
+    const uint32_t n = min(found, kSelCandCap);
+    if (found > kSelCandCap && threadIdx.x == 0) atomicOr(status, kStatusScratch);
+    const uint32_t digit = sel->bin_hi;
+    uint32_t below = sel->below_hi;                    // keys below everything fixed so far
+    uint32_t prefix = digit;                           // the bits of tau fixed so far
+    int fixed = 32 - kSelFirstShift;                   // how many they are
+    // the remaining 21 bits in two digits of 11 and 10 bits
+    for (int round = 0; round < 2; ++round) {
+        const int bits = round == 0 ? 11 : 10;
+        const int shift = 32 - fixed - bits;
+        for (int b = threadIdx.x; b < kSelBins; b += blockDim.x) s_hist[b] = 0u;
+        if (threadIdx.x == 0) { s_bin = 0u; s_before = 0u; }
+        __syncthreads();
+        for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
+            const uint32_t key = job.cand[c].x;
+            if ((key >> (shift + bits)) == prefix) atomicAdd(&s_hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+        }
+        __syncthreads();
+        // thread t owns bins 2t and 2t + 1; the rank looked for is k - 1 - below
+        const uint32_t r = (uint32_t)(job.k - 1) - below;
+        const uint32_t v0 = s_hist[2 * threadIdx.x], v1 = s_hist[2 * threadIdx.x + 1];
+        unsigned long long total;
+        const uint32_t before = (uint32_t)block_exclusive_scan((unsigned long long)(v0 + v1), scratch, &total);
+        if (r >= before && r < before + v0 + v1) {     // exactly one thread
+            const bool second = r >= before + v0;
+            s_bin = 2 * threadIdx.x + (second ? 1u : 0u);
+            s_before = before + (second ? v0 : 0u);
+        }
+        __syncthreads();
+        prefix = (prefix << bits) | s_bin;
+        below += s_before;
+        fixed += bits;
+        __syncthreads();
+    }
+    const uint32_t tau = prefix;
+    if (threadIdx.x == 0) {
+        sel->tau = tau;
+        sel->below = below;
+        sel->rem = (uint32_t)job.k - below;            // ties to keep, >= 1
+    }
+    // the candidates' share of the chunk counts: low word keys below tau, high word keys equal to it
+    for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
+        const uint2 kc = job.cand[c];
+        if (kc.x < tau) atomicAdd(&job.chunks[kc.y >> 10], 1ull);
+        else if (kc.x == tau) atomicAdd(&job.chunks[kc.y >> 10], 1ull << 32);
     }
 }
 

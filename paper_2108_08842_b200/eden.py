@@ -76,7 +76,7 @@ _sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
 _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(_u64),
                                 ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
 
-STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA, STATUS_TIMEOUT = 1, 2, 4, 8
+STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA, STATUS_TIMEOUT, STATUS_SCRATCH = 1, 2, 4, 8, 16
 PACKET_COORDS = 1024
 UNIFORM_MAX_INDEX = 127
 UNIFORM_MIN_DELTA = 0.0625

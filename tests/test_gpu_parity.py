@@ -221,6 +221,18 @@ def test_sub_bit_budgets_and_mask(E, bits, d):
     run_workload(E, work)
 
 
+@pytest.mark.parametrize("bits,d", [(0.1, 200003), (0.5, 70001), (0.9, 9)])
+def test_sub_bit_selection_in_three_histogram_rounds(E, bits, d, monkeypatch):
+    # vectors too long for the candidate list of the two-pass selection find the mask's
+    # threshold in three histogram rounds over all keys; forced here at sizes the oracle sorts quickly
+    monkeypatch.setenv("EDEN_SEL_ROUNDS", "3")
+    n = 3
+    rng = np.random.default_rng(d)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(d + 2, n), 0.0, lambda c: xs[c], d)
+    run_workload(E, work)
+
+
 @pytest.mark.parametrize("bits,d", [(1.5, 100), (1.5, 40000), (2.25, 5000), (7.5, 3000), (3.75, 300000)])
 def test_non_integer_budgets(E, bits, d):
     # Section 4.1: a shared coin per coordinate picks 2^floor(b) or 2^(floor(b)+1) values
