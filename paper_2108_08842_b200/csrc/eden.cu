@@ -144,7 +144,8 @@ extern "C" uint64_t eden_workspace_bytes(uint64_t d_max, uint32_t n_batch)
     const uint64_t D = 1ull << ceil_log2(d_max ? d_max : 1);
     // per client: descriptors, one intermediate vector, and (b < 1) the mask-selection scratch
     const uint64_t n_chunks = (d_max + kSelChunk - 1) / kSelChunk;
-    const uint64_t sel = 256 + kHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) + 256;
+    const uint64_t sel = 256 + kHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) + 256 +
+                         align_up(n_chunks * (kSelChunk / 8), 256);   // the last term: mask bitmap
     // partial sums of the receiver's last pass when a round has too few tiles to fill the
     // GPU (sized for 148 SMs; a split that does not fit is simply not used)
     const uint64_t tiles = std::max<uint64_t>(1, D >> 13);
@@ -513,11 +514,17 @@ bool two_pass_selection(uint64_t d)
     return mean + 12.0 * std::sqrt(mean) + 64.0 <= (double)kSelCandCap;
 }
 
+// mask bitmap of one job: 32 words per chunk of 1024 coordinates
+uint64_t keep_bitmap_bytes(uint64_t d)
+{
+    return align_up((d + kSelChunk - 1) / kSelChunk * (kSelChunk / 8), 256);
+}
+
 uint64_t sel_scratch_bytes(uint64_t d)
 {
     const uint64_t n_chunks = (d + kSelChunk - 1) / kSelChunk;
     return 256 + kBatchHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) +
-           align_up(sizeof(SelJob), 256) + (two_pass_selection(d) ? kCandBytes : 0);
+           align_up(sizeof(SelJob), 256) + (two_pass_selection(d) ? kCandBytes + keep_bitmap_bytes(d) : 0);
 }
 
 // Groups: clients of one rotation dimension (and, within it, of one kind: b >= 1 or
@@ -902,6 +909,7 @@ struct SelBatch {
     SelJob* d_jobs;
     uint32_t n;
     unsigned grid;       // blocks of 1024 coordinates
+    bool two_pass;       // the jobs carry mask bitmaps (k_selc_compact / k_selc_scatter)
 };
 
 int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::vector<SelJob>& partial,
@@ -922,7 +930,9 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
         jobs[j].hist = (uint32_t*)(hist_base + kBatchHistBytes * j);
         jobs[j].chunks = (unsigned long long*)(chunk_base + chunk_bytes * j);
         jobs[j].cand = two_pass ? (uint2*)(cand_base + kCandBytes * j) : nullptr;
+        jobs[j].keep = two_pass ? (uint32_t*)(cand_base + kCandBytes * n + keep_bitmap_bytes(d) * j) : nullptr;
     }
+    batch.two_pass = two_pass;
     batch.d_jobs = (SelJob*)job_base;
     batch.n = n;
     batch.grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
@@ -1102,8 +1112,12 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
             SelBatch batch;
             rc = start_selection_batch(ctx, ctx->ws + lay.work_off + work_end, d, jobs, batch);
             if (rc) return rc;
-            LAUNCH(ctx, "sel_compact", 4.0 * gn * (double)d + 4.0 * (double)kept, k_selb_compact,
-                   dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
+            if (batch.two_pass)
+                LAUNCH(ctx, "sel_compact", 4.0 * gn * (double)d + 4.0 * (double)kept, k_selc_compact,
+                       dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
+            else
+                LAUNCH(ctx, "sel_compact", 4.0 * gn * (double)d + 4.0 * (double)kept, k_selb_compact,
+                       dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
         }
         if (fast_eligible(ctx, g) && (x_aligned || g.subbit)) {
             rc = fast_encode_group(ctx, plan, g, descs.data() + first, d_descs + first, d_states + first, d, d_status);
@@ -1304,8 +1318,12 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             }
         }
         if (g.subbit) {
-            LAUNCH(ctx, "sel_scatter", 8.0 * (double)kept + 4.0 * (double)kept, k_selb_scatter, batch.grid,
-                   kSelThreads, 0, (const SelJob*)batch.d_jobs, gn, d, out);
+            if (batch.two_pass)
+                LAUNCH(ctx, "sel_scatter", 8.0 * (double)kept + 4.0 * (double)kept, k_selc_scatter, batch.grid,
+                       kSelThreads, 0, (const SelJob*)batch.d_jobs, gn, d, out);
+            else
+                LAUNCH(ctx, "sel_scatter", 8.0 * (double)kept + 4.0 * (double)kept, k_selb_scatter, batch.grid,
+                       kSelThreads, 0, (const SelJob*)batch.d_jobs, gn, d, out);
         } else {
             written = true;
         }

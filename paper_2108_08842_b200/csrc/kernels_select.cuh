@@ -215,6 +215,7 @@ struct SelJob {
     const float* in;                 // compact: the client's input row; scatter: its estimate of the kept coordinates
     float* out;                      // compact: the compacted vector
     uint2* cand;                     // two-pass selection: (key, coordinate) of the keys that share tau's first digit
+    uint32_t* keep;                  // two-pass selection: the mask as a bitmap (bit i % 32 of word i / 32)
 };
 
 // Batched selection finds the k-th smallest key in three digit rounds of 10, 11 and 11
@@ -370,10 +371,12 @@ k_selb_chunk_scan(const SelJob* __restrict__ jobs, uint64_t n_chunks)
 // pass over the keys does two things at once: it counts, per chunk of 1024 coordinates, the
 // keys whose first digit is smaller (they are below tau whatever its other bits are), and it
 // appends the keys that share the digit, about one in 2048, to the job's candidate list with
-// their coordinates.  One block per job then finds tau's remaining 21 bits among the
-// candidates alone and adds each candidate below (or equal to) tau to its chunk's count.
-// The keys are generated three times per side (histogram, this pass, compaction or scatter)
-// instead of five.  job.hist[kSelBins] counts the candidates (zeroed with the histograms).
+// their coordinates; the coordinates of the first kind are also marked in the job's mask
+// bitmap.  One block per job then finds tau's remaining 21 bits among the candidates alone
+// and, for each candidate that is kept (below tau, or equal to it and among the first `rem`
+// such coordinates), sets its bit and adds it to its chunk's count.  Compaction and scatter
+// read the bitmap, so the keys are generated twice per side (histogram, this pass) instead
+// of five times.  job.hist[kSelBins] counts the candidates (zeroed with the histograms).
 // ---------------------------------------------------------------------------------
 constexpr int kSelFirstShift = 21;                     // first digit = key >> 21 (11 bits, kSelBins bins)
 constexpr uint32_t kSelCandCap = 61440;                // candidates a job can hold (480 KB)
@@ -413,6 +416,7 @@ k_selc_collect(const SelJob* __restrict__ jobs)
     const uint4 k4 = mask_keys(job.seed, t);
     const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
     unsigned long long mine = 0;
+    uint32_t nibble = 0u;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const uint64_t i = t * 4 + j;
@@ -420,11 +424,18 @@ k_selc_collect(const SelJob* __restrict__ jobs)
         const uint32_t top = keys[j] >> kSelFirstShift;
         if (top < digit) {
             ++mine;
+            nibble |= 1u << j;
         } else if (top == digit) {
             const uint32_t slot = atomicAdd(&job.hist[kSelBins], 1u);
             if (slot < kSelCandCap) job.cand[slot] = make_uint2(keys[j], (uint32_t)i);
         }
     }
+    // eight threads hold the 32 coordinates of one bitmap word
+    uint32_t word = nibble << (4 * (threadIdx.x & 7));
+    word |= __shfl_xor_sync(0xffffffffu, word, 1);
+    word |= __shfl_xor_sync(0xffffffffu, word, 2);
+    word |= __shfl_xor_sync(0xffffffffu, word, 4);
+    if ((threadIdx.x & 7) == 0) job.keep[t >> 3] = word;
     unsigned long long total;
     block_exclusive_scan(mine, scratch, &total);
     if (threadIdx.x == 0) job.chunks[blockIdx.x] = total;
@@ -480,11 +491,95 @@ k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status)
         sel->below = below;
         sel->rem = (uint32_t)job.k - below;            // ties to keep, >= 1
     }
-    // the candidates' share of the chunk counts: low word keys below tau, high word keys equal to it
+    // the candidates that are kept: below tau, or equal to it with fewer than `rem` equal
+    // keys at smaller coordinates.  Equal keys are rare, so their coordinates are gathered
+    // in shared memory and ranked there; a list that does not fit is ranked in place.
+    constexpr uint32_t kTieCap = 256;
+    __shared__ uint32_t s_ties[kTieCap];
+    __shared__ uint32_t s_nties;
+    const uint32_t rem = (uint32_t)job.k - below;
+    if (threadIdx.x == 0) s_nties = 0u;
+    __syncthreads();
     for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
         const uint2 kc = job.cand[c];
-        if (kc.x < tau) atomicAdd(&job.chunks[kc.y >> 10], 1ull);
-        else if (kc.x == tau) atomicAdd(&job.chunks[kc.y >> 10], 1ull << 32);
+        if (kc.x < tau) {
+            atomicOr(&job.keep[kc.y >> 5], 1u << (kc.y & 31u));
+            atomicAdd(&job.chunks[kc.y >> 10], 1ull);
+        } else if (kc.x == tau) {
+            const uint32_t slot = atomicAdd(&s_nties, 1u);
+            if (slot < kTieCap) s_ties[slot] = kc.y;
+        }
+    }
+    __syncthreads();
+    const uint32_t n_ties = s_nties;
+    if (n_ties <= kTieCap) {
+        for (uint32_t i = threadIdx.x; i < n_ties; i += blockDim.x) {
+            const uint32_t coord = s_ties[i];
+            uint32_t before = 0;
+            for (uint32_t o = 0; o < n_ties; ++o) before += s_ties[o] < coord ? 1u : 0u;
+            if (before < rem) {
+                atomicOr(&job.keep[coord >> 5], 1u << (coord & 31u));
+                atomicAdd(&job.chunks[coord >> 10], 1ull);
+            }
+        }
+    } else {
+        for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
+            const uint2 kc = job.cand[c];
+            if (kc.x != tau) continue;
+            uint32_t before = 0;
+            for (uint32_t o = 0; o < n; ++o) {
+                const uint2 ko = job.cand[o];
+                before += (ko.x == tau && ko.y < kc.y) ? 1u : 0u;
+            }
+            if (before < rem) {
+                atomicOr(&job.keep[kc.y >> 5], 1u << (kc.y & 31u));
+                atomicAdd(&job.chunks[kc.y >> 10], 1ull);
+            }
+        }
+    }
+}
+
+// the four mask bits of the thread's coordinates 4t .. 4t + 3
+__device__ __forceinline__ uint32_t keep_nibble(const uint32_t* __restrict__ keep, uint64_t t)
+{
+    return (keep[t >> 3] >> (4 * ((uint32_t)t & 7u))) & 0xFu;
+}
+
+// Sender: y_c[pos] = x_c[i] for the kept coordinates of every job, from the bitmap.
+__global__ void __launch_bounds__(kSelThreads)
+k_selc_compact(const SelJob* __restrict__ jobs)
+{
+    __shared__ unsigned long long scratch[33];
+    const SelJob job = jobs[blockIdx.y];
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t nib = keep_nibble(job.keep, t);
+    unsigned long long total;
+    uint64_t pos = block_exclusive_scan((unsigned long long)__popc(nib), scratch, &total) + job.chunks[blockIdx.x];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        if ((nib >> j) & 1u) job.out[pos++] = job.in[t * 4 + j];
+}
+
+// Receiver: out[i] += sum over the jobs of yhat_c[pos_c(i)] for the coordinates job c kept.
+__global__ void __launch_bounds__(kSelThreads)
+k_selc_scatter(const SelJob* __restrict__ jobs, uint32_t n_jobs, uint64_t d, float* __restrict__ out)
+{
+    __shared__ unsigned long long scratch[33];
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    float add[4] = {0.f, 0.f, 0.f, 0.f};
+    for (uint32_t c = 0; c < n_jobs; ++c) {
+        const SelJob job = jobs[c];
+        const uint32_t nib = keep_nibble(job.keep, t);
+        unsigned long long total;
+        uint64_t pos = block_exclusive_scan((unsigned long long)__popc(nib), scratch, &total) + job.chunks[blockIdx.x];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if ((nib >> j) & 1u) add[j] += job.in[pos++];
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint64_t i = t * 4 + j;
+        if (i < d && add[j] != 0.f) out[i] += add[j];
     }
 }
 
