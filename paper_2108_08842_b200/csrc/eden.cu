@@ -947,8 +947,7 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
         LAUNCH(ctx, "sel_find", n * (double)kSelBins * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, 0);
         LAUNCH(ctx, "sel_collect", keys / 128.0, k_selc_collect, dim3(batch.grid, n), kSelThreads, 0,
                (const SelJob*)batch.d_jobs);
-        LAUNCH(ctx, "sel_resolve", keys / 256.0, k_selc_resolve, n, 1024, 0, (const SelJob*)batch.d_jobs, d_status);
-        LAUNCH(ctx, "sel_chunk_scan", keys / 64.0, k_selb_chunk_scan, n, 1024, 0, (const SelJob*)batch.d_jobs,
+        LAUNCH(ctx, "sel_resolve", keys / 64.0, k_selc_resolve, n, 1024, 0, (const SelJob*)batch.d_jobs, d_status,
                (uint64_t)batch.grid);
         return EDEN_OK;
     }

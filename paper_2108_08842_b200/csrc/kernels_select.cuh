@@ -441,9 +441,10 @@ k_selc_collect(const SelJob* __restrict__ jobs)
     if (threadIdx.x == 0) job.chunks[blockIdx.x] = total;
 }
 
-// One block of 1024 threads per job.
+// One block of 1024 threads per job; ends with the exclusive scan of the job's chunk counts
+// (the positions compaction and scatter start from).
 __global__ void __launch_bounds__(1024)
-k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status)
+k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status, uint64_t n_chunks)
 {
     __shared__ uint32_t s_hist[kSelBins];
     __shared__ unsigned long long scratch[33];
@@ -537,41 +538,76 @@ k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status)
             }
         }
     }
+    // every count is final: scan them in place (reads from L2, where the atomics landed)
+    __syncthreads();
+    const uint64_t per = (n_chunks + blockDim.x - 1) / blockDim.x;
+    const uint64_t lo = min((uint64_t)threadIdx.x * per, n_chunks), hi = min(lo + per, n_chunks);
+    unsigned long long mine = 0;
+    for (uint64_t j = lo; j < hi; ++j) mine += __ldcg(&job.chunks[j]);
+    unsigned long long total;
+    unsigned long long run = block_exclusive_scan(mine, scratch, &total);
+    for (uint64_t j = lo; j < hi; ++j) {
+        const unsigned long long v = __ldcg(&job.chunks[j]);
+        job.chunks[j] = run;
+        run += v;
+    }
 }
 
-// the four mask bits of the thread's coordinates 4t .. 4t + 3
-__device__ __forceinline__ uint32_t keep_nibble(const uint32_t* __restrict__ keep, uint64_t t)
+// Position, among the kept coordinates of the block's chunk of 1024, of the first kept
+// coordinate of thread t's four (coordinates 4t .. 4t + 3), and the thread's four mask bits.
+// Every warp reads the chunk's 32 bitmap words (lane l word l), scans their population
+// counts with shuffles and hands each thread the count before its word; the bits below the
+// thread's nibble inside the word complete it.  No shared memory, no block barrier.
+__device__ __forceinline__ uint32_t keep_position(const uint32_t* __restrict__ keep, uint32_t& nibble)
 {
-    return (keep[t >> 3] >> (4 * ((uint32_t)t & 7u))) & 0xFu;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t word = keep[(uint64_t)blockIdx.x * 32u + lane];
+    uint32_t inc = (uint32_t)__popc(word);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= (uint32_t)o) inc += v;
+    }
+    const uint32_t w = threadIdx.x >> 3;                          // the thread's word in the chunk
+    const uint32_t mine = __shfl_sync(0xffffffffu, word, w);
+    const uint32_t before = __shfl_sync(0xffffffffu, inc, w) - (uint32_t)__popc(mine);
+    const uint32_t shift = 4u * (threadIdx.x & 7u);
+    nibble = (mine >> shift) & 0xFu;
+    return before + (uint32_t)__popc(mine & ((1u << shift) - 1u));
 }
 
 // Sender: y_c[pos] = x_c[i] for the kept coordinates of every job, from the bitmap.
 __global__ void __launch_bounds__(kSelThreads)
 k_selc_compact(const SelJob* __restrict__ jobs)
 {
-    __shared__ unsigned long long scratch[33];
     const SelJob job = jobs[blockIdx.y];
     const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t nib = keep_nibble(job.keep, t);
-    unsigned long long total;
-    uint64_t pos = block_exclusive_scan((unsigned long long)__popc(nib), scratch, &total) + job.chunks[blockIdx.x];
+    uint32_t nib;
+    uint64_t pos = keep_position(job.keep, nib) + job.chunks[blockIdx.x];
+    if (((uintptr_t)job.in & 15u) == 0 && t * 4 + 3 < job.d) {
+        // one coalesced 16-byte load per thread, whatever the mask keeps
+        const float4 x4 = *reinterpret_cast<const float4*>(job.in + t * 4);
+        const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-        if ((nib >> j) & 1u) job.out[pos++] = job.in[t * 4 + j];
+        for (int j = 0; j < 4; ++j)
+            if ((nib >> j) & 1u) job.out[pos++] = xs[j];
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if ((nib >> j) & 1u) job.out[pos++] = job.in[t * 4 + j];
+    }
 }
 
 // Receiver: out[i] += sum over the jobs of yhat_c[pos_c(i)] for the coordinates job c kept.
 __global__ void __launch_bounds__(kSelThreads)
 k_selc_scatter(const SelJob* __restrict__ jobs, uint32_t n_jobs, uint64_t d, float* __restrict__ out)
 {
-    __shared__ unsigned long long scratch[33];
     const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     float add[4] = {0.f, 0.f, 0.f, 0.f};
     for (uint32_t c = 0; c < n_jobs; ++c) {
         const SelJob job = jobs[c];
-        const uint32_t nib = keep_nibble(job.keep, t);
-        unsigned long long total;
-        uint64_t pos = block_exclusive_scan((unsigned long long)__popc(nib), scratch, &total) + job.chunks[blockIdx.x];
+        uint32_t nib;
+        uint64_t pos = keep_position(job.keep, nib) + job.chunks[blockIdx.x];
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             if ((nib >> j) & 1u) add[j] += job.in[pos++];
