@@ -233,6 +233,38 @@ def test_sub_bit_selection_in_three_histogram_rounds(E, bits, d, monkeypatch):
     run_workload(E, work)
 
 
+@pytest.mark.parametrize("rounds", [2, 3])
+@pytest.mark.parametrize("which,extra", [(0, 1), (1, 2), (2, 1)])
+def test_mask_threshold_on_a_pair_of_equal_keys(E, which, extra, rounds, monkeypatch):
+    # Section 4.1 asks for a sample of exactly d*p coordinates.  With seed 1 and d = 2^17 three
+    # pairs of coordinates draw the same 32-bit key; putting the k-th smallest key on such a
+    # pair makes the selection decide by coordinate: extra = 1 keeps only the pair's first
+    # coordinate, extra = 2 keeps both.  Both forms of the batched selection and the
+    # single-mask entry point must agree with the oracle's full sort.
+    if rounds == 3:
+        monkeypatch.setenv("EDEN_SEL_ROUNDS", "3")
+    d, seed = 1 << 17, 1
+    keys = np.array([O.mask_key(seed, i) for i in range(d)], dtype=np.uint64)
+    sk = keys[np.lexsort((np.arange(d), keys))]
+    pairs = np.nonzero(sk[1:] == sk[:-1])[0]
+    assert pairs.size >= 3
+    k = int(pairs[which]) + extra
+    bits = k / d
+    assert 0 < bits < 1 and O.kept_count(d, bits) == k
+    want = O.mask(seed, d, k)
+    assert want.sum() == k
+    ctx = _ctx(E, d, 2)
+    got = ctx.sparsification_mask(seed, d, bits).cpu().numpy().view(np.uint32)
+    bits_got = ((got[:, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(-1)[:d]
+    assert np.array_equal(bits_got.astype(np.uint8), want)
+    ctx.close()
+    rng = np.random.default_rng(k)
+    xs = rng.standard_normal((2, d)).astype(np.float32)
+    work = synth.Workload("adhoc", 2, d, np.full(2, bits), np.array([seed, seed + 1], dtype=np.uint64), 0.0,
+                          lambda c: xs[c], k)
+    run_workload(E, work)
+
+
 @pytest.mark.parametrize("bits,d", [(1.5, 100), (1.5, 40000), (2.25, 5000), (7.5, 3000), (3.75, 300000)])
 def test_non_integer_budgets(E, bits, d):
     # Section 4.1: a shared coin per coordinate picks 2^floor(b) or 2^(floor(b)+1) values
