@@ -289,6 +289,25 @@ def test_mask_exact_size_and_order_rule():
     assert O.kept_count(3, 0.01) == 1 and O.kept_count(10, 1.0) == 10 and O.kept_count(10, 4.0) == 10
 
 
+def test_mask_breaks_equal_keys_by_coordinate():
+    # seed 1 draws the same 32-bit key for three pairs of the first 2^17 coordinates; with the
+    # k-th smallest key on such a pair the smaller coordinate goes first (k = r + 1 keeps only it)
+    seed, d = 1, 1 << 17
+    keys = np.array([O.mask_key(seed, i) for i in range(d)], dtype=np.uint64)
+    order = np.lexsort((np.arange(d), keys))
+    pairs = np.nonzero(keys[order][1:] == keys[order][:-1])[0]
+    assert pairs.size >= 3
+    for r in pairs[:3]:
+        lo, hi = int(order[r]), int(order[r + 1])
+        assert keys[lo] == keys[hi] and lo < hi
+        for k in (int(r) + 1, int(r) + 2):
+            m = O.mask(seed, d, k)
+            expect = np.zeros(d, dtype=np.uint8)
+            expect[order[:k]] = 1
+            assert m.sum() == k and np.array_equal(m, expect)
+            assert m[lo] == 1 and m[hi] == (1 if k == int(r) + 2 else 0)
+
+
 def test_mask_inclusion_frequency_is_uniform():
     d, k, trials = 200, 60, 3000
     counts = np.zeros(d)
