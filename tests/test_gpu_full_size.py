@@ -112,6 +112,20 @@ def test_largest_tested_dimension_2_pow_28(E):
     assert mism <= 120
 
 
+def test_sub_bit_budgets_at_10_pow_8_coordinates(E):
+    # the longest vectors the two-pass mask selection takes (its candidate list then holds
+    # about 49 000 of its 61 440 keys): b = 0.5 rotates 5*10^7 kept coordinates padded to 2^26,
+    # b = 0.1 rotates 10^7 padded to 2^24; the oracle sorts all 10^8 keys of each client
+    d = 100_000_000
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal(d, dtype=np.float32)
+    x[::8191] *= 20.0
+    work = synth.Workload("adhoc", 2, d, np.array([0.5, 0.1]), synth.client_seeds(88, 2), 0.0,
+                          lambda c: x if c == 0 else -x, 88)
+    mism, _, _ = run_workload(E, work, threads=2)
+    assert mism <= 60
+
+
 def test_uniform_family_at_cfg4_size_with_packet_loss(E):
     # Section 4.3's quantiser at configuration 4's dimension and loss rate (eight clients
     # keep the oracle to about a minute): every index byte, scale and the mean
