@@ -1,7 +1,7 @@
 // Register-blocked transform kernels for rotation dimensions of 2^14 and more.
 //
 // Every kernel works on a tile of 8192 floats with 256 threads, 32 values per thread,
-// four resident blocks per SM.  Butterflies run in registers as packed fp32 pairs
+// two to five resident blocks per SM (set per kernel).  Butterflies run in registers as packed fp32 pairs
 // (add.rn.f32x2 / sub.rn.f32x2: one instruction per two coordinates); between register
 // steps the tile is transposed through shared memory with 64- or 128-bit conflict-free
 // accesses; global loads and stores are 64- or 128-bit and fully coalesced.

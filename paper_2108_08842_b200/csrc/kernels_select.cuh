@@ -3,11 +3,13 @@
 // folded into the scale S) and its inverse on the receiver (scatter into the sum).
 //
 // The mask keeps the k coordinates with the smallest (key, index) pairs, key_i being the
-// 32-bit Philox stream-1 word of coordinate i.  The k-th smallest pair is found exactly
-// with two 16-bit histogram rounds; a coordinate is then kept iff key < tau, or key ==
-// tau and fewer than `rem` equal keys precede it.  Positions in the compacted vector are
-// exclusive prefix counts: per 1024-coordinate chunk counts, a scan of the chunk counts,
-// and a block scan inside each chunk.
+// 32-bit Philox stream-1 word of coordinate i.  The k-th smallest pair is found exactly:
+// a coordinate is kept iff key < tau, or key == tau and fewer than `rem` equal keys
+// precede it.  Positions in the compacted vector are exclusive prefix counts: per
+// 1024-coordinate chunk counts, a scan of the chunk counts, and a scan inside each chunk.
+// Three forms: single-job kernels with two 16-bit histogram rounds (the mask entry points),
+// batched kernels with three digit rounds over all keys (long vectors), and the batched
+// two-pass form with a candidate list and a mask bitmap (the default).
 #pragma once
 #include "eden_device.cuh"
 
