@@ -818,8 +818,8 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
 template <int W, int LC, bool FRAC, bool UNI = false>
 // Five resident blocks per SM for integer budgets (51 registers; at most a few words
 // spilled): cfg5's shape 3240 -> 3370 GB/s, cfg4's 5000 -> 5090 GB/s.  Six fit as well but
-// run slower (2940 / 4310 GB/s): 230 KB of shared memory leave the SM almost no L1 to land
-// the tiles' loads in.  The non-integer budgets keep four (their coins cost registers).
+// run slower (2940 / 4310 GB/s, with or without L1 allocation of the tile loads).  The
+// non-integer budgets keep four (their coins cost registers).
 __global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : 5))
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L)
 {
