@@ -772,13 +772,14 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
             EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
                 LAUNCH_CL(ctx, "f_enc_first", gn * (4.0 * std::min<double>((double)d, D) + 4.0 * D),
                           (k_f_col<LR_, LC_, true>), dim3(tiles, gn), dim3(kFastThreads), ps.lc,
-                          (const ClientDesc*)d_descs, d_states, ps.lo)));
+                          (const ClientDesc*)d_descs, d_states, ps.lo, 0)));
         } else {
             EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
                 LAUNCH_CL(ctx, "f_mid", gn * 8.0 * D, (k_f_col<LR_, LC_, false>), dim3(tiles, gn),
-                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo)));
+                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo, 1)));
         }
     }
+    const int inv_ready = pl.cols.size() >= 2 ? 1 : 0;     // a middle pass has left 1/||y|| in the client's state
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
     for (const WidthRun& r : runs) {
@@ -788,7 +789,7 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
         if (g.uniform) {
             LAUNCH(ctx, "f_enc_last", r.count * 5.0 * D, (k_f_enc_last<8, 0, false, true>), dim3(tiles, r.count),
                    kFastThreads, 0, (const ClientDesc*)(d_descs + r.first), d_states + r.first,
-                   (const float*)h_descs[r.first].work, g.L);
+                   (const float*)h_descs[r.first].work, g.L, inv_ready);
             continue;
         }
         if (ctx->row_staging && pl.row_lc == 0) {
@@ -808,7 +809,7 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
             LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_, FRAC_>),
                       dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
                       (const ClientDesc*)(d_descs + r.first), d_states + r.first,
-                      (const float*)h_descs[r.first].work, g.L))));
+                      (const float*)h_descs[r.first].work, g.L, inv_ready))));
     }
     return EDEN_OK;
 }
@@ -837,7 +838,7 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
         if (pi > 0) {
             EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
                 LAUNCH_CL(ctx, "f_mid", gn * 8.0 * D, (k_f_col<LR_, LC_, false>), dim3(tiles, gn),
-                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo)));
+                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo, 0)));
         } else {
             // A round with few tiles leaves most SMs idle if every block walks all clients:
             // split the clients over block rows, each row summing into a partial vector of

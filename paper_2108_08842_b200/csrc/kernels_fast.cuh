@@ -311,7 +311,7 @@ __device__ __forceinline__ void col_cluster_stage(u64 (&v)[16], ulonglong2* s, c
 // =================================================================================
 template <int LR, int LC, bool FIRST>
 __global__ void __launch_bounds__(kFastThreads, 4)
-k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo)
+k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo, int publish_inv)
 {
     __shared__ ulonglong2 s[2048];
     __shared__ uint32_t s_sign[256];
@@ -336,6 +336,12 @@ k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, 
             v[2 * k] = pack2(x0, x1);
             v[2 * k + 1] = pack2(x2, 0.f);
         }
+    }
+    if (!FIRST && publish_inv && blockIdx.x == 0 && t == 0) {
+        // sender's middle pass: ||y||^2 is complete, so one thread per client leaves 1/||y||
+        // (0 for a zero or non-finite vector) for the row pass, off every block's critical path
+        const double n2 = states[blockIdx.y].norm2;
+        states[blockIdx.y].factor = (n2 > 0.0 && n2 < INFINITY) ? (float)(1.0 / sqrt(n2)) : 0.f;
     }
     u64 acc = 0ull;
     if (FIRST) {
@@ -785,18 +791,35 @@ __device__ __forceinline__ void store_words(uint32_t* dst, const uint32_t (&word
 // The 13 stages of one tile held in arrangement A, then quantise, pack and store the tile's
 // code words; returns the thread's part of sum |h| Q(|z|).
 template <int W, bool FRAC, bool UNI = false>
-__device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& cd, double n2, uint64_t base,
-                                               u64* s, const EncTables<W, FRAC>& tab)
+// `norm2` points at the client's sum of squares; thread 0 turns it into 1/||y|| (0 for a
+// zero or non-finite vector) in `s_inv`, which the block barrier of the first exchange
+// publishes: one double-precision square root and division per tile instead of one per
+// thread.  Where a middle pass ran before, it has left the value in `inv_ready` and the
+// thread only copies it (the square root's latency would hold up that barrier).
+// The caller makes sure that no thread still reads `s_inv` from an earlier tile.
+__device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& cd, const double* norm2, uint64_t base,
+                                               u64* s, const EncTables<W, FRAC>& tab, float* s_inv,
+                                               const float* inv_ready = nullptr)
 {
     const int t = threadIdx.x;
+    if (t == 0) {
+        if (W > 1 && inv_ready) {
+            *s_inv = *inv_ready;
+        } else {
+            const double n2 = *norm2;
+            const bool ok = n2 > 0.0 && n2 < INFINITY;
+            if (W == 1) *s_inv = ok ? 1.f : 0.f;       // one-bit codes are the signs of h: only "live" matters
+            else *s_inv = ok ? (float)(1.0 / sqrt(n2)) : 0.f;
+        }
+    }
     row_step<0>(v);                 // e bits 12..9
     row_exchange<0, 1>(v, s);
     row_step<0>(v);                 // e bits 8..5
     row_exchange<1, 2>(v, s);
     row_step<0>(v);                 // e bits 4..1
     row_step_inner(v);              // e bit 0
-    const bool live = n2 > 0.0 && n2 < INFINITY;
-    const float inv_norm = live ? (float)(1.0 / sqrt(n2)) : 0.f;
+    const float inv_norm = *s_inv;
+    const bool live = inv_norm > 0.f;
     uint32_t words[W];
     float dot = 0.f;
     if constexpr (UNI) {
@@ -821,10 +844,12 @@ template <int W, int LC, bool FRAC, bool UNI = false>
 // run slower (2940 / 4310 GB/s, with or without L1 allocation of the tile loads).  The
 // non-integer budgets keep four (their coins cost registers).
 __global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : 5))
-k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L)
+k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L,
+             int inv_ready)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ double red[32];
+    __shared__ float s_inv;
     __shared__ EncTables<W, FRAC> tab;
     const int t = threadIdx.x;
     const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
@@ -861,7 +886,8 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
         for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<0>(t, k))];
         __syncthreads();                               // s is rewritten by the next exchange
     }
-    const float dot = enc_last_tile<W, FRAC, UNI>(v, cd, states[blockIdx.y].norm2, base, s, tab);
+    const float dot = enc_last_tile<W, FRAC, UNI>(v, cd, &states[blockIdx.y].norm2, base, s, tab, &s_inv,
+                                                  inv_ready ? &states[blockIdx.y].factor : nullptr);
     const double tot = block_sum((double)dot, red);
     if (t == 0) atomicAdd(&states[blockIdx.y].dot, tot);
 }
@@ -919,6 +945,7 @@ k_f_enc_last_staged(const ClientDesc* __restrict__ descs, ClientState* __restric
     __shared__ __align__(8) uint64_t bar;
     __shared__ double red[32];
     __shared__ int s_fail;
+    __shared__ float s_inv;
     __shared__ EncTables<W, FRAC> tab;
     const int t = threadIdx.x;
     constexpr uint32_t kTileBytes = 4u << kFastTileLog;
@@ -960,7 +987,7 @@ k_f_enc_last_staged(const ClientDesc* __restrict__ descs, ClientState* __restric
         }
         const ClientDesc cd = descs[client];
         const uint64_t base = (uint64_t)(g & ((1u << tiles_log) - 1u)) << kFastTileLog;
-        acc += (double)enc_last_tile<W, FRAC>(v, cd, states[client].norm2, base, s, tab);
+        acc += (double)enc_last_tile<W, FRAC>(v, cd, &states[client].norm2, base, s, tab, &s_inv);
         // the barrier after the next tile's staging read orders this tile's last exchange
         // reads before the next tile's first exchange writes
     }
