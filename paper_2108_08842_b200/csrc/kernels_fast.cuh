@@ -608,11 +608,37 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
         }
         dot = sum * c_pos_value[0];
         words[0] = live ? ~negs : 0u;
+    } else if constexpr (32 % W == 0) {
+        // Widths that divide 32: a word holds 32 / W whole fields.  The fields collect the
+        // magnitude indices (coordinates in descending order: shift the word up one field, drop
+        // the index into the low bits); the top bit of every field (the code of a non-negative
+        // coordinate is half + m) and the sign flips (a negative one has all W bits inverted)
+        // are applied to the whole word at the end, the signs having been gathered by funnel shifts.
+        constexpr int per = 32 / W;
+        constexpr uint32_t lsb = W == 2 ? 0x55555555u : W == 4 ? 0x11111111u : 0x01010101u;
+        static_assert(W == 2 || W == 4 || W == 8, "field widths that divide 32");
+#pragma unroll
+        for (int j = W - 1; j >= 0; --j) {
+            uint32_t fields = 0u, signs = 0u;
+#pragma unroll
+            for (int i = per - 1; i >= 0; --i) {
+                const int l = j * per + i;
+                float h0, h1;
+                unpack2(v[l >> 1], h0, h1);
+                const float h = (l & 1) ? h1 : h0;
+                const float z = h * inv_norm;
+                const int m = fast_magnitude<W>(fabsf(z), s_tb);
+                dot = fmaf(fabsf(h), W <= 2 ? (m ? c_pos_value[half] : c_pos_value[half - 1]) : s_tv[m], dot);
+                fields = (fields << W) | (uint32_t)m;
+                signs = __funnelshift_l(__float_as_uint(z), signs, W);
+            }
+            const uint32_t neg = (signs >> (W - 1)) & lsb;           // bit 0 of every field whose z is negative
+            words[j] = live ? (fields | (lsb << (W - 1))) ^ ((neg << W) - neg) : 0u;
+        }
     } else {
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = 0u;
-    // coordinates in descending order, so that widths that divide 32 can shift the word up
-    // by one field and drop the code into the low bits
+    // coordinates in descending order
 #pragma unroll
     for (int k = 15; k >= 0; --k) {
         float h[2];
@@ -628,12 +654,8 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
             const uint32_t flip = (uint32_t)((int)__float_as_uint(z) >> 31) & (2u * half - 1u);
             const uint32_t code = ((uint32_t)m | half) ^ flip;
             const int a = (l * W) >> 5, off = (l * W) & 31;
-            if constexpr (32 % W == 0) {
-                words[a] = (words[a] << W) | code;
-            } else {
-                words[a] |= code << off;
-                if (off + W > 32) words[a + 1] |= code >> (32 - off);
-            }
+            words[a] |= code << off;
+            if (off + W > 32) words[a + 1] |= code >> (32 - off);
         }
     }
     if (!live) {
