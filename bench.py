@@ -35,7 +35,7 @@ FALLBACK_HBM_GBS = 6650.0
 # profiles/ncu_full_fast_kernels_cfg5_n1.md (one client of 2^27 coordinates per launch;
 # traffic grows in proportion to the clients a launch covers).  Only kernels that have not
 # changed since that capture are listed.
-NCU_DRAM_BYTES_PER_COORD = {"f_mid": (536.88 + 482.55) * 1e6 / 2 ** 27}
+NCU_DRAM_BYTES_PER_COORD = {"f_mid": (536.9 + 483.3) * 1e6 / 2 ** 27}
 
 
 def host_cores() -> int:
