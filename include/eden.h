@@ -16,9 +16,9 @@
  *     non-finite vector, a client with no packet) are reported through the device
  *     status word, read with eden_status().
  *   - bits (the per-client budget b) and seed (the randomness a sender shares with the
- *     receiver, Section 2.1) are side information both sides agree on (Section 4.1:
- *     "b does need to be sent or otherwise agreed upon"); they are arguments on both
- *     sides and are not stored in the message.  Seeds must differ between clients and
+ *     receiver, Section 2.1) are side information both sides agree on (Section 4.1
+ *     leaves it to the two sides to transmit b or fix it beforehand); they are
+ *     arguments on both sides and are not stored in the message.  Seeds must differ between clients and
  *     between rounds; that is the caller's duty.
  *   - Supported budgets: 0 < b <= 1 (one-bit codes; b < 1 adds the shared-seed
  *     sparsification of Section 4.1), the integers 2..8 (Section 3) and non-integer
@@ -149,10 +149,13 @@ int eden_encode(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32
  *   recv_masks host array of n dev pointers or NULL; entry c (NULL = nothing lost)
  *              points to eden_recv_mask_words() words, bit i of word i/32 = packet i
  *              arrived.  Lost coordinates count as 0 and p_c = received/D (Section 4.2).
- *   acc        dev fp32[d], read and written.
- *   n_used     host, optional: set to n; clients with no packet received are skipped
- *              and flagged (status NO_DATA) but still counted, because the mean of
- *              Section 2.2.2 is over all n senders.
+ *   acc        dev fp32[d], read and written; 4-byte alignment is enough, a vector that
+ *              is also 16-byte aligned takes the faster kernels (the same holds for the
+ *              output of eden_mean and eden_mean_partial).
+ *   n_used     host, optional: n is ADDED to *n_used (the caller zeroes it before the
+ *              first call of a round and divides acc by it after the last); clients
+ *              with no packet received are skipped and flagged (status NO_DATA) but
+ *              still counted, because the mean of Section 2.2.2 is over all n senders.
  * No per-client estimate is stored for b >= 1; clients with b < 1 use the workspace. */
 int eden_decode_accumulate(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
                            const double* bits, const uint64_t* seeds,
@@ -198,7 +201,8 @@ int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bi
  * calls on a device share the one array, which keeps the previous call's contents (the
  * entry point clears what must start at zero): two calls whose GPU work overlaps -- two
  * streams, two threads -- race on it; run them on one stream or order them yourself.
- * Asynchronous on cuda_stream like the other entry points. */
+ * Asynchronous on cuda_stream like the other entry points.  The calling thread's current
+ * device is the same after the call as before it. */
 #define EDEN_NOALLOC_MAX_DIM (1ull << 24)
 int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stream, uint64_t seed,
                                      uint64_t d, double bits, uint32_t* mask_bits);
@@ -287,6 +291,21 @@ uint64_t eden_launch_count(const eden_ctx* ctx);
 /* Cross-checking aid: with on != 0 every call on this context uses the shape-generic
  * kernels instead of the register-blocked ones (same results, slower). */
 int eden_force_generic_kernels(eden_ctx* ctx, int on);
+
+/* Tuning switches of a context (tests and experiments; the defaults are the fastest
+ * measured forms).  Unknown options or values return EDEN_ERR_INVALID_ARG.
+ *   EDEN_OPT_PLAN_VARIANT  0 (default): no thread-block clusters; 1..3: an 8-block cluster
+ *                          stage on the column pass, on the row pass, or on both, which
+ *                          saves one sweep over HBM for 2^24..2^27 coordinates.
+ *   EDEN_OPT_ROW_STAGING   1: the sender's last pass runs as a persistent kernel whose
+ *                          tiles are staged in shared memory by bulk asynchronous copies.
+ *   EDEN_OPT_SEL_ROUNDS    2 (default): the threshold of a b < 1 mask is found in two passes
+ *                          over the keys where the candidate list holds them; 3: always in
+ *                          three histogram rounds (the form very long vectors use). */
+#define EDEN_OPT_PLAN_VARIANT 1
+#define EDEN_OPT_ROW_STAGING  2
+#define EDEN_OPT_SEL_ROUNDS   3
+int eden_set_option(eden_ctx* ctx, int option, int value);
 
 /* Optional per-kernel timing for benchmarks: while enabled, every kernel launch is
  * bracketed by CUDA events on the context's stream.  eden_profile_collect synchronises

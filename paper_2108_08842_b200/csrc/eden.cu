@@ -4,7 +4,6 @@
 
 #include <algorithm>
 #include <cmath>
-#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -222,6 +221,7 @@ struct eden_ctx {
     bool force_generic;
     int plan_variant;
     int row_staging;                 // 1: the sender's row pass runs in its persistent, bulk-copy-staged form
+    int sel_rounds;                  // 3: the b < 1 mask threshold is found in three histogram rounds at every size
     int sm_count;
     std::vector<ProfileRecord> records;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
@@ -296,9 +296,8 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->copy_out = nullptr;
     ctx->force_generic = false;
     ctx->plan_variant = 0;
-    if (const char* pv = std::getenv("EDEN_PLAN_VARIANT")) ctx->plan_variant = std::atoi(pv);
     ctx->row_staging = 0;
-    if (const char* rs = std::getenv("EDEN_ROW_STAGING")) ctx->row_staging = std::atoi(rs);
+    ctx->sel_rounds = 2;
     ctx->sm_count = 0;
     if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cuda_device) != cudaSuccess ||
         ctx->sm_count <= 0) {
@@ -338,6 +337,27 @@ extern "C" int eden_force_generic_kernels(eden_ctx* ctx, int on)
     if (!ctx) return EDEN_ERR_INVALID_ARG;
     ctx->force_generic = on != 0;
     return EDEN_OK;
+}
+
+extern "C" int eden_set_option(eden_ctx* ctx, int option, int value)
+{
+    if (!ctx) return EDEN_ERR_INVALID_ARG;
+    switch (option) {
+        case EDEN_OPT_PLAN_VARIANT:
+            if (value < 0 || value > 3) return EDEN_ERR_INVALID_ARG;
+            ctx->plan_variant = value;
+            return EDEN_OK;
+        case EDEN_OPT_ROW_STAGING:
+            if (value != 0 && value != 1) return EDEN_ERR_INVALID_ARG;
+            ctx->row_staging = value;
+            return EDEN_OK;
+        case EDEN_OPT_SEL_ROUNDS:
+            if (value != 2 && value != 3) return EDEN_ERR_INVALID_ARG;
+            ctx->sel_rounds = value;
+            return EDEN_OK;
+        default:
+            return EDEN_ERR_INVALID_ARG;
+    }
 }
 
 extern "C" int eden_profile_enable(eden_ctx* ctx, int on)
@@ -505,11 +525,9 @@ constexpr uint64_t kCandBytes = (uint64_t)kSelCandCap * sizeof(uint2);
 // The two-pass selection holds the keys that share tau's first digit, about d / 2048 of
 // them (a binomial count): used while that, with a margin of many standard deviations,
 // fits the candidate list.
-bool two_pass_selection(uint64_t d)
+bool two_pass_selection(const eden_ctx* ctx, uint64_t d)
 {
-    // EDEN_SEL_ROUNDS=3 keeps the three histogram rounds at every size (tuning and tests)
-    if (const char* e = std::getenv("EDEN_SEL_ROUNDS"))
-        if (std::atoi(e) == 3) return false;
+    if (ctx->sel_rounds == 3) return false;      // EDEN_OPT_SEL_ROUNDS: three rounds at every size
     const double mean = (double)d / (double)kSelBins;
     return mean + 12.0 * std::sqrt(mean) + 64.0 <= (double)kSelCandCap;
 }
@@ -520,18 +538,18 @@ uint64_t keep_bitmap_bytes(uint64_t d)
     return align_up((d + kSelChunk - 1) / kSelChunk * (kSelChunk / 8), 256);
 }
 
-uint64_t sel_scratch_bytes(uint64_t d)
+uint64_t sel_scratch_bytes(const eden_ctx* ctx, uint64_t d)
 {
     const uint64_t n_chunks = (d + kSelChunk - 1) / kSelChunk;
     return 256 + kBatchHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) +
-           align_up(sizeof(SelJob), 256) + (two_pass_selection(d) ? kCandBytes + keep_bitmap_bytes(d) : 0);
+           align_up(sizeof(SelJob), 256) + (two_pass_selection(ctx, d) ? kCandBytes + keep_bitmap_bytes(d) : 0);
 }
 
 // Groups: clients of one rotation dimension (and, within it, of one kind: b >= 1 or
 // b < 1) are launched together, split so that each group's work buffers and selection
 // scratch fit the workspace.  Larger dimensions first, so that for the mean a group with
 // b >= 1, which covers every output coordinate, comes before any b < 1 group.
-int make_groups(const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_bytes,
+int make_groups(const eden_ctx* ctx, const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_bytes,
                 std::vector<Group>& groups)
 {
     std::vector<uint32_t> idx(plan.size());
@@ -550,7 +568,7 @@ int make_groups(const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_b
         g.fractional = plan[idx[i]].coin_thr != 0;
         g.uniform = plan[idx[i]].delta > 0.0;
         const uint64_t need = (plan[idx[i]].needs_work ? work_buffer_bytes(plan[idx[i]].D) : 0) +
-                              (g.subbit ? sel_scratch_bytes(d) : 0);
+                              (g.subbit ? sel_scratch_bytes(ctx, d) : 0);
         if (need > work_bytes) return EDEN_ERR_WORKSPACE;
         uint64_t used = 0;
         while (i < idx.size() && plan[idx[i]].L == g.L && plan[idx[i]].subbit == g.subbit &&
@@ -924,7 +942,7 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
     char* chunk_base = hist_base + kBatchHistBytes * n;
     char* job_base = chunk_base + chunk_bytes * n;
     char* cand_base = job_base + align_up(sizeof(SelJob), 256) * n;
-    const bool two_pass = two_pass_selection(d);
+    const bool two_pass = two_pass_selection(ctx, d);
     std::vector<SelJob> jobs(partial);
     for (uint32_t j = 0; j < n; ++j) {
         jobs[j].sel = (MaskSelect*)(sel_base + 256ull * j);
@@ -1044,7 +1062,7 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
     rc = carve(ctx, d, n, delta != nullptr, lay);
     if (rc) return rc;
     std::vector<Group> groups;
-    rc = make_groups(plan, d, lay.work_bytes, groups);
+    rc = make_groups(ctx, plan, d, lay.work_bytes, groups);
     if (rc) return rc;
     const FixedLayout f = fixed_layout(d);
     const bool x_aligned = ((uintptr_t)x & 15u) == 0 && (ld_x & 3u) == 0;
@@ -1175,7 +1193,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
                          const uint32_t* const* recv_masks, uint64_t d, uint32_t n,
                          float* out, uint64_t divisor /* 0: accumulate into out; else overwrite out with the sum / divisor */)
 {
-    if (!ctx || !codes || !scales || !seeds || !out) return EDEN_ERR_INVALID_ARG;
+    if (!ctx || !codes || !scales || !seeds || !out || ((uintptr_t)out & 3u)) return EDEN_ERR_INVALID_ARG;
     const bool mean = divisor != 0;
     std::vector<ClientPlan> plan;
     int rc = plan_clients(d, n, bits, delta, plan);
@@ -1187,9 +1205,12 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
     rc = carve(ctx, d, n, delta != nullptr, lay);
     if (rc) return rc;
     std::vector<Group> groups;
-    rc = make_groups(plan, d, lay.work_bytes, groups);
+    rc = make_groups(ctx, plan, d, lay.work_bytes, groups);
     if (rc) return rc;
     const FixedLayout f = fixed_layout(d);
+    // the register-blocked last pass moves `out` 16 bytes at a time; a vector that is not
+    // 16-byte aligned goes through the shape-generic kernels, whose accesses are scalar
+    const bool out_aligned = ((uintptr_t)out & 15u) == 0;
 
     std::vector<ClientDesc> descs;
     descs.reserve(n);
@@ -1270,7 +1291,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         // with OUT_YHAT every member writes its own estimate: one block row per member
         const uint32_t loop_n = g.subbit ? 1u : gn;
         const unsigned rows = g.subbit ? gn : 1u;
-        if (fast_eligible(ctx, g)) {
+        if (fast_eligible(ctx, g) && (out_aligned || g.subbit)) {
             rc = fast_decode_group(ctx, plan, g, d_descs + first, d_states + first, out, d, mode,
                                    (float*)(ctx->ws + lay.work_off + group_work_end[gi]),
                                    lay.work_bytes - group_work_end[gi]);
@@ -1338,7 +1359,7 @@ extern "C" int eden_decode_accumulate(eden_ctx* ctx, const uint8_t* const* codes
 {
     if (!bits) return EDEN_ERR_INVALID_ARG;
     const int rc = decode_common(ctx, codes, scales, bits, nullptr, seeds, recv_masks, d, n, acc, 0);
-    if (rc == EDEN_OK && n_used) *n_used = n;
+    if (rc == EDEN_OK && n_used) *n_used += n;
     return rc;
 }
 
@@ -1350,7 +1371,7 @@ extern "C" int eden_decode_accumulate_uniform(eden_ctx* ctx, const int8_t* const
     if (!delta) return EDEN_ERR_INVALID_ARG;
     const int rc = decode_common(ctx, (const uint8_t* const*)index, scales, nullptr, delta, seeds, recv_masks,
                                  d, n, acc, 0);
-    if (rc == EDEN_OK && n_used) *n_used = n;
+    if (rc == EDEN_OK && n_used) *n_used += n;
     return rc;
 }
 
@@ -1619,6 +1640,24 @@ int noalloc_scratch(int device, unsigned char** out)
     return EDEN_OK;
 }
 
+// Makes `device` current for the life of the object and puts the caller's device back.
+struct DeviceScope {
+    int previous;
+    bool changed;
+    cudaError_t status;
+    explicit DeviceScope(int device) : previous(-1), changed(false), status(cudaGetDevice(&previous))
+    {
+        if (status == cudaSuccess && previous != device) {
+            status = cudaSetDevice(device);
+            changed = status == cudaSuccess;
+        }
+    }
+    ~DeviceScope()
+    {
+        if (changed) cudaSetDevice(previous);
+    }
+};
+
 }  // namespace
 
 extern "C" int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stream, uint64_t seed,
@@ -1626,7 +1665,8 @@ extern "C" int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stre
 {
     if (!mask_bits || d == 0 || !(bits > 0.0) || !(bits < 1.0)) return EDEN_ERR_INVALID_ARG;
     if (d > kNoallocMaxDim) return EDEN_ERR_TOO_LARGE;
-    CUDA_OK(cudaSetDevice(cuda_device));
+    const DeviceScope scope(cuda_device);          // the caller's current device is put back on return
+    CUDA_OK(scope.status);
     unsigned char* base = nullptr;
     const int rc = noalloc_scratch(cuda_device, &base);
     if (rc) return rc;

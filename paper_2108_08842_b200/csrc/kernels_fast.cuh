@@ -921,7 +921,7 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
 // (cp.async.bulk, completion on an mbarrier) while the block works on the tile it holds in
 // registers, so the global-memory latency of a tile is hidden behind the arithmetic of the
 // one before it.  Every wait on the mbarrier is bounded; a wait that runs out raises
-// EDEN_STATUS_TIMEOUT and the block returns.
+// EDEN_STATUS_TIMEOUT and the block returns after one more bounded wait for that copy.
 // ---------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals)
 {
@@ -1014,6 +1014,10 @@ k_f_enc_last_staged(const ClientDesc* __restrict__ descs, ClientState* __restric
         // reads before the next tile's first exchange writes
     }
     if (s_fail) {
+        // the copy whose wait ran out may still be in flight and would land in shared memory
+        // that the next block on this SM owns: give it one more bounded wait before leaving
+        // (no further copy was started after the failure)
+        mbar_wait_bounded(&bar, parity ^ 1u);
         if (t == 0) atomicOr(status, kStatusTimeout);
         return;
     }

@@ -72,11 +72,13 @@ _sig("eden_mean_uniform", _int, [_vp, _vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp])
 _sig("eden_index_histogram", _int, [_vp, _vp, _u64, _u32, _vp])
 _sig("eden_profile_enable", _int, [_vp, _int])
 _sig("eden_force_generic_kernels", _int, [_vp, _int])
+_sig("eden_set_option", _int, [_vp, _int, _int])
 _sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
 _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(_u64),
                                 ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
 
 STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA, STATUS_TIMEOUT, STATUS_SCRATCH = 1, 2, 4, 8, 16
+OPT_PLAN_VARIANT, OPT_ROW_STAGING, OPT_SEL_ROUNDS = 1, 2, 3
 PACKET_COORDS = 1024
 UNIFORM_MAX_INDEX = 127
 UNIFORM_MIN_DELTA = 0.0625
@@ -297,9 +299,10 @@ class Context:
                                       d, n, int(n_total), out.data_ptr()))
         return out
 
-    def decode_accumulate(self, codes, scales, bits, seeds, d: int, acc: torch.Tensor, recv_masks=None):
-        """eden_decode_accumulate: acc += sum_c x_hat_c; returns the number of clients counted."""
-        used = _u32(0)
+    def decode_accumulate(self, codes, scales, bits, seeds, d: int, acc: torch.Tensor, recv_masks=None,
+                          used_so_far: int = 0):
+        """eden_decode_accumulate: acc += sum_c x_hat_c; returns used_so_far + the clients counted."""
+        used = _u32(used_so_far)
         self._decode(_lib.eden_decode_accumulate, codes, scales, bits, seeds, recv_masks, d, acc,
                      extra=(ctypes.byref(used),))
         return int(used.value)
@@ -343,6 +346,10 @@ class Context:
 
     def force_generic_kernels(self, on: bool):
         _check(_lib.eden_force_generic_kernels(self._h, 1 if on else 0))
+
+    def set_option(self, option: int, value: int):
+        """eden_set_option: OPT_PLAN_VARIANT / OPT_ROW_STAGING / OPT_SEL_ROUNDS."""
+        _check(_lib.eden_set_option(self._h, int(option), int(value)))
 
     def profile(self, on: bool):
         _check(_lib.eden_profile_enable(self._h, 1 if on else 0))

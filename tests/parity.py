@@ -14,6 +14,15 @@ def unpack_codes(words: np.ndarray, D: int, W: int) -> np.ndarray:
     return (bits.reshape(D, W).astype(np.uint32) * weights).sum(axis=1).astype(np.uint32)
 
 
+def codes_at(words: np.ndarray, idx: np.ndarray, W: int) -> np.ndarray:
+    """Codes of the coordinates `idx` only (same layout as unpack_codes)."""
+    w = np.concatenate([words.astype(np.uint64), np.zeros(1, dtype=np.uint64)])
+    o = idx.astype(np.uint64) * np.uint64(W)
+    a, off = (o >> np.uint64(5)).astype(np.int64), o & np.uint64(31)
+    both = w[a] | (w[a + 1] << np.uint64(32))
+    return ((both >> off) & np.uint64((1 << W) - 1)).astype(np.uint32)
+
+
 def unpack_fractional(words: np.ndarray, D: int, W0: int, coins: np.ndarray) -> np.ndarray:
     """Codes of a non-integer-budget message: groups of 32 coordinates, W0+1 words each."""
     codes = np.zeros(D, dtype=np.int64)
@@ -46,7 +55,7 @@ def near_boundary(z: np.ndarray, W: int) -> np.ndarray:
 def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, bits: float, seed: int,
                         enc=None):
     """Returns (mismatching coordinates, all inside the boundary window?, scale rel. error, oracle result).
-    `enc` may carry a precomputed oracle result (without z); z is recomputed only on a mismatch."""
+    `enc` may carry a precomputed oracle result; if it has no z, z is recomputed on a mismatch."""
     if enc is None:
         enc = O.encode(x, bits, seed)
     d = x.shape[0]
@@ -56,7 +65,9 @@ def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, 
     mism = 0
     ok = True
     if diff.size:
-        z = O.encode(x, bits, seed, want_z=True)["z"]
+        z = enc.get("z")
+        if z is None:
+            z = O.encode(x, bits, seed, want_z=True)["z"]
         thr = O.coin_threshold(bits)
         if thr:
             # non-integer budget: per-coordinate width; a boundary of either table counts
@@ -69,12 +80,17 @@ def check_encode_client(gpu_words: np.ndarray, gpu_scale: float, x: np.ndarray, 
             ok = ok and bool(np.all(np.abs(g[bad] - o[bad]) == 1))
             rel = abs(gpu_scale - enc["scale"]) / abs(enc["scale"]) if enc["scale"] != 0 else abs(gpu_scale)
             return mism, ok, rel, enc
-        g = unpack_codes(gpu_words, D, W)
-        o = unpack_codes(enc["codes"], D, W)
-        bad = np.nonzero(g != o)[0]
+        # only the coordinates with a bit in a differing word can differ
+        first = (diff.astype(np.int64) * 32) // W
+        last = np.minimum((diff.astype(np.int64) * 32 + 31) // W, D - 1)
+        cand = np.unique(np.concatenate([np.arange(f, l + 1) for f, l in zip(first, last)]))
+        g = codes_at(gpu_words[:nw], cand, W)
+        o = codes_at(enc["codes"], cand, W)
+        differ = g != o
+        bad = cand[differ]
         mism = int(bad.size)
         ok = bool(np.all(near_boundary(z[bad], W)))
         # a mismatch may only move the code to the neighbouring interval
-        ok = ok and bool(np.all(np.abs(g[bad].astype(np.int64) - o[bad].astype(np.int64)) == 1))
+        ok = ok and bool(np.all(np.abs(g[differ].astype(np.int64) - o[differ].astype(np.int64)) == 1))
     rel = abs(gpu_scale - enc["scale"]) / abs(enc["scale"]) if enc["scale"] != 0 else abs(gpu_scale)
     return mism, ok, rel, enc

@@ -37,11 +37,14 @@ def _ctx(E, d, n):
     return E.Context(0, d_max=d, n_batch=n)
 
 
-def run_workload(E, work, threads=8, check_clients=None):
-    """Encode parity for the chosen clients, decode+mean parity for all of them."""
+def run_workload(E, work, threads=8, check_clients=None, options=()):
+    """Encode parity for the chosen clients, decode+mean parity for all of them.
+    `options`: (option, value) pairs for eden_set_option."""
     n, d = work.n, work.d
     xs = work.vectors()
     ctx = _ctx(E, d, n)
+    for opt, val in options:
+        ctx.set_option(opt, val)
     x_gpu = torch.from_numpy(xs).cuda()
     codes, scales = ctx.encode(x_gpu, work.bits, work.seeds)
     torch.cuda.synchronize()
@@ -86,8 +89,9 @@ def run_workload(E, work, threads=8, check_clients=None):
 
     # accumulate entry point: acc += sum of estimates
     acc = torch.full((d,), 0.5, dtype=torch.float32, device="cuda")
-    used = ctx.decode_accumulate(g_codes, torch.from_numpy(o_scales).cuda(), bits, seeds, d, acc, masks_t)
-    assert used == len(clients)
+    used = ctx.decode_accumulate(g_codes, torch.from_numpy(o_scales).cuda(), bits, seeds, d, acc, masks_t,
+                                 used_so_far=5)
+    assert used == 5 + len(clients)          # the count is added to, not overwritten
     err = np.max(np.abs(acc.cpu().numpy().astype(np.float64) - 0.5 - mean_ref * len(clients)))
     assert err <= MEAN_TOL * np.max(np.abs(mean_ref)) * len(clients) + 1e-6
 
@@ -149,35 +153,33 @@ def test_shapes_and_ragged_tails(E, d, bits):
     run_workload(E, work)
 
 
-@pytest.mark.parametrize("variant", ["0", "1", "2", "3"])
-def test_pass_plans_at_2_pow_24_and_25(E, variant, monkeypatch):
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
+def test_pass_plans_at_2_pow_24_and_25(E, variant):
     # plan 0 (default) sweeps three times without clusters; plans 1-3 put an 8-block
     # cluster stage on the column pass, on the row pass or on both (2^25 always needs
     # both).  All plans must give the same answers.
-    monkeypatch.setenv("EDEN_PLAN_VARIANT", variant)
     for d, bits in (((1 << 24) - 3, 2.0), (1 << 25, 1.0)):
-        if variant in ("2", "3") and d == 1 << 25:
+        if variant in (2, 3) and d == 1 << 25:
             continue
         rng = np.random.default_rng(d % 1000)
         n = 2
         xs = rng.standard_normal((n, d)).astype(np.float32)
         work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(d % 77, n), 0.05,
                               lambda c: xs[c], d % 77)
-        run_workload(E, work)
+        run_workload(E, work, options=[(E.OPT_PLAN_VARIANT, variant)])
 
 
 @pytest.mark.parametrize("bits", [1.0, 2.0, 4.0, 8.0, 2.5])
-def test_sender_row_pass_staged_by_bulk_copies(E, bits, monkeypatch):
+def test_sender_row_pass_staged_by_bulk_copies(E, bits):
     # the persistent form of the sender's last pass (tiles staged in shared memory by bulk
     # asynchronous copies) must give the same messages as the default form; three clients of
     # 2^20 rotated coordinates are 384 tiles, several per resident block with a ragged split
-    monkeypatch.setenv("EDEN_ROW_STAGING", "1")
     d, n = (1 << 20) - 5, 3
     rng = np.random.default_rng(int(bits * 10))
     xs = rng.standard_normal((n, d)).astype(np.float32)
     work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(17, n), 0.0,
                           lambda c: xs[c], 17)
-    run_workload(E, work)
+    run_workload(E, work, options=[(E.OPT_ROW_STAGING, 1)])
 
 
 @pytest.mark.parametrize("n,d", [(11, (1 << 17) - 9), (37, (1 << 15) + 5)])
@@ -222,27 +224,24 @@ def test_sub_bit_budgets_and_mask(E, bits, d):
 
 
 @pytest.mark.parametrize("bits,d", [(0.1, 200003), (0.5, 70001), (0.9, 9)])
-def test_sub_bit_selection_in_three_histogram_rounds(E, bits, d, monkeypatch):
+def test_sub_bit_selection_in_three_histogram_rounds(E, bits, d):
     # vectors too long for the candidate list of the two-pass selection find the mask's
     # threshold in three histogram rounds over all keys; forced here at sizes the oracle sorts quickly
-    monkeypatch.setenv("EDEN_SEL_ROUNDS", "3")
     n = 3
     rng = np.random.default_rng(d)
     xs = rng.standard_normal((n, d)).astype(np.float32)
     work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(d + 2, n), 0.0, lambda c: xs[c], d)
-    run_workload(E, work)
+    run_workload(E, work, options=[(E.OPT_SEL_ROUNDS, 3)])
 
 
 @pytest.mark.parametrize("rounds", [2, 3])
 @pytest.mark.parametrize("which,extra", [(0, 1), (1, 2), (2, 1)])
-def test_mask_threshold_on_a_pair_of_equal_keys(E, which, extra, rounds, monkeypatch):
+def test_mask_threshold_on_a_pair_of_equal_keys(E, which, extra, rounds):
     # Section 4.1 asks for a sample of exactly d*p coordinates.  With seed 1 and d = 2^17 three
     # pairs of coordinates draw the same 32-bit key; putting the k-th smallest key on such a
     # pair makes the selection decide by coordinate: extra = 1 keeps only the pair's first
     # coordinate, extra = 2 keeps both.  Both forms of the batched selection and the
     # single-mask entry point must agree with the oracle's full sort.
-    if rounds == 3:
-        monkeypatch.setenv("EDEN_SEL_ROUNDS", "3")
     d, seed = 1 << 17, 1
     keys = np.array([O.mask_key(seed, i) for i in range(d)], dtype=np.uint64)
     sk = keys[np.lexsort((np.arange(d), keys))]
@@ -262,7 +261,7 @@ def test_mask_threshold_on_a_pair_of_equal_keys(E, which, extra, rounds, monkeyp
     xs = rng.standard_normal((2, d)).astype(np.float32)
     work = synth.Workload("adhoc", 2, d, np.full(2, bits), np.array([seed, seed + 1], dtype=np.uint64), 0.0,
                           lambda c: xs[c], k)
-    run_workload(E, work)
+    run_workload(E, work, options=[(E.OPT_SEL_ROUNDS, rounds)])
 
 
 @pytest.mark.parametrize("bits,d", [(1.5, 100), (1.5, 40000), (2.25, 5000), (7.5, 3000), (3.75, 300000)])
@@ -429,6 +428,53 @@ def test_host_buffer_entry_points(E, d, n):
     dev = ctx.mean(dcodes, dscales, work.bits, work.seeds, d,
                    [torch.from_numpy(m.view(np.int32)).cuda() for m in masks]).cpu().numpy()
     assert np.array_equal(out, dev)
+    ctx.close()
+    # the host path against the oracle itself: its messages (Section 2.2.1) and, from those
+    # messages, its mean (Sections 2.2.2, 4.2)
+    total = 0
+    for c in range(n):
+        mism, ok, rel, _ = parity.check_encode_client(codes[c].view(np.uint32), float(scales[c]), xs[c],
+                                                      float(work.bits[c]), int(work.seeds[c]))
+        assert ok and rel <= SCALE_TOL, (c, mism, rel)
+        total += mism
+    assert total <= 20
+    ref, used = O.mean([c.view(np.uint32)[: O.code_words(d, float(b))] for c, b in zip(codes, work.bits)],
+                       [float(s) for s in scales], [float(b) for b in work.bits],
+                       [int(s) for s in work.seeds], d, masks, threads=4)
+    assert used == n
+    assert np.max(np.abs(out.astype(np.float64) - ref)) <= MEAN_TOL * np.max(np.abs(ref))
+
+
+@pytest.mark.parametrize("d,bits", [(20000, 2.0), ((1 << 21) + 7, 1.0)])
+def test_output_vector_that_is_only_4_byte_aligned(E, d, bits):
+    # mean / acc one float past a 16-byte boundary: the receiver must not use its 128-bit
+    # stores on it (it takes the shape-generic kernels) and gives the same mean
+    n = 3
+    rng = np.random.default_rng(d)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    seeds = [int(s) for s in synth.client_seeds(d + 3, n)]
+    enc = [O.encode(xs[c], bits, seeds[c]) for c in range(n)]
+    ref, _ = O.mean([e["codes"] for e in enc], [float(np.float32(e["scale"])) for e in enc], [bits] * n, seeds, d)
+    ctx = _ctx(E, d, n)
+    g_codes = []
+    for e in enc:
+        buf = np.zeros(E.code_bytes(d, bits), dtype=np.uint8)
+        buf[: e["codes"].nbytes] = e["codes"].view(np.uint8)
+        g_codes.append(torch.from_numpy(buf).cuda())
+    g_scales = torch.tensor([np.float32(e["scale"]) for e in enc], dtype=torch.float32, device="cuda")
+    buf = torch.zeros(d + 8, dtype=torch.float32, device="cuda")
+    assert buf.data_ptr() % 16 == 0
+    out = buf[1:1 + d]
+    launches = ctx.launch_count
+    ctx.mean(g_codes, g_scales, [bits] * n, seeds, d, None, out)
+    assert ctx.status() == 0 and ctx.launch_count > launches
+    got = buf.cpu().numpy()
+    assert got[0] == 0 and np.all(got[1 + d:] == 0)                 # nothing outside the vector
+    assert np.max(np.abs(got[1:1 + d].astype(np.float64) - ref)) <= MEAN_TOL * np.max(np.abs(ref))
+    ctx.decode_accumulate(g_codes, g_scales, [bits] * n, seeds, d, out)
+    got = buf.cpu().numpy()
+    assert got[0] == 0 and np.all(got[1 + d:] == 0)
+    assert np.max(np.abs(got[1:1 + d].astype(np.float64) - (1 + n) * ref)) <= MEAN_TOL * (1 + n) * np.max(np.abs(ref))
     ctx.close()
 
 

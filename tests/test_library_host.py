@@ -83,6 +83,15 @@ def test_bad_arguments_are_rejected_without_a_gpu(lib):
     assert lib.eden_encode(None, None, 0, 0, 0, None, None, None, None) == -1
     assert lib.eden_mean(None, None, None, None, None, None, 0, 0, None) == -1
     assert lib.eden_status(None, None) == -1
+    lib.eden_set_option.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int]
+    assert lib.eden_set_option(None, 1, 0) == -1
+
+
+def test_the_library_reads_no_environment_variable():
+    # tuning switches are eden_set_option arguments: nothing in the sources asks the environment
+    csrc = os.path.join(ROOT, "paper_2108_08842_b200", "csrc")
+    for name in os.listdir(csrc):
+        assert "getenv" not in open(os.path.join(csrc, name)).read(), name
 
 
 def test_product_package_never_imports_the_oracle():

@@ -147,6 +147,76 @@ def test_quantiser_properties(W):
         assert O.quantise(float(np.nextafter(np.float32(t32), np.float32(np.inf))), W) == half + j + 1
 
 
+@pytest.mark.parametrize("W,count", [(2, 150000), (3, 150000), (4, 400000), (6, 150000), (8, 150000)])
+def test_fp32_interval_decision_leaves_the_double_one_only_inside_the_window(W, count):
+    # The oracle takes the interval of Section 2.2.1 on fp32-rounded operands (the precision
+    # the kernels decide in).  Against the same rule taken in double on the unrounded
+    # boundaries, the code may differ only where |z - t| <= 1e-6 * max(1, |t|) for a
+    # boundary t (the window inside which a mismatch is tolerated), and then only by one.
+    c, b = O.table(W)
+    half = 1 << (W - 1)
+    pos = b[half:]                                       # positive boundaries, ascending
+    rng = np.random.default_rng(100 + W)
+    parts = [rng.standard_normal(count) * 1.3]
+    for t in pos:                                        # dense samples around every boundary
+        parts.append(t * (1.0 + rng.uniform(-4e-7, 4e-7, 600)))
+        parts.append(-t * (1.0 + rng.uniform(-4e-7, 4e-7, 200)))
+        t32 = np.float32(t)
+        ulps = [t32, np.nextafter(t32, np.float32(np.inf)), np.nextafter(t32, np.float32(0))]
+        parts.append(np.array([float(u) for u in ulps] + [-float(u) for u in ulps] +
+                              [float(np.nextafter(t, np.inf)), float(np.nextafter(t, 0.0)), float(t)]))
+    zs = np.concatenate(parts)
+    m = np.searchsorted(pos, np.abs(zs), side="left")    # boundaries strictly below |z|, in double
+    want = np.where(zs < 0, half - 1 - m, half + m)
+    got = np.array([O.quantise(float(z), W) for z in zs])
+    differ = np.nonzero(got != want)[0]
+    if W > 1:
+        assert differ.size > 0                           # the samples do reach the rounding band
+    for i in differ:
+        z = zs[i]
+        dist = np.abs(np.abs(z) - pos)
+        j = int(np.argmin(dist))
+        assert dist[j] <= 1e-6 * max(1.0, pos[j]), (z, pos[j])
+        assert abs(int(got[i]) - int(want[i])) == 1
+    # the widest band in which fp32 rounding can move a decision is far narrower than the window
+    if differ.size:
+        worst = max(np.min(np.abs(np.abs(zs[i]) - pos) / np.maximum(1.0, pos)) for i in differ)
+        assert worst < 2.5e-7
+
+
+def test_mean_divides_by_all_senders_and_skips_one_without_packets():
+    # Section 2.2.2: the estimate is the mean over all n senders.  A sender none of whose
+    # packets arrived contributes nothing, is reported, and the divisor stays n.
+    n, d = 3, 64
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal(d).astype(np.float32)
+    seeds = [11, 12, 13]
+    enc = [O.encode(x, 2.0, s) for s in seeds]           # the same vector under three rotations
+    codes, scales = [e["codes"] for e in enc], [e["scale"] for e in enc]
+    xh = [O.decode(codes[c], scales[c], 2.0, seeds[c], d)[0] for c in range(n)]
+    x64 = x.astype(np.float64)
+    n2 = float(np.dot(x64, x64))
+    for c in range(n):                                   # scale identity per sender (Section 2.3)
+        assert abs(np.dot(xh[c], x64) - n2) < 1e-9 * n2
+    mean, used = O.mean(codes, scales, [2.0] * n, seeds, d)
+    assert used == 3
+    assert np.array_equal(mean, (xh[0] + xh[1] + xh[2]) / 3)
+    # independent of the sum above: <mean, x> = ||x||^2 only if the divisor is n
+    assert abs(np.dot(mean, x64) - n2) < 1e-9 * n2
+    # sender 1 loses its only packet (d = 64 is one short packet)
+    lost = np.zeros(1, dtype=np.uint32)
+    got = np.ones(1, dtype=np.uint32)
+    xh1, nodata = O.decode(codes[1], scales[1], 2.0, seeds[1], d, lost)
+    assert nodata and not np.any(xh1)
+    mean, used = O.mean(codes, scales, [2.0] * n, seeds, d, [got, lost, got])
+    assert used == 2
+    assert np.array_equal(mean, (xh[0] + xh[2]) / 3)
+    assert abs(np.dot(mean, x64) - (2.0 / 3.0) * n2) < 1e-9 * n2
+    # the threaded route takes the same decisions
+    mean_t, used_t = O.mean(codes, scales, [2.0] * n, seeds, d, [got, lost, got], threads=3)
+    assert used_t == 2 and np.array_equal(mean_t, mean)
+
+
 # ----------------------------------------------------------------------------- transform
 @pytest.mark.parametrize("D", [1, 2, 4, 8, 32, 64])
 def test_fwht_against_dense_sylvester_matrix(D):

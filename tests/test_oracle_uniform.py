@@ -146,6 +146,32 @@ def test_index_is_round_to_nearest_with_ties_to_the_inner_interval():
 
 
 # ----------------------------------------------------------------------------- sender / receiver
+@pytest.mark.parametrize("bits", [1.5, 3.0, 5.5])
+def test_fp32_index_decision_leaves_the_double_one_only_inside_the_window(bits):
+    # Section 4.3's index is taken on fp32 operands (boundaries fl32(fl32(Delta) (k - 1/2)));
+    # against round-to-nearest in double with the unrounded Delta it may differ only within
+    # 1e-6 * max(1, |t|) of a boundary t = Delta (k - 1/2), and then by one.
+    delta = O.uniform_delta(bits)
+    ks = np.arange(1, 128, dtype=np.float64)
+    pos = delta * (ks - 0.5)
+    rng = np.random.default_rng(int(bits * 10))
+    parts = [rng.standard_normal(200000) * 1.5]
+    for t in pos[pos < 9.0]:
+        parts.append(t * (1.0 + rng.uniform(-5e-7, 5e-7, 300)))
+        parts.append(-t * (1.0 + rng.uniform(-5e-7, 5e-7, 100)))
+    zs = np.concatenate(parts)
+    m = np.searchsorted(pos, np.abs(zs), side="left")
+    want = np.where(zs < 0, -m, m)
+    got = np.array([O.uniform_index(float(z), delta) for z in zs])
+    differ = np.nonzero(got != want)[0]
+    assert differ.size > 0
+    for i in differ:
+        dist = np.abs(np.abs(zs[i]) - pos)
+        j = int(np.argmin(dist))
+        assert dist[j] <= 1e-6 * max(1.0, pos[j]), (zs[i], pos[j])
+        assert abs(int(got[i]) - int(want[i])) == 1
+
+
 def test_scale_identity_and_reconstruction():
     rng = np.random.default_rng(11)
     for d, b in ((64, 3.0), (1000, 2.0), (4096, 4.0)):
