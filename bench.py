@@ -31,11 +31,29 @@ if ROOT not in sys.path:
 METRIC = "encode and decode+mean GB/s (fp32 in)"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes (read + write) per rotated coordinate and client from the ncu capture in
-# profiles/ncu_full_fast_kernels_cfg5_n1.md (one client of 2^27 coordinates per launch;
-# traffic grows in proportion to the clients a launch covers).  Only kernels that have not
-# changed since that capture are listed.
-NCU_DRAM_BYTES_PER_COORD = {"f_mid": (536.9 + 483.3) * 1e6 / 2 ** 27}
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2108_08842_b200", "csrc", "kernels_fast.cuh")
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+
+
+def ncu_dram_bytes_per_coord():
+    """DRAM bytes (read + write) per rotated coordinate and client of each kernel, from the
+    ncu captures summarised under profiles/ (one client per launch there; traffic grows in
+    proportion to the clients a launch covers).  Each line of the file names the kernel, the
+    figure and the SHA-256 of the kernels' source file at the time of the capture: a figure
+    taken on other source than the one now built is dropped, not reported."""
+    import hashlib
+    out = {}
+    try:
+        with open(KERNEL_SOURCE, "rb") as f:
+            now = hashlib.sha256(f.read()).hexdigest()
+        with open(TRAFFIC_FILE) as f:
+            for line in f:
+                line = line.split("#", 1)[0].split()
+                if len(line) == 3 and line[2] == now:
+                    out[line[0]] = float(line[1])
+    except OSError:
+        pass
+    return out
 
 
 def host_cores() -> int:
@@ -149,16 +167,37 @@ def oracle_sample(work, clients, threads):
     return dt, len(clients) * work.d * 4, mean
 
 
+def full_config(work, n_total, world, sharded=False):
+    return config_of(work, {"parallelism": ("senders split over %d ranks, one all-reduce" % world)
+                            if sharded else "replicas x%d" % world,
+                            "n_clients_total": int(n_total) * (1 if sharded else world)})
+
+
 def run_reference(args):
+    """The oracle, as it stands, on the host cores: per step `threads` clients of the workload
+    in parallel, each at the workload's own dimension where the run still ends within a few
+    minutes, else cut to the largest power of two that does (never below 2^22, so that the
+    transform stays out of the caches and keeps most of its stages)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    import oracle as O
     from paper_2108_08842_b200 import synth
     work = synth.make(args.workload)
     cores = host_cores()
-    # bounded sample per step: `threads` clients, each cut to its first d_s coordinates
     threads = min(cores, work.n, 8)
-    d_s = min(work.d, 1 << 21)
+    # seconds per coordinate and stage, from a probe of one client at 2^21 coordinates; large
+    # transforms that share the memory bus run about twice as slow per butterfly as the probe
+    probe = synth.make(args.workload, d=1 << 21, n=1)
+    t_probe, _, _ = oracle_sample(probe, [0], 1)
+    rate = 2.0 * t_probe / ((1 << 21) * 21.0)
+    budget = 240.0 / (args.steps + args.warmup)
+    d_s = work.d
+    while d_s > (1 << 22):
+        D = O.rot_dim(d_s, 1.0)
+        if rate * D * np.log2(D) <= budget:
+            break
+        d_s = (1 << int(np.log2(d_s))) if d_s & (d_s - 1) else d_s >> 1
     sample = synth.make(args.workload, d=d_s, n=threads)
     times = []
     for step in range(args.warmup + args.steps):
@@ -167,11 +206,14 @@ def run_reference(args):
             times.append(dt)
     ms = 1e3 * float(np.mean(times))
     value = threads * d_s * 4 / (ms * 1e-3) / 1e9
-    desc = "%d clients x first %d coordinates of %s per step, %d threads" % (threads, d_s, work.name, threads)
+    desc = ("%d of the %d clients per step, %s coordinates each (%s), encode + decode+mean, %d threads" %
+            (threads, work.n, d_s, "the workload's dimension" if d_s == work.d else
+             "cut from %d to keep the run within minutes" % work.d, threads))
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": config_of(work),
+            "config": full_config(work, work.n, max(1, args.gpus)),
+            "sample": {"n_clients": threads, "d": int(d_s), "rotation_dim": int(O.rot_dim(d_s, 1.0))},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -300,14 +342,16 @@ def run_gpu(args):
 
     # ---- roofline of the dominant kernel (by event time inside the timed region)
     peak, peak_kind = measured_hbm_peak()
+    traffic_table = ncu_dram_bytes_per_coord()
     top_name = max(kernels, key=lambda k: kernels[k]["ms"])
     top = kernels[top_name]
     achieved = top["bytes"] / top["launches"] / (top["ms"] / top["launches"] * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": top_name, "achieved": achieved, "peak": peak,
                 "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": (NCU_DRAM_BYTES_PER_COORD[top_name] * n * float(eden.rot_dim(d, float(bits[0])))
-                            if top_name in NCU_DRAM_BYTES_PER_COORD and len(set(map(float, bits))) == 1 else None),
-                "traffic_source": "ncu dram__bytes_read+write, one client, scaled by clients per launch",
+                "traffic": (traffic_table[top_name] * n * float(eden.rot_dim(d, float(bits[0])))
+                            if top_name in traffic_table and len(set(map(float, bits))) == 1 else None),
+                "traffic_source": "ncu dram__bytes_read+write, one client, scaled by clients per launch "
+                                  "(profiles/ncu_dram_traffic.txt; null if the kernels changed since the capture)",
                 "algorithmic_bytes_per_launch": top["bytes"] / top["launches"],
                 "ms_per_launch": top["ms"] / top["launches"]}
     kernel_table = {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
@@ -361,21 +405,22 @@ def run_gpu(args):
     # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not uniform and not args.sharded:
+        # one wave of clients at the workload's own dimension (the same rotation the GPU is timed on)
         threads = min(cores, n, 8)
-        d_s = min(d, 1 << 26)       # about 10-30 s of CPU work
-        sample = synth.make(args.workload, d=d_s, n=threads, seed=rank)
+        sample = synth.make(args.workload, d=d, n=threads, seed=rank)
+        if args.bits is not None:
+            sample.bits = np.full(sample.n, float(args.bits))
         dt, nbytes, _ = oracle_sample(sample, list(range(threads)), threads)
         cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": "%d clients x first %d coordinates of %s, encode + decode+mean, %.1f s" %
-                         (threads, d_s, work.name, dt)}
+               "sample": "%d of the %d clients of %s at its own dimension (%d coordinates, rotation of %d), "
+                         "encode + decode+mean, %d threads, %.1f s" %
+                         (threads, n, work.name, d, eden.rot_dim(d, float(bits[0])), threads, dt)}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "strong" if args.sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": config_of(work, {"parallelism": ("senders split over %d ranks, one all-reduce" % world)
-                                           if args.sharded else "replicas x%d" % world,
-                                           "n_clients_total": int(n_total) * (1 if args.sharded else world)}),
+                "config": full_config(work, n_total, world, args.sharded),
                 "encode_gbs": in_bytes / (enc_ms * 1e-3) / 1e9, "decode_mean_gbs": in_bytes / (dec_ms * 1e-3) / 1e9,
                 "encode_ms": enc_ms, "decode_mean_ms": dec_ms,
                 "roofline": roofline, "kernels": kernel_table, "cpu_baseline": cpu, "e2e": e2e,

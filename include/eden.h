@@ -117,6 +117,12 @@ int eden_pass_plan(uint64_t d, double bits, uint32_t* pass_bits, uint32_t max_pa
  * (Section 3: Lloyd-Max for N(0,1), centre-of-mass values).  Host arrays, host only. */
 int eden_table(uint32_t W, float* centroids, float* boundaries);
 
+/* Host only.  The kernels search the intervals of code widths 2..4 with multiply-adds whose
+ * constants are derived from the table above; EDEN_OK if every boundary that search can
+ * form is bit-identical to the table's fp32 boundary (it is, for the tables of Section 3;
+ * eden_create refuses to run otherwise). */
+int eden_self_check(void);
+
 /* ---- context ---------------------------------------------------------------------- */
 
 /* Creates a context bound to a device, a stream (cudaStream_t passed as void*, NULL =
@@ -206,6 +212,38 @@ int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d, double bi
 #define EDEN_NOALLOC_MAX_DIM (1ull << 24)
 int eden_sparsification_mask_noalloc(int cuda_device, void* cuda_stream, uint64_t seed,
                                      uint64_t d, double bits, uint32_t* mask_bits);
+
+/* ---- Section 4.1, the other order: sparsification after the rotation ---------------- */
+
+/* Section 4.1 notes that the random mask of a budget b < 1 can be applied before or after
+ * the rotation, with about the same error; eden_encode applies it before (it shrinks the
+ * transform).  These entry points apply it after: the sender rotates and codes the whole
+ * vector with one bit per coordinate exactly as for b = 1 (same scale S) and sends only the
+ * codes of a random mask over the D = eden_rot_dim(d, 1) ROTATED coordinates, exactly
+ * k' = eden_after_kept_count(d, b) = floor(D b + 1/2) of them (at least 1): the k' smallest
+ * (key, index) pairs of the seed's mask keys, indexed by rotated coordinate.  The message is
+ * the kept codes in increasing index order, one bit each (bit j of the stream = code of the
+ * j-th kept coordinate), eden_after_code_bytes(d, b) bytes, plus S.  The receiver rebuilds
+ * the mask, takes it as the pattern of what arrived, puts 0 elsewhere and multiplies by
+ * 1/p, p = k'/D: the receiver of Section 4.2 (Lemma 4.3) with this mask.  0 < b < 1 for
+ * every client; D up to about 10^8 (larger returns EDEN_ERR_TOO_LARGE); no packet loss on
+ * top.  The workspace must hold eden_after_workspace_bytes(d, n). */
+uint64_t eden_after_kept_count(uint64_t d, double bits);
+uint64_t eden_after_code_bytes(uint64_t d, double bits);
+uint64_t eden_after_workspace_bytes(uint64_t d, uint32_t n);
+/* codes: host array of n dev pointers, each eden_after_code_bytes(d, bits[c]) bytes, 16-byte
+ * aligned, overwritten; other arguments as for eden_encode. */
+int eden_encode_sparsify_after(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                               const double* bits, const uint64_t* seeds,
+                               uint8_t* const* codes, float* scales);
+/* mean[i] = (1/n) sum_c x_hat_c[i] (overwritten) / acc[i] += sum_c x_hat_c[i], *n_used += n;
+ * codes 4-byte aligned; other arguments as for eden_mean / eden_decode_accumulate. */
+int eden_mean_sparsify_after(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                             const double* bits, const uint64_t* seeds,
+                             uint64_t d, uint32_t n, float* mean);
+int eden_decode_accumulate_sparsify_after(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                                          const double* bits, const uint64_t* seeds,
+                                          uint64_t d, uint32_t n, float* acc, uint32_t* n_used);
 
 /* ---- Section 4.3: the uniform-interval family --------------------------------------- */
 

@@ -7,8 +7,10 @@ the product package; only the tests, the smoke check and the benchmark's CPU-bas
 leg may use it.
 
 Parity unpinned (conventions of this implementation, fixed only by oracle == GPU): the wire
-layout of the packed codes, the Philox stream layout, and the tie-breaks at interval
-endpoints and at zero.  Everything else is pinned by ``tests/test_oracle_*.py``.
+layout of the packed codes, the Philox stream layout, the tie-breaks at interval
+endpoints and at zero, and, for the sparsify-after-rotation variant, that its mask is
+drawn over the rotated coordinates with the same key rule and its message is the kept
+sign bits in index order.  Everything else is pinned by ``tests/test_oracle_*.py``.
 """
 from __future__ import annotations
 
@@ -84,6 +86,12 @@ def _L():
         lib.eden_oracle_encode.restype = ctypes.c_int
         lib.eden_oracle_decode.argtypes = [vp, f64, f64, u64, vp, u64, vp]
         lib.eden_oracle_decode.restype = ctypes.c_int
+        lib.eden_oracle_after_kept_count.argtypes = [u64, f64]
+        lib.eden_oracle_after_kept_count.restype = u64
+        lib.eden_oracle_encode_after.argtypes = [vp, u64, f64, u64, vp, vp, vp, vp]
+        lib.eden_oracle_encode_after.restype = ctypes.c_int
+        lib.eden_oracle_decode_after.argtypes = [vp, f64, f64, u64, u64, vp]
+        lib.eden_oracle_decode_after.restype = ctypes.c_int
         for name in ("eden_oracle_uniform_entropy", "eden_oracle_uniform_delta",
                      "eden_oracle_uniform_second_moment"):
             getattr(lib, name).argtypes = [f64]
@@ -284,6 +292,50 @@ def mean(codes, scales, bits, seeds, d: int, recv_masks=None, threads: int = 1):
                     acc += xh
                     used += 1
     return acc / n, used
+
+
+# --------------------------------------------------------------------------- Section 4.1, sparsify after the rotation
+def after_kept_count(d: int, bits: float) -> int:
+    """k' = round(D * bits) rotated coordinates are sent, D = the rotation dimension of d."""
+    return int(_L().eden_oracle_after_kept_count(int(d), float(bits)))
+
+
+def encode_after(x: np.ndarray, bits: float, seed: int, want_z: bool = False, want_mask: bool = False):
+    """One sender, b < 1 with the mask applied to the ROTATED coordinates.
+    Returns dict(codes uint32[ceil(k'/32)], scale, z[D], mask[D])."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    d = x.shape[0]
+    D = rot_dim(d, 1.0)
+    k = after_kept_count(d, bits)
+    codes = np.zeros((k + 31) // 32, dtype=np.uint32)
+    scale = np.zeros(1, dtype=np.float64)
+    z = np.zeros(D, dtype=np.float64) if want_z else None
+    m = np.zeros(D, dtype=np.uint8) if want_mask else None
+    rc = _L().eden_oracle_encode_after(_ptr(x), d, float(bits), int(seed), _ptr(codes), _ptr(scale),
+                                       _ptr(z) if want_z else None, _ptr(m) if want_mask else None)
+    if rc:
+        raise MemoryError("oracle encode_after")
+    return {"codes": codes, "scale": float(scale[0]), "z": z, "mask": m}
+
+
+def decode_after(codes: np.ndarray, scale: float, bits: float, seed: int, d: int) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint32)
+    xhat = np.zeros(d, dtype=np.float64)
+    if _L().eden_oracle_decode_after(_ptr(codes), float(scale), float(bits), int(seed), int(d), _ptr(xhat)):
+        raise MemoryError("oracle decode_after")
+    return xhat
+
+
+def mean_after(codes, scales, bits, seeds, d: int, threads: int = 1) -> np.ndarray:
+    """(1/n) sum_c x_hat_c for senders that sparsified after the rotation."""
+    n = len(seeds)
+    table(1)
+    with ThreadPoolExecutor(max_workers=max(1, threads)) as ex:
+        parts = list(ex.map(lambda c: decode_after(codes[c], scales[c], bits[c], seeds[c], d), range(n)))
+    acc = np.zeros(d, dtype=np.float64)
+    for xh in parts:
+        acc += xh
+    return acc / n
 
 
 # --------------------------------------------------------------------------- Section 4.3

@@ -521,6 +521,88 @@ int eden_oracle_decode(const uint32_t *codes, double S, double bits, uint64_t se
 }
 
 /* ------------------------------------------------------------------------- */
+/* Section 4.1, the other order: sparsify AFTER the rotation.                  */
+/* The sender rotates and codes the whole vector with one bit per coordinate   */
+/* exactly as for b = 1 (same S), then sends only the coordinates of a random  */
+/* mask over the D ROTATED coordinates: exactly k' = floor(D b + 1/2) ones,    */
+/* the k' smallest (key, index) pairs of the shared seed's mask keys, now      */
+/* indexed by the rotated coordinate.  The message is the sign bits of the     */
+/* kept coordinates in increasing index order (k' bits).  The receiver puts 0  */
+/* for the others and multiplies by 1/p, p = k'/D, which is Lemma 4.3 with     */
+/* this mask as the deterministic one.           [mask rule and layout unpinned] */
+/* ------------------------------------------------------------------------- */
+uint64_t eden_oracle_after_kept_count(uint64_t d, double bits)
+{
+    uint64_t D = eden_oracle_rot_dim(d, 1.0);
+    return eden_oracle_kept_count(D, bits);
+}
+
+int eden_oracle_encode_after(const float *x, uint64_t d, double bits, uint64_t seed,
+                             uint32_t *codes, double *scale_out, double *z_out, uint8_t *mask_out)
+{
+    uint64_t D = eden_oracle_rot_dim(d, 1.0);
+    uint64_t k = eden_oracle_after_kept_count(d, bits);
+    double *y = (double *)calloc(D, sizeof(double));
+    uint8_t *mask = (uint8_t *)malloc(D);
+    if (!y || !mask) { free(y); free(mask); return -1; }
+    if (eden_oracle_mask(seed, D, k, mask)) { free(y); free(mask); return -1; }
+    if (mask_out) memcpy(mask_out, mask, D);
+    for (uint64_t i = 0; i < d; ++i) y[i] = (double)x[i];
+    double N2 = 0.0;
+    for (uint64_t i = 0; i < D; ++i) N2 += y[i] * y[i];
+    memset(codes, 0, sizeof(uint32_t) * ((k + 31u) / 32u));
+    if (N2 == 0.0) {
+        *scale_out = 0.0;
+        if (z_out) memset(z_out, 0, sizeof(double) * D);
+        free(y); free(mask);
+        return 0;
+    }
+    for (uint64_t i = 0; i < D; ++i) y[i] *= eden_oracle_sign(seed, i);
+    eden_oracle_fwht(y, D);
+    double inv_sqrt_D = 1.0 / sqrt((double)D);
+    for (uint64_t i = 0; i < D; ++i) y[i] *= inv_sqrt_D;          /* r = R(x) */
+    double eta = sqrt((double)D) / sqrt(N2);
+    double dot = 0.0;
+    uint64_t j = 0;                                               /* next bit of the message */
+    for (uint64_t i = 0; i < D; ++i) {
+        double z = eta * y[i];
+        uint32_t code = eden_oracle_quantise(z, 1);
+        dot += y[i] * eden_oracle_value(code, 1);                 /* over ALL coordinates: S as for b = 1 */
+        if (mask[i]) {
+            codes[j / 32u] |= code << (j % 32u);
+            ++j;
+        }
+        if (z_out) z_out[i] = z;
+    }
+    *scale_out = N2 / dot;
+    free(y); free(mask);
+    return 0;
+}
+
+int eden_oracle_decode_after(const uint32_t *codes, double S, double bits, uint64_t seed,
+                             uint64_t d, double *xhat)
+{
+    uint64_t D = eden_oracle_rot_dim(d, 1.0);
+    uint64_t k = eden_oracle_after_kept_count(d, bits);
+    double *q = (double *)calloc(D, sizeof(double));
+    uint8_t *mask = (uint8_t *)malloc(D);
+    if (!q || !mask) { free(q); free(mask); return -1; }
+    if (eden_oracle_mask(seed, D, k, mask)) { free(q); free(mask); return -1; }
+    uint64_t j = 0;
+    for (uint64_t i = 0; i < D; ++i)
+        if (mask[i]) {
+            q[i] = eden_oracle_value((codes[j / 32u] >> (j % 32u)) & 1u, 1);
+            ++j;
+        }
+    double p = (double)k / (double)D;
+    eden_oracle_fwht(q, D);
+    double f = S / (p * sqrt((double)D));
+    for (uint64_t i = 0; i < d; ++i) xhat[i] = q[i] * f * eden_oracle_sign(seed, i);
+    free(q); free(mask);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Section 4.3: the uniform-interval family                                    */
 /*   I_Delta = { [Delta (n - 1/2), Delta (n + 1/2)] : n integer },             */
 /* its entropy H = -sum_n p_n log2 p_n under N(0,1), Delta_b = the smallest    */

@@ -90,7 +90,86 @@ struct Tables {
     float pos_boundary[256];
     float pos_value[256];
     std::vector<float> centroids[9], boundaries[9];
+    FmaTree tree[5];
+    bool tree_exact;
 };
+
+// fma(a, b, c) rounded towards zero, for a in {0, 1} and operands whose exact sum fits a double
+float fma_rz_host(float a, float b, float c)
+{
+    const double exact = (double)a * (double)b + (double)c;
+    float f = (float)exact;
+    if ((double)f != exact && std::fabs((double)f) > std::fabs(exact)) f = std::nextafterf(f, 0.f);
+    return f;
+}
+
+// x and its two neighbours
+void neighbours(double x, float out[3])
+{
+    const float f = (float)x;
+    out[0] = std::nextafterf(f, -INFINITY);
+    out[1] = f;
+    out[2] = std::nextafterf(f, INFINITY);
+}
+
+// Constants of the multiply-add interval search (FmaTree) for W = 2..4 from the positive
+// fp32 boundaries: every boundary the search forms must be bit-identical to -2^30 times the
+// table's boundary, so each difference is picked among the rounded difference and its two
+// neighbours, checked over all indicator combinations.  Returns false if no choice works.
+bool build_fma_tree(int W, const float* pb, const float* pv, FmaTree& tr)
+{
+    std::memset(&tr, 0, sizeof(tr));
+    const float big = 1073741824.f;                       // 2^30
+    tr.big = big;
+    float T[7];
+    for (int j = 0; j + 1 < (1 << (W - 1)); ++j) T[j] = -big * pb[j];     // exact: a power of two
+    if (W == 2) {
+        tr.k_root = T[0];
+        tr.v0 = pv[0];
+        tr.dv = pv[1] - pv[0];
+        return true;
+    }
+    if (W == 3) {
+        tr.k_root = T[1];
+        tr.b1 = T[0];
+        float cand[3];
+        neighbours((double)T[2] - (double)T[0], cand);
+        for (float a : cand)
+            if (fma_rz_host(1.f, a, T[0]) == T[2]) { tr.a1 = a; return true; }
+        return false;
+    }
+    tr.k_root = T[3];
+    tr.b1 = T[1];
+    tr.b_lo = T[0];
+    bool ok = false;
+    float c1[3], cl[3], ch[3], cb[3];
+    neighbours((double)T[5] - (double)T[1], c1);
+    for (float a : c1)
+        if (fma_rz_host(1.f, a, T[1]) == T[5]) { tr.a1 = a; ok = true; break; }
+    if (!ok) return false;
+    neighbours((double)T[2] - (double)T[0], cl);
+    neighbours((double)T[6] - (double)T[4], ch);
+    neighbours((double)T[4] - (double)T[0], cb);
+    for (float a_lo : cl)
+        for (float a_hi : ch)
+            for (float db : cb) {
+                float cd[3];
+                neighbours((double)a_hi - (double)a_lo, cd);
+                for (float da : cd) {
+                    bool good = true;
+                    for (int i2 = 0; i2 < 2 && good; ++i2)
+                        for (int i1 = 0; i1 < 2 && good; ++i1) {
+                            const float p = fma_rz_host((float)i2, da, a_lo), q = fma_rz_host((float)i2, db, T[0]);
+                            good = fma_rz_host((float)i1, p, q) == T[4 * i2 + 2 * i1];
+                        }
+                    if (good) {
+                        tr.a_lo = a_lo; tr.da = da; tr.db = db;
+                        return true;
+                    }
+                }
+            }
+    return false;
+}
 
 const Tables& tables()
 {
@@ -107,6 +186,12 @@ const Tables& tables()
             const int half = 1 << (W - 1), off = half - 1;
             for (int j = 0; j < half; ++j) t.pos_value[off + j] = (float)c[half + j];
             for (int j = 0; j + 1 < half; ++j) t.pos_boundary[off + j] = (float)b[half + j];
+        }
+        t.tree_exact = true;
+        std::memset(t.tree, 0, sizeof(t.tree));
+        for (int W = 2; W <= 4; ++W) {
+            const int off = (1 << (W - 1)) - 1;
+            t.tree_exact = build_fma_tree(W, t.pos_boundary + off, t.pos_value + off, t.tree[W]) && t.tree_exact;
         }
     });
     return t;
@@ -161,6 +246,11 @@ extern "C" int eden_table(uint32_t W, float* centroids, float* boundaries)
     std::copy(t.centroids[W].begin(), t.centroids[W].end(), centroids);
     std::copy(t.boundaries[W].begin(), t.boundaries[W].end(), boundaries);
     return EDEN_OK;
+}
+
+extern "C" int eden_self_check(void)
+{
+    return tables().tree_exact ? EDEN_OK : EDEN_ERR_INVALID_ARG;
 }
 
 extern "C" double eden_uniform_entropy(double delta)
@@ -305,7 +395,12 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
         return EDEN_ERR_CUDA;
     }
     const Tables& t = tables();
-    if (cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
+    if (!t.tree_exact) {                      // cannot happen with the Lloyd-Max tables (eden_self_check)
+        delete ctx;
+        return EDEN_ERR_INVALID_ARG;
+    }
+    if (cudaMemcpyToSymbol(c_tree, t.tree, sizeof(t.tree)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_pos_value, t.pos_value, sizeof(t.pos_value)) != cudaSuccess ||
         cudaMemsetAsync(ctx->ws, 0, 256, ctx->stream) != cudaSuccess ||
         cudaStreamSynchronize(ctx->stream) != cudaSuccess) {
@@ -929,6 +1024,7 @@ struct SelBatch {
     uint32_t n;
     unsigned grid;       // blocks of 1024 coordinates
     bool two_pass;       // the jobs carry mask bitmaps (k_selc_compact / k_selc_scatter)
+    std::vector<const uint32_t*> keep;   // two_pass: device address of each job's bitmap
 };
 
 int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::vector<SelJob>& partial,
@@ -952,6 +1048,8 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
         jobs[j].keep = two_pass ? (uint32_t*)(cand_base + kCandBytes * n + keep_bitmap_bytes(d) * j) : nullptr;
     }
     batch.two_pass = two_pass;
+    batch.keep.clear();
+    for (uint32_t j = 0; j < n; ++j) batch.keep.push_back(jobs[j].keep);
     batch.d_jobs = (SelJob*)job_base;
     batch.n = n;
     batch.grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
@@ -1084,6 +1182,7 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
             cd.src = p.subbit ? cd.work : x + (uint64_t)p.index * ld_x;
             cd.codes = (uint32_t*)codes[p.index];
             cd.recv = nullptr;
+            cd.recv_shift = 10;
             cd.seed = seeds[p.index];
             cd.valid = p.k;
             cd.d = d;
@@ -1188,10 +1287,13 @@ extern "C" int eden_encode_uniform(eden_ctx* ctx, const float* x, uint64_t ld_x,
 // ------------------------------------------------------------------------------------
 // receiver
 // ------------------------------------------------------------------------------------
+// recv_shift: log2 of the coordinates one bit of a recv_masks bitmap stands for: 10 for
+// packets (Section 4.2); 0 for a bitmap with one bit per rotated coordinate (one-bit codes only).
 static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
                          const double* bits, const double* delta, const uint64_t* seeds,
                          const uint32_t* const* recv_masks, uint64_t d, uint32_t n,
-                         float* out, uint64_t divisor /* 0: accumulate into out; else overwrite out with the sum / divisor */)
+                         float* out, uint64_t divisor /* 0: accumulate into out; else overwrite out with the sum / divisor */,
+                         uint32_t recv_shift = 10)
 {
     if (!ctx || !codes || !scales || !seeds || !out || ((uintptr_t)out & 3u)) return EDEN_ERR_INVALID_ARG;
     const bool mean = divisor != 0;
@@ -1231,6 +1333,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             cd.src = nullptr;
             cd.codes = (uint32_t*)codes[p.index];
             cd.recv = recv_masks ? recv_masks[p.index] : nullptr;
+            cd.recv_shift = recv_shift;
             cd.seed = seeds[p.index];
             cd.valid = p.k;
             cd.d = d;
@@ -1268,7 +1371,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         const Group& g = groups[gi];
         const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
         int mode = g.subbit ? OUT_YHAT : (written ? OUT_ACC : OUT_WRITE);
-        SelBatch batch{nullptr, 0, 0};
+        SelBatch batch{nullptr, 0, 0, false, {}};
         uint64_t kept = 0;
         if (g.subbit) {
             // exact-size masks of all members (the estimates of their kept coordinates will
@@ -1442,6 +1545,167 @@ extern "C" int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d
            (const MaskSelect*)(ctx->ws + f.sel), (const unsigned long long*)(ctx->ws + f.chunks),
            (const float*)nullptr, (float*)nullptr, mask_bits);
     return EDEN_OK;
+}
+
+// ------------------------------------------------------------------------------------
+// Section 4.1, the other order: sparsification after the rotation.  The sender runs the
+// one-bit encode of the whole vector and keeps the codes of a random mask over the
+// rotated coordinates; the receiver spreads them back, takes the mask as the pattern of
+// what arrived (Lemma 4.3) and decodes as under loss.  The full code streams, the masks
+// and the selection scratch live at the tail of the workspace for the call.
+// ------------------------------------------------------------------------------------
+extern "C" uint64_t eden_after_kept_count(uint64_t d, double bits)
+{
+    return eden_kept_count(eden_rot_dim(d, 1.0), bits);
+}
+
+extern "C" uint64_t eden_after_code_bytes(uint64_t d, double bits)
+{
+    const uint64_t words = (eden_after_kept_count(d, bits) + 31) / 32;
+    return (words * 4 + 15) / 16 * 16;
+}
+
+namespace {
+
+uint64_t after_tail_bytes(const eden_ctx* ctx, uint64_t D, uint32_t n)
+{
+    return (uint64_t)n * (align_up(eden_code_bytes(D, 1.0), 256) + sel_scratch_bytes(ctx, D) + 256) + 4096;
+}
+
+struct AfterCall {
+    std::vector<uint8_t*> full;          // full one-bit code stream of each client (device)
+    SelBatch batch;
+    uint64_t D, head_bytes;              // head_bytes: what is left of the workspace for the ordinary call
+    unsigned chunk_grid;
+};
+
+// carves the tail of the workspace and starts the mask selection over the D rotated coordinates
+int after_begin(eden_ctx* ctx, uint64_t d, uint32_t n, const double* bits, const uint64_t* seeds, AfterCall& ac)
+{
+    if (!ctx || !bits || !seeds || d == 0 || n == 0) return EDEN_ERR_INVALID_ARG;
+    if (d > EDEN_MAX_DIM) return EDEN_ERR_TOO_LARGE;
+    for (uint32_t c = 0; c < n; ++c)
+        if (!(bits[c] > 0.0) || !(bits[c] < 1.0)) return EDEN_ERR_UNSUPPORTED_BITS;
+    ac.D = eden_rot_dim(d, 1.0);
+    if (!two_pass_selection(ctx, ac.D)) return EDEN_ERR_TOO_LARGE;      // the bitmap form of the selection only
+    CUDA_OK(cudaSetDevice(ctx->device));
+    const uint64_t tail = after_tail_bytes(ctx, ac.D, n);
+    if (tail + fixed_layout(1).end > ctx->ws_bytes) return EDEN_ERR_WORKSPACE;
+    ac.head_bytes = (ctx->ws_bytes - tail) / 256 * 256;
+    char* p = ctx->ws + ac.head_bytes;
+    const uint64_t full_bytes = align_up(eden_code_bytes(ac.D, 1.0), 256);
+    ac.full.resize(n);
+    for (uint32_t c = 0; c < n; ++c) ac.full[c] = (uint8_t*)(p + full_bytes * c);
+    ac.chunk_grid = (unsigned)(((ac.D + kSelChunk - 1) / kSelChunk + kSelThreads / 32 - 1) / (kSelThreads / 32));
+    return EDEN_OK;
+}
+
+// starts the selection with the jobs' stream pointers set (in -> out as k_after_rotation_bits reads them)
+int after_select(eden_ctx* ctx, AfterCall& ac, uint32_t n, const double* bits, const uint64_t* seeds,
+                 const std::vector<const void*>& in, const std::vector<void*>& out)
+{
+    std::vector<SelJob> jobs(n);
+    for (uint32_t c = 0; c < n; ++c) {
+        std::memset(&jobs[c], 0, sizeof(SelJob));
+        jobs[c].seed = seeds[c];
+        jobs[c].d = ac.D;
+        jobs[c].k = eden_kept_count(ac.D, bits[c]);
+        jobs[c].in = (const float*)in[c];
+        jobs[c].out = (float*)out[c];
+    }
+    char* region = ctx->ws + ac.head_bytes + align_up(eden_code_bytes(ac.D, 1.0), 256) * (uint64_t)n;
+    return start_selection_batch(ctx, region, ac.D, jobs, ac.batch);
+}
+
+}  // namespace
+
+extern "C" uint64_t eden_after_workspace_bytes(uint64_t d, uint32_t n)
+{
+    const uint64_t D = eden_rot_dim(d ? d : 1, 1.0);
+    const uint64_t n_chunks = (D + kSelChunk - 1) / kSelChunk;
+    // the larger of the two selection forms, as eden_workspace_bytes reserves it
+    const uint64_t sel = 256 + kBatchHistBytes + align_up(n_chunks * sizeof(unsigned long long), 256) +
+                         align_up(sizeof(SelJob), 256) + kCandBytes + keep_bitmap_bytes(D);
+    return eden_workspace_bytes(d, n) +
+           (uint64_t)(n ? n : 1) * (align_up(eden_code_bytes(D, 1.0), 256) + sel + 256) + 4096 + 512;
+}
+
+extern "C" int eden_encode_sparsify_after(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint32_t n,
+                                          const double* bits, const uint64_t* seeds,
+                                          uint8_t* const* codes, float* scales)
+{
+    if (!codes) return EDEN_ERR_INVALID_ARG;
+    AfterCall ac;
+    int rc = after_begin(ctx, d, n, bits, seeds, ac);
+    if (rc) return rc;
+    for (uint32_t c = 0; c < n; ++c)
+        if (!codes[c] || ((uintptr_t)codes[c] & 15u)) return EDEN_ERR_INVALID_ARG;
+    // the whole vector with one bit per rotated coordinate, exactly as for b = 1
+    const std::vector<double> one(n, 1.0);
+    const uint64_t saved = ctx->ws_bytes;
+    ctx->ws_bytes = ac.head_bytes;
+    rc = encode_common(ctx, x, ld_x, d, n, one.data(), nullptr, seeds, ac.full.data(), scales);
+    ctx->ws_bytes = saved;
+    if (rc) return rc;
+    std::vector<const void*> in(n);
+    std::vector<void*> out(n);
+    for (uint32_t c = 0; c < n; ++c) {
+        in[c] = ac.full[c];
+        out[c] = codes[c];
+        CUDA_OK(cudaMemsetAsync(codes[c], 0, eden_after_code_bytes(d, bits[c]), ctx->stream));
+    }
+    rc = after_select(ctx, ac, n, bits, seeds, in, out);
+    if (rc) return rc;
+    const uint64_t n_chunks = (ac.D + kSelChunk - 1) / kSelChunk;
+    LAUNCH(ctx, "after_pack", n * (double)ac.D / 4.0, k_after_rotation_bits<true>, dim3(ac.chunk_grid, n), kSelThreads, 0,
+           (const SelJob*)ac.batch.d_jobs, n_chunks);
+    return EDEN_OK;
+}
+
+static int after_decode(eden_ctx* ctx, const uint8_t* const* codes, const float* scales, const double* bits,
+                        const uint64_t* seeds, uint64_t d, uint32_t n, float* out, uint64_t divisor)
+{
+    if (!codes || !scales || !out) return EDEN_ERR_INVALID_ARG;
+    AfterCall ac;
+    int rc = after_begin(ctx, d, n, bits, seeds, ac);
+    if (rc) return rc;
+    for (uint32_t c = 0; c < n; ++c)
+        if (!codes[c] || ((uintptr_t)codes[c] & 3u)) return EDEN_ERR_INVALID_ARG;
+    std::vector<const void*> in(n);
+    std::vector<void*> full(n);
+    for (uint32_t c = 0; c < n; ++c) {
+        in[c] = codes[c];
+        full[c] = ac.full[c];
+    }
+    rc = after_select(ctx, ac, n, bits, seeds, in, full);
+    if (rc) return rc;
+    const uint64_t n_chunks = (ac.D + kSelChunk - 1) / kSelChunk;
+    LAUNCH(ctx, "after_unpack", n * (double)ac.D / 4.0, k_after_rotation_bits<false>, dim3(ac.chunk_grid, n), kSelThreads, 0,
+           (const SelJob*)ac.batch.d_jobs, n_chunks);
+    // the mask is the pattern of what arrived: the receiver counts it and divides by p (Lemma 4.3)
+    const std::vector<double> one(n, 1.0);
+    const uint64_t saved = ctx->ws_bytes;
+    ctx->ws_bytes = ac.head_bytes;
+    rc = decode_common(ctx, (const uint8_t* const*)ac.full.data(), scales, one.data(), nullptr, seeds,
+                       ac.batch.keep.data(), d, n, out, divisor, 0);
+    ctx->ws_bytes = saved;
+    return rc;
+}
+
+extern "C" int eden_mean_sparsify_after(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                                        const double* bits, const uint64_t* seeds,
+                                        uint64_t d, uint32_t n, float* mean)
+{
+    return after_decode(ctx, codes, scales, bits, seeds, d, n, mean, n);
+}
+
+extern "C" int eden_decode_accumulate_sparsify_after(eden_ctx* ctx, const uint8_t* const* codes, const float* scales,
+                                                     const double* bits, const uint64_t* seeds,
+                                                     uint64_t d, uint32_t n, float* acc, uint32_t* n_used)
+{
+    const int rc = after_decode(ctx, codes, scales, bits, seeds, d, n, acc, 0);
+    if (rc == EDEN_OK && n_used) *n_used += n;
+    return rc;
 }
 
 // ------------------------------------------------------------------------------------

@@ -12,7 +12,7 @@ struct ClientDesc {
     const float* src;        // encode: fp32 input row (x_c, or the compacted vector for b < 1)
     float* work;             // fp32[D] intermediate of the multi-pass transform
     uint32_t* codes;         // packed codes (encode writes, decode reads)
-    const uint32_t* recv;    // decode: received-packet bitmap or nullptr
+    const uint32_t* recv;    // decode: bitmap of what arrived (bit j = coordinates [j << recv_shift, (j + 1) << recv_shift)) or nullptr
     uint64_t seed;           // shared seed
     uint64_t valid;          // number of meaningful coordinates before padding (d or k)
     uint64_t d;              // input dimension
@@ -22,6 +22,8 @@ struct ClientDesc {
     uint32_t index;          // position of this client in the caller's arrays
     uint32_t coin_thr;       // non-integer b > 1: coin threshold round(frac * 65536); else 0
     float delta;             // uniform-interval family (Section 4.3): interval width; else 0
+    uint32_t recv_shift;     // log2 coordinates per bit of `recv`: 10 (packets), or 0 (one bit per coordinate, W = 1 only)
+    uint32_t reserved;
     double extra_scale;      // encode: d/k for b < 1 (folded into S), else 1
     double mean_scale;       // decode: 1/n for the mean, 1 for accumulate
     const float* utable;     // uniform-interval family: values of magnitude index 0..127; else nullptr

@@ -494,6 +494,17 @@ __device__ __forceinline__ int row_u(int t, int k)
 __device__ __forceinline__ int row_pad(int u) { return u + 2 * (u >> 4); }
 constexpr int kRowSmemUnits = 4096 + 512;
 
+// row_pad(row_u<ARR>(t, k)) = row_base<ARR>(t) + kRowStride<ARR> * k: the part that depends
+// on the thread is computed once, register k sits at a compile-time offset from it.
+template <int ARR>
+__device__ __forceinline__ int row_base(int t)
+{
+    if (ARR == 0) return t + 2 * (t >> 4);
+    if (ARR == 1) return ((t >> 4) << 8) + ((t >> 4) << 5) + (t & 15);
+    return 18 * t;
+}
+template <int ARR> struct RowStride { static constexpr int value = ARR == 0 ? 288 : ARR == 1 ? 18 : 1; };
+
 template <int LC>
 __device__ __forceinline__ int slice_u(int rank, int t, int k)
 {
@@ -510,17 +521,18 @@ __device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
 {
     const int t = threadIdx.x;
     if (FROM == 2) {
-        ulonglong2* p = reinterpret_cast<ulonglong2*>(s + row_pad(row_u<2>(t, 0)));
+        ulonglong2* p = reinterpret_cast<ulonglong2*>(s + row_base<2>(t));
 #pragma unroll
         for (int k = 0; k < 8; ++k) p[k] = make_ulonglong2(v[2 * k], v[2 * k + 1]);
     } else {
+        u64* p = s + row_base<FROM>(t);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) s[row_pad(row_u<FROM>(t, k))] = v[k];
+        for (int k = 0; k < 16; ++k) p[RowStride<FROM>::value * k] = v[k];
     }
     if (FROM + TO == 3) __syncwarp();
     else __syncthreads();
     if (TO == 2) {
-        const ulonglong2* p = reinterpret_cast<const ulonglong2*>(s + row_pad(row_u<2>(t, 0)));
+        const ulonglong2* p = reinterpret_cast<const ulonglong2*>(s + row_base<2>(t));
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             const ulonglong2 w = p[k];
@@ -528,8 +540,9 @@ __device__ __forceinline__ void row_exchange(u64 (&v)[16], u64* s)
             v[2 * k + 1] = w.y;
         }
     } else {
+        const u64* p = s + row_base<TO>(t);
 #pragma unroll
-        for (int k = 0; k < 16; ++k) v[k] = s[row_pad(row_u<TO>(t, k))];
+        for (int k = 0; k < 16; ++k) v[k] = p[RowStride<TO>::value * k];
     }
 }
 
@@ -585,8 +598,88 @@ __device__ __forceinline__ int fast_magnitude(float az, const float* s_tb)
     return m;
 }
 
+// The same magnitude index for W = 2..4 as arithmetic on the multiply-add pipe, which the
+// butterflies leave half idle, instead of compares and selects on the half-rate ALU pipe.
+// With a boundary t held as T = -2^30 t, the saturated multiply-add sat(az 2^30 + T) is
+// exactly 1 if az > t and exactly 0 otherwise: az - t is zero or at least one unit in the
+// last place of the smaller operand (2^-26 for the smallest boundary), which the factor
+// 2^30 lifts above 1, and the multiply-add rounds once.  The boundary of the next level is
+// itself a multiply-add of that indicator (constants chosen on the host so that, rounded
+// towards zero, it lands exactly on the fp32 boundary), and the index is the sum of the
+// indicators (as a float 0..7) times the subnormal number 2^-149, whose bit pattern is the
+// integer.  A NaN saturates to 0, so the index is always in range.
+__device__ __forceinline__ float fma_sat(float a, float b, float c)
+{
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ u64 fma2_rz(u64 a, u64 b, u64 c)
+{
+    u64 r;
+    asm("fma.rz.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ u64 mul2(u64 a, u64 b)
+{
+    u64 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+// The constants of the search, those of the inner levels in both halves of a packed pair:
+// two coordinates go through the tree together, their saturated multiply-adds one by one
+// (no packed form saturates), everything else as one packed instruction for the two.
+struct TreePairs {
+    float big, k_root;
+    u64 a1, b1, da, a_lo, db, b_lo, two, w1;
+};
+template <int W>
+__device__ __forceinline__ TreePairs load_tree_pairs()
+{
+    const FmaTree& tr = c_tree[W];
+    TreePairs tp;
+    tp.big = tr.big;
+    tp.k_root = tr.k_root;
+    tp.a1 = pack2(tr.a1, tr.a1);
+    tp.b1 = pack2(tr.b1, tr.b1);
+    tp.da = pack2(tr.da, tr.da);
+    tp.a_lo = pack2(tr.a_lo, tr.a_lo);
+    tp.db = pack2(tr.db, tr.db);
+    tp.b_lo = pack2(tr.b_lo, tr.b_lo);
+    tp.two = pack2(2.f, 2.f);
+    // W = 4 takes the index times four, the byte offset of its value in the table
+    tp.w1 = pack2(__uint_as_float(W == 4 ? 4u : 1u), __uint_as_float(W == 4 ? 4u : 1u));
+    return tp;
+}
+// `root`: the pair's indicators of the first level (for W = 2 they are the index itself)
+template <int W>
+__device__ __forceinline__ void fma_magnitude_pair(float az0, float az1, const TreePairs& tp, uint32_t& m0, uint32_t& m1,
+                                                   u64& root)
+{
+    static_assert(W >= 2 && W <= 4, "search trees of one to three levels");
+    const u64 ir = pack2(fma_sat(az0, tp.big, tp.k_root), fma_sat(az1, tp.big, tp.k_root));
+    root = ir;
+    u64 m = ir;                                       // Horner form of 4 i_root + 2 i_1 + i_0
+    if (W >= 3) {
+        float t0, t1;
+        unpack2(fma2_rz(ir, tp.a1, tp.b1), t0, t1);
+        const u64 i1 = pack2(fma_sat(az0, tp.big, t0), fma_sat(az1, tp.big, t1));
+        m = fma2(m, tp.two, i1);
+        if (W == 4) {
+            unpack2(fma2_rz(i1, fma2_rz(ir, tp.da, tp.a_lo), fma2_rz(ir, tp.db, tp.b_lo)), t0, t1);
+            const u64 i0 = pack2(fma_sat(az0, tp.big, t0), fma_sat(az1, tp.big, t1));
+            m = fma2(m, tp.two, i0);
+        }
+    }
+    float f0, f1;
+    unpack2(mul2(m, tp.w1), f0, f1);                  // times 2^-149 (W = 4: 2^-147): the bit pattern is the integer
+    m0 = __float_as_uint(f0);
+    m1 = __float_as_uint(f1);
+}
+
 // The thread's 32 consecutive coordinates -> their W words of the code bit stream
-// (coordinate l in bits [l*W, l*W + W) of the 32*W-bit group), and sum |h| Q(|z|).
+// (coordinate l in bits [l*W, l*W + W) of the 32*W-bit group), and sum |h| Q(|z|)
+// (accumulated as sum |z| Q(|z|) for W > 1, so that |z| = |h| / ||y|| is formed once).
 template <int W>
 __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_norm, bool live,
                                                  const float* s_tb, const float* s_tv,
@@ -617,42 +710,86 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
         constexpr int per = 32 / W;
         constexpr uint32_t lsb = W == 2 ? 0x55555555u : W == 4 ? 0x11111111u : 0x01010101u;
         static_assert(W == 2 || W == 4 || W == 8, "field widths that divide 32");
+        TreePairs tp;
+        if constexpr (W <= 4) tp = load_tree_pairs<W>();
+        const u64 value_low2 = pack2(c_tree[2].v0, c_tree[2].v0), value_step2 = pack2(c_tree[2].dv, c_tree[2].dv);
+        u64 dot2 = 0ull;
 #pragma unroll
         for (int j = W - 1; j >= 0; --j) {
-            uint32_t fields = 0u, signs = 0u;
+            // W = 4: the search returns 4 m (see load_tree_pairs), so the fields of a word are
+            // collected times four, in two halves of four fields that cannot overflow
+            uint32_t fields = 0u, fields_hi = 0u, signs = 0u;
 #pragma unroll
-            for (int i = per - 1; i >= 0; --i) {
-                const int l = j * per + i;
+            for (int i = per - 1; i >= 1; i -= 2) {
+                const int l = j * per + i;                           // coordinates l (odd) and l - 1: one unit
                 float h0, h1;
                 unpack2(v[l >> 1], h0, h1);
-                const float h = (l & 1) ? h1 : h0;
-                const float z = h * inv_norm;
-                const int m = fast_magnitude<W>(fabsf(z), s_tb);
-                dot = fmaf(fabsf(h), W <= 2 ? (m ? c_pos_value[half] : c_pos_value[half - 1]) : s_tv[m], dot);
-                fields = (fields << W) | (uint32_t)m;
-                signs = __funnelshift_l(__float_as_uint(z), signs, W);
+                const float az0 = fabsf(h0) * inv_norm, az1 = fabsf(h1) * inv_norm;
+                uint32_t m0, m1;
+                float q0, q1;
+                u64 root = 0ull;
+                if constexpr (W <= 4) {
+                    fma_magnitude_pair<W>(az0, az1, tp, m0, m1, root);
+                } else {
+                    m0 = (uint32_t)fast_magnitude<W>(az0, s_tb);
+                    m1 = (uint32_t)fast_magnitude<W>(az1, s_tb);
+                }
+                if constexpr (W == 2) {
+                    // two values: the smaller plus the indicator times their distance (the sum may
+                    // miss the larger value by one unit in the last place, far inside the scale's tolerance)
+                    dot2 = fma2(pack2(az0, az1), fma2(root, value_step2, value_low2), dot2);
+                } else {
+                    if constexpr (W == 4) {
+                        q0 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_tv) + m0);
+                        q1 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_tv) + m1);
+                    } else {
+                        q0 = s_tv[m0];
+                        q1 = s_tv[m1];
+                    }
+                    dot2 = fma2(pack2(az0, az1), pack2(q0, q1), dot2);
+                }
+                // sums, not ORs: the compiler cannot know that an index fits its field
+                if (W == 4 && i >= per / 2) fields_hi = (fields_hi * 16u + m1) * 16u + m0;
+                else fields = ((((fields << W) + m1) << W) + m0);
+                signs = __funnelshift_l(__float_as_uint(h1), signs, W);
+                signs = __funnelshift_l(__float_as_uint(h0), signs, W);
             }
+            if constexpr (W == 4) fields = (fields_hi << 14) + (fields >> 2);
             const uint32_t neg = (signs >> (W - 1)) & lsb;           // bit 0 of every field whose z is negative
             words[j] = live ? (fields | (lsb << (W - 1))) ^ ((neg << W) - neg) : 0u;
         }
+        float d0, d1;
+        unpack2(dot2, d0, d1);
+        dot = d0 + d1;
     } else {
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = 0u;
+    TreePairs tp;
+    if constexpr (W <= 4) tp = load_tree_pairs<W>();
     // coordinates in descending order
 #pragma unroll
     for (int k = 15; k >= 0; --k) {
         float h[2];
         unpack2(v[k], h[0], h[1]);
+        const float az2[2] = {fabsf(h[0]) * inv_norm, fabsf(h[1]) * inv_norm};
+        uint32_t m2[2];
+        if constexpr (W <= 4) {
+            u64 root;
+            fma_magnitude_pair<W>(az2[0], az2[1], tp, m2[0], m2[1], root);
+        } else {
+            m2[0] = (uint32_t)fast_magnitude<W>(az2[0], s_tb);
+            m2[1] = (uint32_t)fast_magnitude<W>(az2[1], s_tb);
+        }
 #pragma unroll
         for (int e = 1; e >= 0; --e) {
             const int l = 2 * k + e;
-            const float z = h[e] * inv_norm;
-            const int m = fast_magnitude<W>(fabsf(z), s_tb);
-            dot = fmaf(fabsf(h[e]), W <= 2 ? (m ? c_pos_value[half] : c_pos_value[half - 1]) : s_tv[m], dot);
+            const float az = az2[e];
+            const uint32_t m = m2[e];
+            dot = fmaf(az, s_tv[m], dot);
             // code = half + m for z >= 0 and half - 1 - m otherwise: set the top bit, then
-            // flip all W bits where the sign bit of z is set
-            const uint32_t flip = (uint32_t)((int)__float_as_uint(z) >> 31) & (2u * half - 1u);
-            const uint32_t code = ((uint32_t)m | half) ^ flip;
+            // flip all W bits where the sign bit of z (that of h) is set
+            const uint32_t flip = (uint32_t)((int)__float_as_uint(h[e]) >> 31) & (2u * half - 1u);
+            const uint32_t code = (m | half) ^ flip;
             const int a = (l * W) >> 5, off = (l * W) & 31;
             words[a] |= code << off;
             if (off + W > 32) words[a + 1] |= code >> (32 - off);
@@ -662,7 +799,9 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
 #pragma unroll
         for (int j = 0; j < W; ++j) words[j] = 0u;
     }
-    }   // W > 1
+    }
+    // wider codes summed |z| Q(|z|): back to the units of h (one division per thread and tile)
+    if constexpr (W > 1) dot = live ? dot * __frcp_rn(inv_norm) : 0.f;
 }
 
 // ---------------------------------------------------------------------------------
@@ -853,6 +992,7 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
     } else {
         quantise_pack_32<W>(v, inv_norm, live, tab.tb, tab.tv, words, dot);
     }
+    __builtin_assume(__isGlobal(cd.codes));
     store_words<W>(cd.codes + ((base >> 5) + t) * W, words);
     return dot;
 }
@@ -865,12 +1005,15 @@ template <int W, int LC, bool FRAC, bool UNI = false>
 // spilled): cfg5's shape 3240 -> 3370 GB/s, cfg4's 5000 -> 5090 GB/s.  Six fit as well but
 // run slower (2940 / 4310 GB/s, with or without L1 allocation of the tile loads).  The
 // non-integer budgets keep four (their coins cost registers).
-__global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : 5))
+#ifndef EDEN_ENC_LAST_BLOCKS
+#define EDEN_ENC_LAST_BLOCKS (W >= 3 ? 4 : 5)
+#endif
+__global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : EDEN_ENC_LAST_BLOCKS))
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L,
              int inv_ready)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
-    __shared__ double red[32];
+    __shared__ float s_warp_dot[kFastThreads / 32];
     __shared__ float s_inv;
     __shared__ EncTables<W, FRAC> tab;
     const int t = threadIdx.x;
@@ -910,8 +1053,19 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
     }
     const float dot = enc_last_tile<W, FRAC, UNI>(v, cd, &states[blockIdx.y].norm2, base, s, tab, &s_inv,
                                                   inv_ready ? &states[blockIdx.y].factor : nullptr);
-    const double tot = block_sum((double)dot, red);
-    if (t == 0) atomicAdd(&states[blockIdx.y].dot, tot);
+    // the tile's 8192 terms are summed in fp32 (warp shuffles, then eight warp totals), which
+    // is good to a few parts in 10^7; the tiles are summed in double
+    float w = dot;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(0xffffffffu, w, o);
+    if ((t & 31) == 0) s_warp_dot[t >> 5] = w;
+    __syncthreads();
+    if (t == 0) {
+        float tot = 0.f;
+#pragma unroll
+        for (int j = 0; j < kFastThreads / 32; ++j) tot += s_warp_dot[j];
+        atomicAdd(&states[blockIdx.y].dot, (double)tot);
+    }
 }
 
 // ---------------------------------------------------------------------------------
@@ -1062,12 +1216,34 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
     // the tile is 8 packets of 1024 coordinates; this thread's 32 coordinates lie in one.
     // A lost packet reads the zero half of the table (Section 4.2: lost coordinates are 0).
     const uint64_t pkt = (base >> 10) + (uint64_t)(t >> 5);
-    const bool arrived = cd.recv ? ((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u) != 0u : true;
+    const bool per_coord = W == 1 && cd.recv && cd.recv_shift == 0u;      // one bit per coordinate (W = 1 only)
+    const bool arrived = cd.recv && !per_coord ? ((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u) != 0u : true;
     const float* tbl = s_val + (arrived ? 0 : (1 << W));
     uint32_t words[W];
     const uint32_t* src = cd.codes + ((base >> 5) + t) * W;
+    __builtin_assume(__isGlobal(src));
+    __builtin_assume(__isGlobal(cd.work));
+    // the thread's W words in one or two 128-bit (W = 2: 64-bit) loads where the message is
+    // 16-byte aligned (the C ABI asks only for 4 bytes on this side)
+    if ((W == 2 || W == 4 || W == 8) && (reinterpret_cast<uintptr_t>(cd.codes) & 15u) == 0) {
+        if constexpr (W == 2) {
+            const uint2 w2 = __ldg(reinterpret_cast<const uint2*>(src));
+            words[0] = w2.x;
+            words[W > 1 ? 1 : 0] = w2.y;
+        } else {
 #pragma unroll
-    for (int j = 0; j < W; ++j) words[j] = src[j];
+            for (int j = 0; j + 3 < W; j += 4) {
+                const uint4 w4 = __ldg(reinterpret_cast<const uint4*>(src + j));
+                words[j] = w4.x;
+                words[j + 1 < W ? j + 1 : 0] = w4.y;
+                words[j + 2 < W ? j + 2 : 0] = w4.z;
+                words[j + 3 < W ? j + 3 : 0] = w4.w;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < W; ++j) words[j] = __ldg(src + j);
+    }
     u64 v[16];
     if constexpr (FRAC && W >= 2) {
         // non-integer budget: (W-1)-bit fields, then the extra bits of the coordinates whose coin is set
@@ -1095,13 +1271,31 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
     } else if (W == 1) {
         // one bit per coordinate: +-c (or +-0 for a lost packet) by moving the bit into the sign
         const uint32_t minus_c = __float_as_uint(tbl[0]) | 0x80000000u;
+        if (per_coord) {
+            // the thread's 32 coordinates are one word of the bitmap: a coordinate that was not sent is 0
+            const uint32_t kept = cd.recv[(base >> 5) + t];
+#pragma unroll
+            for (int k = 0; k < 16; ++k) {
+                const uint32_t b0 = (words[0] << (31 - 2 * k)) & 0x80000000u;
+                const uint32_t b1 = (words[0] << (30 - 2 * k)) & 0x80000000u;
+                const uint32_t k0 = (uint32_t)((int)(kept << (31 - 2 * k)) >> 31);
+                const uint32_t k1 = (uint32_t)((int)(kept << (30 - 2 * k)) >> 31);
+                v[k] = pack2(__uint_as_float((minus_c ^ b0) & k0), __uint_as_float((minus_c ^ b1) & k1));
+            }
+        } else {
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             const uint32_t b0 = (words[0] << (31 - 2 * k)) & 0x80000000u;
             const uint32_t b1 = (words[0] << (30 - 2 * k)) & 0x80000000u;
             v[k] = pack2(__uint_as_float(minus_c ^ b0), __uint_as_float(minus_c ^ b1));
         }
+        }
     } else {
+        // the field is moved straight to bits [2, W + 2) (one shift), masked and merged with
+        // the bit that selects the zero half of the table (one logic operation): that is
+        // the byte offset of the value, added to the table's address by the load itself
+        const uint32_t lost = arrived ? 0u : (4u << W);
+        const char* tbl_bytes = reinterpret_cast<const char*>(s_val);
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             float q[2];
@@ -1109,9 +1303,12 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
             for (int e = 0; e < 2; ++e) {
                 const int l = 2 * k + e;
                 const int a = (l * W) >> 5, off = (l * W) & 31;
-                uint32_t code = words[a] >> off;
-                if (off + W > 32) code |= words[a + 1] << (32 - off);
-                q[e] = tbl[code & ((1u << W) - 1u)];
+                uint32_t x;
+                if (off >= 2) x = off + W > 32 ? __funnelshift_r(words[a], words[a + 1 < W ? a + 1 : a], off - 2)
+                                               : words[a] >> (off - 2);
+                else x = words[a] << (2 - off);
+                const uint32_t byte_off = (x & (((1u << W) - 1u) << 2)) | lost;
+                q[e] = *reinterpret_cast<const float*>(tbl_bytes + byte_off);
             }
             v[k] = pack2(q[0], q[1]);
         }

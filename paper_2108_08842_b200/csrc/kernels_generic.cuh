@@ -80,6 +80,20 @@ __constant__ float c_pos_value[256];
 
 __device__ __forceinline__ int table_offset(int W) { return (1 << (W - 1)) - 1; }
 
+// The interval search of Section 2.2.1 for code widths 2..4 as arithmetic on the
+// multiply-add pipe (see fma_magnitude in kernels_fast.cuh).  A boundary t is held as
+// -2^30 t; `a*`/`d*` are differences of such values, chosen on the host so that the
+// multiply-adds below (rounded towards zero) land exactly on the fp32 boundaries.
+struct FmaTree {
+    float big;                   // 2^30
+    float k_root;                // the root of the search tree
+    float a1, b1;                // second level (W >= 3):  fma(i_root, a1, b1)
+    float a_lo, da, b_lo, db;    // third level (W = 4):     fma(i_2, fma(i_root, da, a_lo), fma(i_root, db, b_lo))
+    float v0, dv;                // W = 2: the smaller positive value and the step to the larger
+    float pad[6];
+};
+__constant__ FmaTree c_tree[5];  // by code width
+
 // Interval rule of Section 2.2.1 on one normalised coordinate: magnitude index m =
 // number of positive boundaries strictly below |z| (an endpoint belongs to the interval
 // nearer zero), by a branch-free binary search over the sorted boundaries in `tb`.
@@ -268,7 +282,8 @@ k_dec_prep(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     __shared__ double red[32];
     const ClientDesc cd = descs[blockIdx.x];
     const uint64_t D = 1ull << cd.L;
-    const uint64_t packets = (D + 1023) >> 10;
+    const uint64_t per_bit = 1ull << cd.recv_shift;                  // coordinates per bit of the bitmap
+    const uint64_t packets = (D + per_bit - 1) >> cd.recv_shift;
     double cnt = 0.0;
     if (cd.recv) {
         const uint64_t words = (packets + 31) >> 5;
@@ -283,7 +298,7 @@ k_dec_prep(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     }
     const double tot = block_sum(cnt, red);
     if (threadIdx.x == 0) {
-        const double coords = D >= 1024 ? tot * 1024.0 : tot * (double)D;
+        const double coords = D >= per_bit ? tot * (double)per_bit : tot * (double)D;
         const double p = coords / (double)D;
         uint32_t flags = 0;
         float f = 0.f;
@@ -309,7 +324,7 @@ __device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i
     const uint32_t coins = frac ? __ballot_sync(0xffffffffu, coin) : 0u;
     if (!valid) return 0.f;
     if (cd.recv) {
-        const uint64_t pkt = i >> 10;
+        const uint64_t pkt = i >> cd.recv_shift;
         if (!((cd.recv[pkt >> 5] >> (pkt & 31)) & 1u)) return 0.f;
     }
     if (!frac) {

@@ -621,6 +621,81 @@ k_selc_scatter(const SelJob* __restrict__ jobs, uint32_t n_jobs, uint64_t d, flo
     }
 }
 
+// ---------------------------------------------------------------------------------
+// Sparsification after the rotation (Section 4.1, the other order): the mask is over the
+// rotated coordinates and the message is the one-bit codes of the kept ones, in index
+// order.  One warp per chunk of 1024 coordinates (lane l: word l of the chunk's 32 code
+// words and 32 bitmap words); job.in is the full code stream, job.out the message
+// (sender), or the other way round (receiver); both are word arrays passed through the
+// job's float pointers.
+// ---------------------------------------------------------------------------------
+// the bits of `code` at the set positions of `mask`, packed from bit 0
+__device__ __forceinline__ uint32_t bits_extract(uint32_t code, uint32_t mask)
+{
+    uint32_t out = 0u, n = 0u;
+    while (mask) {
+        const uint32_t b = mask & (0u - mask);
+        out |= (code & b) ? (1u << n) : 0u;
+        ++n;
+        mask &= mask - 1u;
+    }
+    return out;
+}
+// the low bits of `bits`, spread to the set positions of `mask`
+__device__ __forceinline__ uint32_t bits_deposit(uint32_t bits, uint32_t mask)
+{
+    uint32_t out = 0u;
+    while (mask) {
+        const uint32_t b = mask & (0u - mask);
+        out |= (bits & 1u) ? b : 0u;
+        bits >>= 1;
+        mask &= mask - 1u;
+    }
+    return out;
+}
+
+// words of the full code stream / the bitmap of one job (both cover whole chunks in the
+// bitmap; the code stream ends at ceil(d / 32) words)
+template <bool PACK>
+__global__ void __launch_bounds__(kSelThreads)
+k_after_rotation_bits(const SelJob* __restrict__ jobs, uint64_t n_chunks)
+{
+    const SelJob job = jobs[blockIdx.y];
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t chunk = (uint64_t)blockIdx.x * (kSelThreads / 32) + (threadIdx.x >> 5);
+    if (chunk >= n_chunks) return;                                    // whole warps leave together
+    const uint64_t w = chunk * 32u + lane;
+    const uint64_t code_words = (job.d + 31u) >> 5;
+    const uint32_t mask = job.keep[w];
+    const uint32_t cnt = (uint32_t)__popc(mask);
+    uint32_t inc = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= (uint32_t)o) inc += v;
+    }
+    const uint64_t pos = job.chunks[chunk] + (uint64_t)(inc - cnt);   // the message bit of the word's first kept coordinate
+    const uint32_t sh = (uint32_t)(pos & 31u);
+    if (PACK) {
+        const uint32_t* full = reinterpret_cast<const uint32_t*>(job.in);
+        uint32_t* msg = reinterpret_cast<uint32_t*>(job.out);
+        if (cnt == 0u) return;
+        const uint32_t bits = bits_extract(w < code_words ? full[w] : 0u, mask);
+        atomicOr(&msg[pos >> 5], bits << sh);                         // the message was cleared before
+        if (sh + cnt > 32u) atomicOr(&msg[(pos >> 5) + 1], bits >> (32u - sh));
+    } else {
+        const uint32_t* msg = reinterpret_cast<const uint32_t*>(job.in);
+        uint32_t* full = reinterpret_cast<uint32_t*>(job.out);
+        uint32_t bits = 0u;
+        if (cnt) {
+            const uint32_t lo = msg[pos >> 5];
+            const uint32_t hi = sh + cnt > 32u ? msg[(pos >> 5) + 1] : 0u;
+            bits = __funnelshift_r(lo, hi, sh);
+        }
+        if (w < code_words) full[w] = bits_deposit(bits, mask);
+    }
+}
+
 // Sender: y_c[pos] = x_c[i] for the kept coordinates of every job.
 __global__ void __launch_bounds__(kSelThreads)
 k_selb_compact(const SelJob* __restrict__ jobs)

@@ -73,6 +73,13 @@ _sig("eden_index_histogram", _int, [_vp, _vp, _u64, _u32, _vp])
 _sig("eden_profile_enable", _int, [_vp, _int])
 _sig("eden_force_generic_kernels", _int, [_vp, _int])
 _sig("eden_set_option", _int, [_vp, _int, _int])
+_sig("eden_self_check", _int, [])
+_sig("eden_after_kept_count", _u64, [_u64, _f64])
+_sig("eden_after_code_bytes", _u64, [_u64, _f64])
+_sig("eden_after_workspace_bytes", _u64, [_u64, _u32])
+_sig("eden_encode_sparsify_after", _int, [_vp, _vp, _u64, _u64, _u32, _vp, _vp, _vp, _vp])
+_sig("eden_mean_sparsify_after", _int, [_vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp])
+_sig("eden_decode_accumulate_sparsify_after", _int, [_vp, _vp, _vp, _vp, _vp, _u64, _u32, _vp, _vp])
 _sig("eden_profile_collect", _int, [_vp, ctypes.POINTER(_u32)])
 _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(_u64),
                                 ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
@@ -122,6 +129,18 @@ def recv_mask_words(d: int, bits: float) -> int:
 
 def workspace_bytes(d_max: int, n_batch: int) -> int:
     return int(_lib.eden_workspace_bytes(d_max, n_batch))
+
+
+def after_kept_count(d: int, bits: float) -> int:
+    return int(_lib.eden_after_kept_count(d, bits))
+
+
+def after_code_bytes(d: int, bits: float) -> int:
+    return int(_lib.eden_after_code_bytes(d, bits))
+
+
+def after_workspace_bytes(d: int, n: int) -> int:
+    return int(_lib.eden_after_workspace_bytes(d, n))
 
 
 def host_workspace_bytes(d: int, n: int) -> int:
@@ -305,6 +324,40 @@ class Context:
         used = _u32(used_so_far)
         self._decode(_lib.eden_decode_accumulate, codes, scales, bits, seeds, recv_masks, d, acc,
                      extra=(ctypes.byref(used),))
+        return int(used.value)
+
+    # ------------------------------------------------------------------ sparsification after the rotation
+    def encode_sparsify_after(self, x: torch.Tensor, bits, seeds, codes: Optional[List[torch.Tensor]] = None,
+                              scales: Optional[torch.Tensor] = None):
+        """eden_encode_sparsify_after: b < 1 with the mask over the rotated coordinates."""
+        assert x.is_cuda and x.dtype == torch.float32 and x.dim() == 2 and x.stride(1) == 1
+        n, d = x.shape
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        if codes is None:
+            codes = [torch.empty(after_code_bytes(d, float(b)), dtype=torch.uint8, device=x.device) for b in bits]
+        if scales is None:
+            scales = torch.empty(n, dtype=torch.float32, device=x.device)
+        _check(_lib.eden_encode_sparsify_after(self._h, x.data_ptr(), x.stride(0), d, n, bits.ctypes.data,
+                                               seeds.ctypes.data, _ptr_table(codes), scales.data_ptr()))
+        return codes, scales
+
+    def mean_sparsify_after(self, codes, scales, bits, seeds, d: int, out: Optional[torch.Tensor] = None):
+        n = len(codes)
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        if out is None:
+            out = torch.empty(d, dtype=torch.float32, device=scales.device)
+        _check(_lib.eden_mean_sparsify_after(self._h, _ptr_table(codes), scales.data_ptr(), bits.ctypes.data,
+                                             seeds.ctypes.data, d, n, out.data_ptr()))
+        return out
+
+    def decode_accumulate_sparsify_after(self, codes, scales, bits, seeds, d: int, acc: torch.Tensor,
+                                         used_so_far: int = 0):
+        n = len(codes)
+        bits, seeds = _f64s(bits), _u64s(seeds)
+        used = _u32(used_so_far)
+        _check(_lib.eden_decode_accumulate_sparsify_after(self._h, _ptr_table(codes), scales.data_ptr(),
+                                                          bits.ctypes.data, seeds.ctypes.data, d, n,
+                                                          acc.data_ptr(), ctypes.byref(used)))
         return int(used.value)
 
     def sparsification_mask(self, seed: int, d: int, bits: float) -> torch.Tensor:

@@ -27,6 +27,9 @@ def test_reference_arm_line():
     assert COMMON <= set(j) and j["impl"] == "reference" and j["unit"] == "GB/s"
     assert j["cpu_baseline"]["kind"] == "oracle" and j["cpu_baseline"]["value"] == j["value"] > 0
     assert j["e2e"]["h2d_bytes_per_step"] == 0 and j["config"]["workload"] == "cfg2"
+    # the configuration is the library arm's, key for key; what the oracle was timed on is said beside it
+    assert j["config"]["parallelism"] == "replicas x1" and j["config"]["n_clients_total"] == 10
+    assert j["sample"]["d"] == 1 << 20 and 1 <= j["sample"]["n_clients"] <= 10
 
 
 @pytest.mark.gpu

@@ -71,6 +71,12 @@ def test_library_tables_match_oracle_tables(lib):
     assert lib.eden_table(9, c.ctypes.data, b.ctypes.data) < 0
 
 
+def test_multiply_add_interval_search_lands_on_the_table_boundaries(lib):
+    # the kernels' search for W = 2..4 forms its boundaries by multiply-adds of constants
+    # derived on the host; the library checks that each lands exactly on the fp32 boundary
+    assert lib.eden_self_check() == 0
+
+
 def test_bad_arguments_are_rejected_without_a_gpu(lib):
     lib.eden_create.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64]
     h = ctypes.c_void_p()

@@ -661,3 +661,88 @@ def test_fractional_budget_unbiased_at_d64():
     vnmse = err2 / trials / np.dot(xd, xd)
     bias2 = np.dot(acc / trials - xd, acc / trials - xd) / np.dot(xd, xd)
     assert bias2 < 3 * vnmse / trials, (bias2, vnmse / trials)
+
+
+# ----------------------------------------------------------------------------- Section 4.1: sparsify after the rotation
+def _dense_after(x, bits, seed):
+    """The sparsify-after-rotation sender and receiver written with a dense rotation matrix
+    (scipy's Sylvester matrix), numpy's sort for the mask and the closed-form one-bit value."""
+    d = x.shape[0]
+    D = 1 << max(0, (d - 1).bit_length())
+    k = min(D, max(1, int(math.floor(D * bits + 0.5))))
+    y = np.zeros(D)
+    y[:d] = x.astype(np.float64)
+    s = O.signs(seed, D)
+    R = scipy.linalg.hadamard(D).astype(np.float64) / math.sqrt(D) * s[None, :] if D > 1 else np.array([[s[0]]])
+    r = R @ y
+    c = math.sqrt(2 / math.pi)
+    q = np.where(r >= 0, c, -c)
+    S = np.dot(y, y) / np.dot(r, q)
+    keys = np.array([O.mask_key(seed, i) for i in range(D)], dtype=np.uint64)
+    kept = np.sort(np.lexsort((np.arange(D), keys))[:k])
+    q_sent = np.zeros(D)
+    q_sent[kept] = q[kept]
+    xhat = (S / (k / D)) * (R.T @ q_sent)
+    return (r >= 0)[kept].astype(np.uint8), S, xhat[:d], kept
+
+
+@pytest.mark.parametrize("d,bits", [(64, 0.5), (100, 0.25), (37, 0.9), (1, 0.5), (256, 0.03)])
+def test_sparsify_after_rotation_against_dense_reference(d, bits):
+    rng = np.random.default_rng(d)
+    x = (rng.standard_normal(d) * 3).astype(np.float32)
+    seed = 900 + d
+    want_bits, S, xhat, kept = _dense_after(x, bits, seed)
+    enc = O.encode_after(x, bits, seed, want_mask=True)
+    k = O.after_kept_count(d, bits)
+    assert k == len(kept) and np.array_equal(np.nonzero(enc["mask"])[0], kept)
+    got_bits = ((enc["codes"][:, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(-1)
+    assert np.array_equal(got_bits[:k], want_bits) and not got_bits[k:].any()
+    assert abs(enc["scale"] - S) <= 1e-12 * abs(S)
+    got = O.decode_after(enc["codes"], enc["scale"], bits, seed, d)
+    assert np.max(np.abs(got - xhat)) <= 1e-10 * max(1.0, np.max(np.abs(xhat)))
+
+
+def test_sparsify_after_rotation_keeping_everything_is_the_one_bit_scheme():
+    # a mask that keeps all D rotated coordinates: the message and the estimate are those of b = 1
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal(1000).astype(np.float32)
+    bits = 1.0 - 1e-9
+    assert O.after_kept_count(1000, bits) == 1024
+    a, b = O.encode_after(x, bits, 77), O.encode(x, 1.0, 77)
+    assert np.array_equal(a["codes"], b["codes"]) and a["scale"] == b["scale"]
+    assert np.array_equal(O.decode_after(a["codes"], a["scale"], bits, 77, 1000),
+                          O.decode(b["codes"], b["scale"], 1.0, 77, 1000)[0])
+
+
+@pytest.mark.parametrize("bits,d", [(0.5, 1 << 13), (0.125, 1 << 13)])
+def test_sparsify_after_rotation_vnmse_matches_lemma_4_3_and_the_other_order(bits, d):
+    # vNMSE -> 1/(p 2/pi) - 1 = pi/(2p) - 1 (Lemma 4.3 with a random mask; Corollary 4.2 gives
+    # the same limit for the mask applied before the rotation; the appendix on loss versus
+    # sub-bit budgets reports the two as identical).  d and d*b are powers of two, so neither
+    # order pads its rotation (padding would drop the share of the error that falls on it)
+    rng = np.random.default_rng(int(bits * 100))
+    x = rng.standard_normal(d).astype(np.float32)
+    n2 = float(np.dot(x.astype(np.float64), x.astype(np.float64)))
+    after = before = 0.0
+    seeds = range(300, 330)
+    for s in seeds:
+        e = O.encode_after(x, bits, s)
+        after += np.sum((O.decode_after(e["codes"], e["scale"], bits, s, d) - x) ** 2) / n2
+        e = O.encode(x, bits, s)
+        before += np.sum((O.decode(e["codes"], e["scale"], bits, s, d)[0] - x) ** 2) / n2
+    p_after = O.after_kept_count(d, bits) / O.rot_dim(d, 1.0)
+    limit = math.pi / (2 * p_after) - 1
+    assert abs(after / len(seeds) - limit) < 0.04 * limit, (after / len(seeds), limit)
+    assert abs(after - before) / len(seeds) < 0.06 * limit
+
+
+def test_sparsify_after_rotation_is_unbiased_at_d64():
+    d, trials = 64, 10000
+    x = np.random.default_rng(64).standard_normal(d).astype(np.float32)
+    acc = np.zeros(d)
+    for s in range(trials):
+        e = O.encode_after(x, 0.5, 50000 + s)
+        acc += O.decode_after(e["codes"], e["scale"], 0.5, 50000 + s, d)
+    x64 = x.astype(np.float64)
+    bias = np.sum((acc / trials - x64) ** 2) / np.sum(x64 ** 2)
+    assert bias < 3 * (math.pi - 1) / trials
