@@ -432,6 +432,71 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------- the paper's sweep
+def run_sweep(args):
+    """The shape of the paper's encode-speed and error sweep (Section 5.2, its Figure 2 and the
+    appendix on vNMSE against dimension): one LogNormal(0,1) vector, d = 2^10 ... 2^lmax by
+    powers of four, b = 1..8.  Prints a markdown table: encode and decode time per vector
+    (median of --steps runs after --warmup, CUDA events on the library's stream, L2 flushed
+    before every run), GB/s of fp32 input, and the estimate's vNMSE beside the limit of
+    Corollary 2.4, 1 / E[Q^2] - 1."""
+    import math
+    import torch
+    import __graft_entry__
+    __graft_entry__.build()
+    from paper_2108_08842_b200 import eden, synth
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)       # larger than the 126 MB L2
+    lmax = args.sweep_max_log2
+
+    def limit(W):                                                       # Corollary 2.4 from the library's own table
+        c, b = eden.table(W)
+        edges = [-math.inf] + [float(t) for t in b] + [math.inf]
+        cdf = lambda t: 0.5 * (1.0 + math.erf(t / math.sqrt(2.0)))
+        eq2 = sum((cdf(edges[j + 1]) - cdf(edges[j])) * float(c[j]) ** 2 for j in range(len(c)))
+        return 1.0 / eq2 - 1.0
+
+    print("| d | b | encode us | encode GB/s | decode us | decode GB/s | vNMSE | Corollary 2.4 | ratio |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    ctx = eden.Context(0, d_max=1 << lmax, n_batch=1)
+    for L in range(10, lmax + 1, 2):
+        d = 1 << L
+        work = synth.make("sweep", d=d, n=1)
+        x = torch.from_numpy(work.vectors()).to(dev)
+        energy = float((x.double() ** 2).sum())
+        for b in range(1, 9):
+            bits = [float(b)]
+            codes = ctx.alloc_codes(d, bits)
+            scales = torch.empty(1, dtype=torch.float32, device=dev)
+            out = torch.empty(d, dtype=torch.float32, device=dev)
+            enc_t, dec_t = [], []
+            for it in range(args.warmup + args.steps):
+                flush.fill_(it & 0xFF)
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record()
+                ctx.encode(x, bits, work.seeds, codes, scales)
+                e1.record()
+                flush.fill_((it + 1) & 0xFF)
+                e1b = torch.cuda.Event(enable_timing=True)
+                e1b.record()
+                ctx.mean(codes, scales, bits, work.seeds, d, None, out)
+                e2.record()
+                torch.cuda.synchronize()
+                if it >= args.warmup:
+                    enc_t.append(e0.elapsed_time(e1) * 1e3)
+                    dec_t.append(e1b.elapsed_time(e2) * 1e3)
+            enc_us, dec_us = float(np.median(enc_t)), float(np.median(dec_t))
+            vnmse = float(((out.double() - x[0].double()) ** 2).sum()) / energy
+            lim = limit(b)
+            print("| 2^%d | %d | %.1f | %.1f | %.1f | %.1f | %.5g | %.5g | %.3f |" %
+                  (L, b, enc_us, 4.0 * d / enc_us / 1e3, dec_us, 4.0 * d / dec_us / 1e3, vnmse, lim, vnmse / lim))
+            assert ctx.status() == 0
+        del x
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -451,8 +516,13 @@ def main():
     ap.add_argument("--uniform-bits", type=float, default=None,
                     help="use the uniform-interval family (Section 4.3) at this entropy budget instead of the "
                          "Lloyd-Max tables; device-resident timing only (no end-to-end or CPU leg)")
+    ap.add_argument("--sweep", action="store_true",
+                    help="print the LogNormal sweep table (d = 2^10 ... by powers of four, b = 1..8) instead of the JSON line")
+    ap.add_argument("--sweep-max-log2", type=int, default=26)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

@@ -90,7 +90,7 @@ struct Tables {
     float pos_boundary[256];
     float pos_value[256];
     std::vector<float> centroids[9], boundaries[9];
-    FmaTree tree[5];
+    FmaTree tree[9];
     bool tree_exact;
 };
 
@@ -189,9 +189,18 @@ const Tables& tables()
         }
         t.tree_exact = true;
         std::memset(t.tree, 0, sizeof(t.tree));
-        for (int W = 2; W <= 4; ++W) {
+        for (int W = 2; W <= 8; ++W) {
             const int off = (1 << (W - 1)) - 1;
-            t.tree_exact = build_fma_tree(W, t.pos_boundary + off, t.pos_value + off, t.tree[W]) && t.tree_exact;
+            if (W <= 4) {
+                t.tree_exact = build_fma_tree(W, t.pos_boundary + off, t.pos_value + off, t.tree[W]) && t.tree_exact;
+            } else {
+                // wider tables: the tree settles the top three bits of the index, i.e. it
+                // searches the seven boundaries at the eighth points of the table
+                float coarse[7];
+                const int eighth = (1 << (W - 1)) / 8;
+                for (int j = 0; j < 7; ++j) coarse[j] = t.pos_boundary[off + (j + 1) * eighth - 1];
+                t.tree_exact = build_fma_tree(4, coarse, t.pos_value + off, t.tree[W]) && t.tree_exact;
+            }
         }
     });
     return t;

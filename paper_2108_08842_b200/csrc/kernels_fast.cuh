@@ -568,38 +568,8 @@ __device__ __forceinline__ void row_step_inner(u64 (&v)[16])
 // W code words itself.
 // =================================================================================
 // Magnitude index of |z| in the 2^(W-1) positive intervals (Section 2.2.1): the number of
-// positive boundaries strictly below |z|.  Up to four bits the boundaries are
-// compile-time-indexed constants and the search is a tree of selects; wider tables are
-// searched in shared memory.
-template <int W>
-__device__ __forceinline__ int fast_magnitude(float az, const float* s_tb)
-{
-    constexpr int off = (1 << (W - 1)) - 1;
-    if (W == 1) return 0;
-    if (W == 2) return az > c_pos_boundary[off] ? 1 : 0;
-    if (W == 3) {
-        const bool b1 = az > c_pos_boundary[off + 1];
-        const float t0 = b1 ? c_pos_boundary[off + 2] : c_pos_boundary[off + 0];
-        return (b1 ? 2 : 0) + (az > t0 ? 1 : 0);
-    }
-    if (W == 4) {
-        const bool b2 = az > c_pos_boundary[off + 3];
-        const float t1 = b2 ? c_pos_boundary[off + 5] : c_pos_boundary[off + 1];
-        const bool b1 = az > t1;
-        const float lo = b1 ? c_pos_boundary[off + 2] : c_pos_boundary[off + 0];
-        const float hi = b1 ? c_pos_boundary[off + 6] : c_pos_boundary[off + 4];
-        const float t0 = b2 ? hi : lo;
-        return (b2 ? 4 : 0) + (b1 ? 2 : 0) + (az > t0 ? 1 : 0);
-    }
-    int m = 0;
-#pragma unroll
-    for (int step = (1 << (W - 1)) >> 1; step >= 1; step >>= 1)
-        m += (az > s_tb[m + step - 1]) ? step : 0;
-    return m;
-}
-
-// The same magnitude index for W = 2..4 as arithmetic on the multiply-add pipe, which the
-// butterflies leave half idle, instead of compares and selects on the half-rate ALU pipe.
+// positive boundaries strictly below |z|, found by arithmetic on the multiply-add pipe
+// instead of compares and selects on the half-rate ALU pipe.
 // With a boundary t held as T = -2^30 t, the saturated multiply-add sat(az 2^30 + T) is
 // exactly 1 if az > t and exactly 0 otherwise: az - t is zero or at least one unit in the
 // last place of the smaller operand (2^-26 for the smallest boundary), which the factor
@@ -647,16 +617,23 @@ __device__ __forceinline__ TreePairs load_tree_pairs()
     tp.db = pack2(tr.db, tr.db);
     tp.b_lo = pack2(tr.b_lo, tr.b_lo);
     tp.two = pack2(2.f, 2.f);
-    // W = 4 takes the index times four, the byte offset of its value in the table
-    tp.w1 = pack2(__uint_as_float(W == 4 ? 4u : 1u), __uint_as_float(W == 4 ? 4u : 1u));
+    // W >= 4 takes the index times four, the byte offset of its value in the table; for
+    // W >= 5 the tree of constants settles the top three bits of the index only
+    const uint32_t unit = W >= 4 ? 4u << (W - 4) : 1u;
+    tp.w1 = pack2(__uint_as_float(unit), __uint_as_float(unit));
     return tp;
 }
 // `root`: the pair's indicators of the first level (for W = 2 they are the index itself)
+// Returns the magnitude indices (W <= 3) or four times them, the byte offsets into a table
+// of floats (W >= 4).  For W >= 5 the tree of constants finds the top three bits of the
+// index (the seven boundaries at the eighth points of the table); the lower bits follow by
+// bisection in `tbn`, the shared-memory table of the boundaries held as -2^30 t: one load,
+// one saturated multiply-add and one (packed) multiply-add per level.
 template <int W>
 __device__ __forceinline__ void fma_magnitude_pair(float az0, float az1, const TreePairs& tp, uint32_t& m0, uint32_t& m1,
-                                                   u64& root)
+                                                   u64& root, const float* tbn = nullptr)
 {
-    static_assert(W >= 2 && W <= 4, "search trees of one to three levels");
+    static_assert(W >= 2 && W <= 8, "code widths of the Lloyd-Max tables");
     const u64 ir = pack2(fma_sat(az0, tp.big, tp.k_root), fma_sat(az1, tp.big, tp.k_root));
     root = ir;
     u64 m = ir;                                       // Horner form of 4 i_root + 2 i_1 + i_0
@@ -665,14 +642,27 @@ __device__ __forceinline__ void fma_magnitude_pair(float az0, float az1, const T
         unpack2(fma2_rz(ir, tp.a1, tp.b1), t0, t1);
         const u64 i1 = pack2(fma_sat(az0, tp.big, t0), fma_sat(az1, tp.big, t1));
         m = fma2(m, tp.two, i1);
-        if (W == 4) {
+        if (W >= 4) {
             unpack2(fma2_rz(i1, fma2_rz(ir, tp.da, tp.a_lo), fma2_rz(ir, tp.db, tp.b_lo)), t0, t1);
             const u64 i0 = pack2(fma_sat(az0, tp.big, t0), fma_sat(az1, tp.big, t1));
             m = fma2(m, tp.two, i0);
         }
     }
     float f0, f1;
-    unpack2(mul2(m, tp.w1), f0, f1);                  // times 2^-149 (W = 4: 2^-147): the bit pattern is the integer
+    m = mul2(m, tp.w1);                               // times a subnormal unit: the bit pattern is the integer
+    if constexpr (W >= 5) {
+        const char* base = reinterpret_cast<const char*>(tbn);
+#pragma unroll
+        for (int step = 1 << (W - 5); step >= 1; step >>= 1) {
+            unpack2(m, f0, f1);
+            const float b0 = *reinterpret_cast<const float*>(base + __float_as_uint(f0) + 4 * (step - 1));
+            const float b1 = *reinterpret_cast<const float*>(base + __float_as_uint(f1) + 4 * (step - 1));
+            const u64 i = pack2(fma_sat(az0, tp.big, b0), fma_sat(az1, tp.big, b1));
+            const float w = __uint_as_float(4u * (uint32_t)step);
+            m = fma2(i, pack2(w, w), m);
+        }
+    }
+    unpack2(m, f0, f1);
     m0 = __float_as_uint(f0);
     m1 = __float_as_uint(f1);
 }
@@ -710,8 +700,7 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
         constexpr int per = 32 / W;
         constexpr uint32_t lsb = W == 2 ? 0x55555555u : W == 4 ? 0x11111111u : 0x01010101u;
         static_assert(W == 2 || W == 4 || W == 8, "field widths that divide 32");
-        TreePairs tp;
-        if constexpr (W <= 4) tp = load_tree_pairs<W>();
+        const TreePairs tp = load_tree_pairs<W>();
         const u64 value_low2 = pack2(c_tree[2].v0, c_tree[2].v0), value_step2 = pack2(c_tree[2].dv, c_tree[2].dv);
         u64 dot2 = 0ull;
 #pragma unroll
@@ -728,25 +717,19 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
                 uint32_t m0, m1;
                 float q0, q1;
                 u64 root = 0ull;
-                if constexpr (W <= 4) {
-                    fma_magnitude_pair<W>(az0, az1, tp, m0, m1, root);
-                } else {
-                    m0 = (uint32_t)fast_magnitude<W>(az0, s_tb);
-                    m1 = (uint32_t)fast_magnitude<W>(az1, s_tb);
-                }
+                fma_magnitude_pair<W>(az0, az1, tp, m0, m1, root, s_tb);
                 if constexpr (W == 2) {
                     // two values: the smaller plus the indicator times their distance (the sum may
                     // miss the larger value by one unit in the last place, far inside the scale's tolerance)
                     dot2 = fma2(pack2(az0, az1), fma2(root, value_step2, value_low2), dot2);
                 } else {
-                    if constexpr (W == 4) {
-                        q0 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_tv) + m0);
-                        q1 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_tv) + m1);
-                    } else {
-                        q0 = s_tv[m0];
-                        q1 = s_tv[m1];
-                    }
+                    q0 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_tv) + m0);
+                    q1 = *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_tv) + m1);
                     dot2 = fma2(pack2(az0, az1), pack2(q0, q1), dot2);
+                    if constexpr (W == 8) {            // the fields take the index itself
+                        m0 >>= 2;
+                        m1 >>= 2;
+                    }
                 }
                 // sums, not ORs: the compiler cannot know that an index fits its field
                 if (W == 4 && i >= per / 2) fields_hi = (fields_hi * 16u + m1) * 16u + m0;
@@ -764,8 +747,7 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
     } else {
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = 0u;
-    TreePairs tp;
-    if constexpr (W <= 4) tp = load_tree_pairs<W>();
+    const TreePairs tp = load_tree_pairs<W>();
     // coordinates in descending order
 #pragma unroll
     for (int k = 15; k >= 0; --k) {
@@ -773,19 +755,19 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
         unpack2(v[k], h[0], h[1]);
         const float az2[2] = {fabsf(h[0]) * inv_norm, fabsf(h[1]) * inv_norm};
         uint32_t m2[2];
-        if constexpr (W <= 4) {
-            u64 root;
-            fma_magnitude_pair<W>(az2[0], az2[1], tp, m2[0], m2[1], root);
-        } else {
-            m2[0] = (uint32_t)fast_magnitude<W>(az2[0], s_tb);
-            m2[1] = (uint32_t)fast_magnitude<W>(az2[1], s_tb);
-        }
+        u64 root;
+        fma_magnitude_pair<W>(az2[0], az2[1], tp, m2[0], m2[1], root, s_tb);
 #pragma unroll
         for (int e = 1; e >= 0; --e) {
             const int l = 2 * k + e;
             const float az = az2[e];
-            const uint32_t m = m2[e];
-            dot = fmaf(az, s_tv[m], dot);
+            uint32_t m = m2[e];
+            if constexpr (W >= 4) {                    // the search returned the byte offset 4 m
+                dot = fmaf(az, *reinterpret_cast<const float*>(reinterpret_cast<const char*>(s_tv) + m), dot);
+                m >>= 2;
+            } else {
+                dot = fmaf(az, s_tv[m], dot);
+            }
             // code = half + m for z >= 0 and half - 1 - m otherwise: set the top bit, then
             // flip all W bits where the sign bit of z (that of h) is set
             const uint32_t flip = (uint32_t)((int)__float_as_uint(h[e]) >> 31) & (2u * half - 1u);
@@ -920,8 +902,9 @@ struct EncTables {
     __device__ __forceinline__ void fill(int t)
     {
         constexpr int half = 1 << (W - 1);
+        // integer budgets search with saturated multiply-adds: boundaries are held as -2^30 t
         for (int j = t; j < half; j += kFastThreads) {
-            tb[j] = c_pos_boundary[table_offset(W) + j];
+            tb[j] = (FRAC ? 1.f : -1073741824.f) * c_pos_boundary[table_offset(W) + j];
             tv[j] = c_pos_value[table_offset(W) + j];
         }
         if (FRAC)

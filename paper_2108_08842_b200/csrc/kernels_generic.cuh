@@ -80,8 +80,9 @@ __constant__ float c_pos_value[256];
 
 __device__ __forceinline__ int table_offset(int W) { return (1 << (W - 1)) - 1; }
 
-// The interval search of Section 2.2.1 for code widths 2..4 as arithmetic on the
-// multiply-add pipe (see fma_magnitude in kernels_fast.cuh).  A boundary t is held as
+// The interval search of Section 2.2.1 as arithmetic on the multiply-add pipe (see
+// fma_magnitude_pair in kernels_fast.cuh); for code widths above 4 the tree covers the
+// seven boundaries at the eighth points of the table.  A boundary t is held as
 // -2^30 t; `a*`/`d*` are differences of such values, chosen on the host so that the
 // multiply-adds below (rounded towards zero) land exactly on the fp32 boundaries.
 struct FmaTree {
@@ -92,7 +93,7 @@ struct FmaTree {
     float v0, dv;                // W = 2: the smaller positive value and the step to the larger
     float pad[6];
 };
-__constant__ FmaTree c_tree[5];  // by code width
+__constant__ FmaTree c_tree[9];  // by code width
 
 // Interval rule of Section 2.2.1 on one normalised coordinate: magnitude index m =
 // number of positive boundaries strictly below |z| (an endpoint belongs to the interval
