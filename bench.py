@@ -258,6 +258,10 @@ def run_gpu(args):
         masks_np = [work.recv_mask(c, eden.num_packets(d, float(bits[c]))) for c in range(n)]
         masks_gpu = [torch.from_numpy(m.view(np.int32)).to(dev) for m in masks_np]
     ctx = eden.Context(local_rank, d_max=d, n_batch=n, host_staging=True)
+    if args.slab_mib:
+        ctx.set_option(eden.OPT_SLAB_MIB, args.slab_mib)
+        ctx.set_option(eden.OPT_SLAB_STREAMS, args.slab_streams)
+        ctx.set_option(eden.OPT_SLAB_SIDES, args.slab_sides)
     scales = torch.empty(n, dtype=torch.float32, device=dev)
     mean = torch.empty(d, dtype=torch.float32, device=dev)
     uniform = args.uniform_bits is not None
@@ -311,7 +315,7 @@ def run_gpu(args):
     sampler.start()
     time.sleep(0.3)
     launches0 = ctx.launch_count
-    ctx.profile(True)
+    ctx.profile(not args.no_kernel_events)
     e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
     enc_ms = dec_ms = 0.0
     barrier()
@@ -325,7 +329,7 @@ def run_gpu(args):
         c.record()
         t_events.append((a, b, c))
     barrier()
-    kernels = ctx.profile_collect()
+    kernels = ctx.profile_collect() if not args.no_kernel_events else {}
     ctx.profile(False)
     launches = ctx.launch_count - launches0
     clocks = sampler.stop()
@@ -343,17 +347,19 @@ def run_gpu(args):
     # ---- roofline of the dominant kernel (by event time inside the timed region)
     peak, peak_kind = measured_hbm_peak()
     traffic_table = ncu_dram_bytes_per_coord()
-    top_name = max(kernels, key=lambda k: kernels[k]["ms"])
-    top = kernels[top_name]
-    achieved = top["bytes"] / top["launches"] / (top["ms"] / top["launches"] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": top_name, "achieved": achieved, "peak": peak,
-                "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": (traffic_table[top_name] * n * float(eden.rot_dim(d, float(bits[0])))
-                            if top_name in traffic_table and len(set(map(float, bits))) == 1 else None),
-                "traffic_source": "ncu dram__bytes_read+write, one client, scaled by clients per launch "
-                                  "(profiles/ncu_dram_traffic.txt; null if the kernels changed since the capture)",
-                "algorithmic_bytes_per_launch": top["bytes"] / top["launches"],
-                "ms_per_launch": top["ms"] / top["launches"]}
+    roofline = None
+    if kernels:
+        top_name = max(kernels, key=lambda k: kernels[k]["ms"])
+        top = kernels[top_name]
+        achieved = top["bytes"] / top["launches"] / (top["ms"] / top["launches"] * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": top_name, "achieved": achieved, "peak": peak,
+                    "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": (traffic_table[top_name] * n * float(eden.rot_dim(d, float(bits[0])))
+                                if top_name in traffic_table and len(set(map(float, bits))) == 1 else None),
+                    "traffic_source": "ncu dram__bytes_read+write, one client, scaled by clients per launch "
+                                      "(profiles/ncu_dram_traffic.txt; null if the kernels changed since the capture)",
+                    "algorithmic_bytes_per_launch": top["bytes"] / top["launches"],
+                    "ms_per_launch": top["ms"] / top["launches"]}
     kernel_table = {k: {"launches": v["launches"], "ms": round(v["ms"], 4),
                         "share": round(v["ms"] / sum(x["ms"] for x in kernels.values()), 4),
                         "algo_GBps": round(v["bytes"] / (v["ms"] * 1e-3) / 1e9, 1) if v["ms"] > 0 else None}
@@ -516,6 +522,12 @@ def main():
     ap.add_argument("--uniform-bits", type=float, default=None,
                     help="use the uniform-interval family (Section 4.3) at this entropy budget instead of the "
                          "Lloyd-Max tables; device-resident timing only (no end-to-end or CPU leg)")
+    ap.add_argument("--no-kernel-events", action="store_true",
+                    help="experiment: no per-kernel event bracketing in the timed region (no kernel table, no roofline)")
+    ap.add_argument("--slab-streams", type=int, default=1)
+    ap.add_argument("--slab-sides", type=int, default=3)
+    ap.add_argument("--slab-mib", type=int, default=0,
+                    help="experiment: launch the middle and row passes slab by slab (MiB of intermediate per slab)")
     ap.add_argument("--sweep", action="store_true",
                     help="print the LogNormal sweep table (d = 2^10 ... by powers of four, b = 1..8) instead of the JSON line")
     ap.add_argument("--sweep-max-log2", type=int, default=26)

@@ -339,10 +339,19 @@ int eden_force_generic_kernels(eden_ctx* ctx, int on);
  *                          tiles are staged in shared memory by bulk asynchronous copies.
  *   EDEN_OPT_SEL_ROUNDS    2 (default): the threshold of a b < 1 mask is found in two passes
  *                          over the keys where the candidate list holds them; 3: always in
- *                          three histogram rounds (the form very long vectors use). */
+ *                          three histogram rounds (the form very long vectors use).
+ *   EDEN_OPT_SLAB_MIB      0 (default): every pass of the transform is one launch over all
+ *                          clients of a group; m > 0: vectors that take three sweeps run
+ *                          their middle and last (receiver: first and middle) pass slab by
+ *                          slab, m MiB of intermediate per slab, so that the second pass
+ *                          of a slab may find the first one's output in the L2 cache. */
 #define EDEN_OPT_PLAN_VARIANT 1
 #define EDEN_OPT_ROW_STAGING  2
 #define EDEN_OPT_SEL_ROUNDS   3
+#define EDEN_OPT_SLAB_MIB     4
+#define EDEN_OPT_SLAB_SIDES   6   /* 1: sender only, 2: receiver only, 3 (default): both */
+#define EDEN_OPT_SLAB_STREAMS 5   /* 1 (default)..4: slabs are dealt round-robin to this many streams, so that
+                                     one slab's second pass can overlap the next slab's first */
 int eden_set_option(eden_ctx* ctx, int option, int value);
 
 /* Optional per-kernel timing for benchmarks: while enabled, every kernel launch is

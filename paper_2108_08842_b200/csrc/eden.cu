@@ -321,6 +321,11 @@ struct eden_ctx {
     int plan_variant;
     int row_staging;                 // 1: the sender's row pass runs in its persistent, bulk-copy-staged form
     int sel_rounds;                  // 3: the b < 1 mask threshold is found in three histogram rounds at every size
+    int slab_mib;                    // > 0: middle and row pass are launched slab by slab (MiB of intermediate per slab)
+    int slab_streams;                // slabs are dealt round-robin to this many streams (1 = the context's own)
+    int slab_sides;                  // bit 0: the sender uses the slab order, bit 1: the receiver
+    std::vector<cudaStream_t> side;  // side streams of the slab order
+    std::vector<cudaEvent_t> slab_events;   // fork (0) and join (1 + stream) events of the slab order
     int sm_count;
     std::vector<ProfileRecord> records;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> event_pool;
@@ -397,6 +402,9 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->plan_variant = 0;
     ctx->row_staging = 0;
     ctx->sel_rounds = 2;
+    ctx->slab_mib = 0;
+    ctx->slab_streams = 1;
+    ctx->slab_sides = 3;
     ctx->sm_count = 0;
     if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, cuda_device) != cudaSuccess ||
         ctx->sm_count <= 0) {
@@ -428,6 +436,8 @@ extern "C" int eden_destroy(eden_ctx* ctx)
         cudaEventDestroy(e.second);
     }
     for (cudaEvent_t e : ctx->sync_events) cudaEventDestroy(e);
+    for (cudaStream_t st : ctx->side) cudaStreamDestroy(st);
+    for (cudaEvent_t e : ctx->slab_events) cudaEventDestroy(e);
     if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
     if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     delete ctx;
@@ -458,6 +468,18 @@ extern "C" int eden_set_option(eden_ctx* ctx, int option, int value)
         case EDEN_OPT_SEL_ROUNDS:
             if (value != 2 && value != 3) return EDEN_ERR_INVALID_ARG;
             ctx->sel_rounds = value;
+            return EDEN_OK;
+        case EDEN_OPT_SLAB_MIB:
+            if (value < 0 || value > 4096) return EDEN_ERR_INVALID_ARG;
+            ctx->slab_mib = value;
+            return EDEN_OK;
+        case EDEN_OPT_SLAB_SIDES:
+            if (value < 1 || value > 3) return EDEN_ERR_INVALID_ARG;
+            ctx->slab_sides = value;
+            return EDEN_OK;
+        case EDEN_OPT_SLAB_STREAMS:
+            if (value < 1 || value > 4) return EDEN_ERR_INVALID_ARG;
+            ctx->slab_streams = value;
             return EDEN_OK;
         default:
             return EDEN_ERR_INVALID_ARG;
@@ -878,6 +900,43 @@ int resident_blocks(const eden_ctx* ctx, K kernel, uint32_t dynamic_smem)
     return cache[key] = per_sm * ctx->sm_count;
 }
 
+// Slab order on several streams: the slabs are independent, so they are dealt round-robin
+// to side streams that fork from the context's stream and join it again; the launch macros
+// follow ctx->stream, which SlabStreams points at the stream of the current slab.
+struct SlabStreams {
+    eden_ctx* ctx;
+    cudaStream_t main;
+    int n;
+    bool ok;
+    explicit SlabStreams(eden_ctx* c) : ctx(c), main(c->stream), n(c->slab_streams), ok(true)
+    {
+        if (n <= 1) return;
+        while ((int)ctx->side.size() < n && ok) {
+            cudaStream_t st;
+            ok = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) == cudaSuccess;
+            if (ok) ctx->side.push_back(st);
+        }
+        while (ctx->slab_events.size() < (size_t)n + 1 && ok) {
+            cudaEvent_t e;
+            ok = cudaEventCreateWithFlags(&e, cudaEventDisableTiming) == cudaSuccess;
+            if (ok) ctx->slab_events.push_back(e);
+        }
+        if (!ok) return;
+        ok = cudaEventRecord(ctx->slab_events[0], main) == cudaSuccess;
+        for (int j = 0; j < n && ok; ++j) ok = cudaStreamWaitEvent(ctx->side[j], ctx->slab_events[0], 0) == cudaSuccess;
+    }
+    void use(unsigned slab) { if (n > 1 && ok) ctx->stream = ctx->side[slab % (unsigned)n]; }
+    ~SlabStreams()
+    {
+        ctx->stream = main;
+        if (n <= 1 || !ok) return;
+        for (int j = 0; j < n; ++j) {
+            cudaEventRecord(ctx->slab_events[1 + j], ctx->side[j]);
+            cudaStreamWaitEvent(main, ctx->slab_events[1 + j], 0);
+        }
+    }
+};
+
 // Sender passes of one group on the register-blocked path.
 // `h_descs`: the host copy of the group's descriptors (d_descs is the same array on the device).
 int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g, const ClientDesc* h_descs,
@@ -888,30 +947,66 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     const unsigned tiles = (unsigned)((1ull << g.L) >> kFastTileLog);
     // the uniform-interval family has no cluster form of the row pass
     const FastPlan pl = fast_plan(g.L, g.uniform ? 0 : ctx->plan_variant);
+    // Slab order (EDEN_OPT_SLAB_MIB, three-sweep plans without clusters): after the top pass
+    // the sub-vectors of 2^(13 + middle bits) coordinates are independent, so the middle and
+    // the row pass can run slab by slab (some sub-vectors of some clients at a time), the row
+    // pass reading what the middle pass has just written while it may still be in L2.
+    const bool slabs = ctx->slab_mib > 0 && (ctx->slab_sides & 1) && pl.cols.size() == 2 && pl.row_lc == 0 &&
+                       pl.cols[0].lc == 0 && pl.cols[1].lc == 0 && !g.uniform && !ctx->row_staging;
+    std::vector<WidthRun> runs;
+    width_runs(plan, g, runs);
+    for (const WidthRun& r : runs)
+        // the row pass addresses client j of the run at work0 + j * 2^L
+        for (uint32_t j = 0; j < r.count; ++j)
+            if (h_descs[r.first + j].work != h_descs[r.first].work + ((uint64_t)j << g.L)) return EDEN_ERR_INVALID_ARG;
     for (size_t pi = 0; pi < pl.cols.size(); ++pi) {
         const FastPass& ps = pl.cols[pi];
         if (pi == 0) {
             EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
                 LAUNCH_CL(ctx, "f_enc_first", gn * (4.0 * std::min<double>((double)d, D) + 4.0 * D),
                           (k_f_col<LR_, LC_, true>), dim3(tiles, gn), dim3(kFastThreads), ps.lc,
-                          (const ClientDesc*)d_descs, d_states, ps.lo, 0)));
-        } else {
+                          (const ClientDesc*)d_descs, d_states, ps.lo, 0, 0u)));
+        } else if (!slabs) {
             EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
                 LAUNCH_CL(ctx, "f_mid", gn * 8.0 * D, (k_f_col<LR_, LC_, false>), dim3(tiles, gn),
-                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo, 1)));
+                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo, 1, 0u)));
         }
     }
     const int inv_ready = pl.cols.size() >= 2 ? 1 : 0;     // a middle pass has left 1/||y|| in the client's state
-    std::vector<WidthRun> runs;
-    width_runs(plan, g, runs);
+    if (slabs) {
+        const FastPass& ps = pl.cols[1];
+        const unsigned sub_tiles = 1u << ps.lr;                         // tiles of one independent sub-vector
+        const uint64_t sub_mib = ((uint64_t)sub_tiles << kFastTileLog) * 4 >> 20;
+        SlabStreams fork(ctx);
+        if (!fork.ok) return EDEN_ERR_CUDA;
+        unsigned slab = 0;
+        for (const WidthRun& r : runs) {
+            const uint32_t cl = (uint32_t)std::min<uint64_t>(r.count, std::max<uint64_t>(1, ctx->slab_mib / std::max<uint64_t>(1, sub_mib)));
+            const unsigned subs = (unsigned)std::max<uint64_t>(1, ctx->slab_mib / std::max<uint64_t>(1, sub_mib * cl));
+            for (uint32_t c0 = 0; c0 < r.count; c0 += cl) {
+                const uint32_t cn = std::min(cl, r.count - c0);
+                const ClientDesc* dd = d_descs + r.first + c0;
+                ClientState* ds = d_states + r.first + c0;
+                for (unsigned t0 = 0; t0 < tiles; t0 += subs * sub_tiles) {
+                    const unsigned tn = std::min(subs * sub_tiles, tiles - t0);
+                    fork.use(slab++);
+                    EDEN_DISPATCH_LR(ps.lr,
+                        LAUNCH_CL(ctx, "f_mid", cn * 8.0 * 8192.0 * tn, (k_f_col<LR_, 0, false>), dim3(tn, cn),
+                                  dim3(kFastThreads), 0, dd, ds, ps.lo, 1, t0));
+                    EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_W(r.W,
+                        LAUNCH_CL(ctx, "f_enc_last", cn * (4.0 + r.W / 8.0) * 8192.0 * tn, (k_f_enc_last<W_, 0, FRAC_>),
+                                  dim3(tn, cn), dim3(kFastThreads), 0, dd, ds,
+                                  (const float*)h_descs[r.first + c0].work, g.L, inv_ready, t0)));
+                }
+            }
+        }
+        return EDEN_OK;
+    }
     for (const WidthRun& r : runs) {
-        // the row pass addresses client j of the run at work0 + j * 2^L
-        for (uint32_t j = 0; j < r.count; ++j)
-            if (h_descs[r.first + j].work != h_descs[r.first].work + ((uint64_t)j << g.L)) return EDEN_ERR_INVALID_ARG;
         if (g.uniform) {
             LAUNCH(ctx, "f_enc_last", r.count * 5.0 * D, (k_f_enc_last<8, 0, false, true>), dim3(tiles, r.count),
                    kFastThreads, 0, (const ClientDesc*)(d_descs + r.first), d_states + r.first,
-                   (const float*)h_descs[r.first].work, g.L, inv_ready);
+                   (const float*)h_descs[r.first].work, g.L, inv_ready, 0u);
             continue;
         }
         if (ctx->row_staging && pl.row_lc == 0) {
@@ -931,7 +1026,7 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
             LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_, FRAC_>),
                       dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
                       (const ClientDesc*)(d_descs + r.first), d_states + r.first,
-                      (const float*)h_descs[r.first].work, g.L, inv_ready))));
+                      (const float*)h_descs[r.first].work, g.L, inv_ready, 0u))));
     }
     return EDEN_OK;
 }
@@ -948,19 +1043,50 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     const FastPlan pl = fast_plan(g.L, ctx->plan_variant);
     std::vector<WidthRun> runs;
     width_runs(plan, g, runs);
-    for (const WidthRun& r : runs) {
-        EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
-            LAUNCH_CL(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, (k_f_dec_first<W_, LC_, FRAC_>),
-                      dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
-                      (const ClientDesc*)(d_descs + r.first)))));
+    // slab order as on the sender (EDEN_OPT_SLAB_MIB): row pass, then middle pass, slab by slab
+    const bool slabs = ctx->slab_mib > 0 && (ctx->slab_sides & 2) && pl.cols.size() == 2 && pl.row_lc == 0 &&
+                       pl.cols[0].lc == 0 && pl.cols[1].lc == 0;
+    if (slabs) {
+        const FastPass& ps = pl.cols[1];
+        const unsigned sub_tiles = 1u << ps.lr;
+        const uint64_t sub_mib = ((uint64_t)sub_tiles << kFastTileLog) * 4 >> 20;
+        SlabStreams fork(ctx);
+        if (!fork.ok) return EDEN_ERR_CUDA;
+        unsigned slab = 0;
+        for (const WidthRun& r : runs) {
+            const uint32_t cl = (uint32_t)std::min<uint64_t>(r.count, std::max<uint64_t>(1, ctx->slab_mib / std::max<uint64_t>(1, sub_mib)));
+            const unsigned subs = (unsigned)std::max<uint64_t>(1, ctx->slab_mib / std::max<uint64_t>(1, sub_mib * cl));
+            for (uint32_t c0 = 0; c0 < r.count; c0 += cl) {
+                const uint32_t cn = std::min(cl, r.count - c0);
+                const ClientDesc* dd = d_descs + r.first + c0;
+                for (unsigned t0 = 0; t0 < tiles; t0 += subs * sub_tiles) {
+                    const unsigned tn = std::min(subs * sub_tiles, tiles - t0);
+                    fork.use(slab++);
+                    EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_W(r.W,
+                        LAUNCH_CL(ctx, "f_dec_first", cn * (4.0 + r.W / 8.0) * 8192.0 * tn, (k_f_dec_first<W_, 0, FRAC_>),
+                                  dim3(tn, cn), dim3(kFastThreads), 0, dd, t0)));
+                    EDEN_DISPATCH_LR(ps.lr,
+                        LAUNCH_CL(ctx, "f_mid", cn * 8.0 * 8192.0 * tn, (k_f_col<LR_, 0, false>), dim3(tn, cn),
+                                  dim3(kFastThreads), 0, dd, d_states + r.first + c0, ps.lo, 0, t0));
+                }
+            }
+        }
+    } else {
+        for (const WidthRun& r : runs) {
+            EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
+                LAUNCH_CL(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, (k_f_dec_first<W_, LC_, FRAC_>),
+                          dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
+                          (const ClientDesc*)(d_descs + r.first), 0u))));
+        }
     }
     // the receiver walks the column ranges bottom-up so that the top range comes last
     for (size_t pi = pl.cols.size(); pi-- > 0;) {
         const FastPass& ps = pl.cols[pi];
         if (pi > 0) {
+            if (slabs) continue;
             EDEN_DISPATCH_LC(ps.lc, EDEN_DISPATCH_LR(ps.lr,
                 LAUNCH_CL(ctx, "f_mid", gn * 8.0 * D, (k_f_col<LR_, LC_, false>), dim3(tiles, gn),
-                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo, 0)));
+                          dim3(kFastThreads), ps.lc, (const ClientDesc*)d_descs, d_states, ps.lo, 0, 0u)));
         } else {
             // A round with few tiles leaves most SMs idle if every block walks all clients:
             // split the clients over block rows, each row summing into a partial vector of

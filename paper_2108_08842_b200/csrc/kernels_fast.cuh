@@ -311,13 +311,14 @@ __device__ __forceinline__ void col_cluster_stage(u64 (&v)[16], ulonglong2* s, c
 // =================================================================================
 template <int LR, int LC, bool FIRST>
 __global__ void __launch_bounds__(kFastThreads, 4)
-k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo, int publish_inv)
+k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, int lo, int publish_inv,
+        uint32_t tile0 /* first tile of this launch (launches that cover a slab of the vector) */)
 {
     __shared__ ulonglong2 s[2048];
     __shared__ uint32_t s_sign[256];
     __shared__ double red[32];
     const ClientDesc cd = descs[blockIdx.y];
-    const ColTile ct = col_tile<LR, LC>(blockIdx.x, lo);
+    const ColTile ct = col_tile<LR, LC>(blockIdx.x + tile0, lo);
     const int t = threadIdx.x;
     const float* __restrict__ src = FIRST ? cd.src : cd.work;
     if (FIRST) col_sign_words<LR>(cd.seed, ct, s_sign);
@@ -337,7 +338,7 @@ k_f_col(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, 
             v[2 * k + 1] = pack2(x2, 0.f);
         }
     }
-    if (!FIRST && publish_inv && blockIdx.x == 0 && t == 0) {
+    if (!FIRST && publish_inv && blockIdx.x + tile0 == 0 && t == 0) {
         // sender's middle pass: ||y||^2 is complete, so one thread per client leaves 1/||y||
         // (0 for a zero or non-finite vector) for the row pass, off every block's critical path
         const double n2 = states[blockIdx.y].norm2;
@@ -993,14 +994,14 @@ template <int W, int LC, bool FRAC, bool UNI = false>
 #endif
 __global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : EDEN_ENC_LAST_BLOCKS))
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L,
-             int inv_ready)
+             int inv_ready, uint32_t tile0)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ float s_warp_dot[kFastThreads / 32];
     __shared__ float s_inv;
     __shared__ EncTables<W, FRAC> tab;
     const int t = threadIdx.x;
-    const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
+    const uint64_t base = (uint64_t)(blockIdx.x + tile0) << kFastTileLog;
     u64 v[16];
     if (LC == 0) {
         const u64* __restrict__ src = reinterpret_cast<const u64*>(work0 + ((uint64_t)blockIdx.y << L) + base);
@@ -1169,7 +1170,7 @@ k_f_enc_last_staged(const ClientDesc* __restrict__ descs, ClientState* __restric
 // =================================================================================
 template <int W, int LC, bool FRAC>
 __global__ void __launch_bounds__(kFastThreads, 4)
-k_f_dec_first(const ClientDesc* __restrict__ descs)
+k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ float s_val[2 << W];                    // the 2^W values by code, then 2^W zeros
@@ -1195,7 +1196,7 @@ k_f_dec_first(const ClientDesc* __restrict__ descs)
             s_val0[j] = c;
         }
     __syncthreads();
-    const uint64_t base = (uint64_t)blockIdx.x << kFastTileLog;
+    const uint64_t base = (uint64_t)(blockIdx.x + tile0) << kFastTileLog;
     // the tile is 8 packets of 1024 coordinates; this thread's 32 coordinates lie in one.
     // A lost packet reads the zero half of the table (Section 4.2: lost coordinates are 0).
     const uint64_t pkt = (base >> 10) + (uint64_t)(t >> 5);

@@ -85,7 +85,7 @@ _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctyp
                                 ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
 
 STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA, STATUS_TIMEOUT, STATUS_SCRATCH = 1, 2, 4, 8, 16
-OPT_PLAN_VARIANT, OPT_ROW_STAGING, OPT_SEL_ROUNDS = 1, 2, 3
+OPT_PLAN_VARIANT, OPT_ROW_STAGING, OPT_SEL_ROUNDS, OPT_SLAB_MIB, OPT_SLAB_STREAMS, OPT_SLAB_SIDES = 1, 2, 3, 4, 5, 6
 PACKET_COORDS = 1024
 UNIFORM_MAX_INDEX = 127
 UNIFORM_MIN_DELTA = 0.0625

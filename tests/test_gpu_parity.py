@@ -169,6 +169,22 @@ def test_pass_plans_at_2_pow_24_and_25(E, variant):
         run_workload(E, work, options=[(E.OPT_PLAN_VARIANT, variant)])
 
 
+@pytest.mark.parametrize("slab_mib,streams,sides,bits", [(8, 1, 3, 4.0), (32, 2, 3, 1.0), (24, 3, 2, 2.5), (8, 4, 1, 2.0)])
+def test_middle_and_row_pass_launched_slab_by_slab(E, slab_mib, streams, sides, bits):
+    # three-sweep vectors (2^22 and more): the sub-vectors of 2^21 coordinates are independent
+    # after the top pass, so middle and row pass may be launched slab by slab (a ragged last
+    # slab of clients and of sub-vectors included); same messages, same mean
+    d, n = (1 << 23) - 11, 3
+    rng = np.random.default_rng(slab_mib)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(slab_mib, n), 0.05,
+                          lambda c: xs[c], slab_mib)
+    # the slabs may be dealt to several streams (one slab's second pass then overlaps the next
+    # slab's first) and the order may be used on one side only
+    run_workload(E, work, options=[(E.OPT_SLAB_MIB, slab_mib), (E.OPT_SLAB_STREAMS, streams),
+                                   (E.OPT_SLAB_SIDES, sides)])
+
+
 @pytest.mark.parametrize("bits", [1.0, 2.0, 4.0, 8.0, 2.5])
 def test_sender_row_pass_staged_by_bulk_copies(E, bits):
     # the persistent form of the sender's last pass (tiles staged in shared memory by bulk
