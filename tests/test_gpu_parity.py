@@ -220,6 +220,30 @@ def test_every_code_width(E, W):
     assert mism <= 8 * W
 
 
+def test_lognormal_sweep_point_meets_corollary_2_4(E):
+    # the paper's sweep law (LogNormal(0,1), Section 5.2) at d = 2^20: the GPU's own round
+    # trip (encode, then the mean of that one message) has vNMSE = 1 / E[Q^2] - 1 for every
+    # b = 1..8 (Corollary 2.4), within 3 % (one rotation: the O(sqrt(log d / d)) term and
+    # the draw's own noise)
+    from scipy.stats import norm
+    d = 1 << 20
+    work = synth.make("sweep", d=d, n=1)
+    xs = work.vectors()
+    x64 = xs[0].astype(np.float64)
+    ctx = _ctx(E, d, 1)
+    x_gpu = torch.from_numpy(xs).cuda()
+    for b in range(1, 9):
+        codes, scales = ctx.encode(x_gpu, [float(b)], work.seeds)
+        est = ctx.mean(codes, scales, [float(b)], work.seeds, d).cpu().numpy().astype(np.float64)
+        assert ctx.status() == 0
+        vnmse = np.sum((est - x64) ** 2) / np.sum(x64 ** 2)
+        c, t = O.table(b)
+        edges = np.concatenate(([-np.inf], t, [np.inf]))
+        limit = 1.0 / float(np.sum((norm.cdf(edges[1:]) - norm.cdf(edges[:-1])) * c * c)) - 1.0
+        assert abs(vnmse - limit) < 0.03 * limit, (b, vnmse, limit)
+    ctx.close()
+
+
 @pytest.mark.parametrize("bits,d", [(0.1, 1 << 16), (0.5, 3000), (0.25, 70001), (0.9, 9), (0.01, 50)])
 def test_sub_bit_budgets_and_mask(E, bits, d):
     n = 3
