@@ -24,8 +24,10 @@
  *     sparsification of Section 4.1), the integers 2..8 (Section 3) and non-integer
  *     1 < b < 8 (Section 4.1: each coordinate is coded with 2^(floor(b)+1) values if its
  *     shared coin is set, with 2^floor(b) otherwise; coins are Philox stream 2, call t
- *     giving eight 16-bit numbers for coordinates 8t..8t+7, set iff the number is below
- *     round((b - floor(b)) * 65536)).  Other values return EDEN_ERR_UNSUPPORTED_BITS.
+ *     giving sixteen 8-bit numbers (the bytes of its four words, low byte first) for
+ *     coordinates 16t..16t+15, set iff the number is below round((b - floor(b)) * 256),
+ *     so the share of wider codes is a multiple of 1/256).  Other values return
+ *     EDEN_ERR_UNSUPPORTED_BITS.
  *   - Rotation (Section 5): R = (1/sqrt D) H_D Diag(s), H_D the Sylvester-ordered
  *     Walsh-Hadamard matrix, D = 2^ceil(log2 d') with d' = d for b >= 1 and d' = the
  *     kept count k for b < 1; shorter vectors are zero-padded, all D coordinates are
@@ -40,9 +42,10 @@
  *     coordinates = 128*W bytes.  The scale S travels beside the codes as one fp32.
  *     Non-integer b: groups of 32 coordinates of W = floor(b)+1 words each: first the bit
  *     stream of floor(b)-bit fields (an unset coordinate's code, or the upper bits of a
- *     set coordinate's code), then one word with the lowest code bit of the set
- *     coordinates packed in order from bit 0.  Only floor(b)*32 + (coins set) bits of a
- *     group carry information; the padding keeps packets at 128*W bytes.
+ *     set coordinate's code), then one word whose bit l is the lowest code bit of the
+ *     group's coordinate l if its coin is set, else 0.  Only floor(b)*32 + (coins set) bits
+ *     of a group carry information (both sides know the coins); whole words keep packets
+ *     at 128*W bytes.
  */
 #ifndef EDEN_H_
 #define EDEN_H_

@@ -134,7 +134,7 @@ def code_words(d: int, bits: float) -> int:
 
 
 def coin_threshold(bits: float) -> int:
-    """0 for integer and sub-bit budgets, else round(frac(b) * 65536)."""
+    """0 for integer and sub-bit budgets, else round(frac(b) * 256)."""
     return int(_L().eden_oracle_coin_threshold(float(bits)))
 
 

@@ -40,14 +40,16 @@
  *   - A packet is 1024 consecutive rotated coordinates.
  *   - Non-integer budgets b > 1 (Section 4.1): coordinate i is coded with 2^(floor(b)+1)
  *     values if its coin is set, else with 2^floor(b).  Coins are Philox stream 2:
- *     call t yields eight 16-bit numbers (low half of word 0, high half of word 0,
- *     low half of word 1, ...) for rotated coordinates 8t..8t+7; the coin is set iff
- *     the number is below round((b - floor(b)) * 65536).              [stream layout unpinned]
+ *     call t yields sixteen 8-bit numbers (the bytes of word 0 from the low one up,
+ *     then those of word 1, ...) for rotated coordinates 16t..16t+15; the coin is set
+ *     iff the number is below round((b - floor(b)) * 256).            [stream layout unpinned]
  *     Wire layout for such b: groups of 32 coordinates, floor(b)+1 words each: first a
  *     bit stream of floor(b)-bit fields (the code of an unset coordinate, or the
- *     upper floor(b) bits of a set coordinate's code), then one word holding the lowest
- *     code bit of the set coordinates, packed in coordinate order from bit 0.
- *     Only floor(b)*32 + (number of coins) bits of a group are meaningful.  [layout unpinned]
+ *     upper floor(b) bits of a set coordinate's code), then one word whose bit l is the
+ *     lowest code bit of coordinate l of the group if its coin is set, else 0.
+ *     Only floor(b)*32 + (number of coins) bits of a group carry information (both
+ *     sides know the coins); the group keeps whole words so that packets keep
+ *     their size.                                                      [layout unpinned]
  *   - Section 4.3's uniform-interval family I_Delta (functions *_uniform_* at the end):
  *     index n = round(z / Delta), an endpoint going to the interval nearer zero like
  *     everywhere else; indices are clamped to +-127, i.e. the family is made finite by
@@ -145,13 +147,13 @@ uint32_t eden_oracle_code_width(double bits)
     return (uint32_t)floor(bits) + 1u;
 }
 
-/* 0 for an integer (or sub-bit) budget, else the coin threshold round(frac * 65536) */
+/* 0 for an integer (or sub-bit) budget, else the coin threshold round(frac * 256) in 1..255 */
 uint32_t eden_oracle_coin_threshold(double bits)
 {
     if (bits <= 1.0 || bits == floor(bits)) return 0u;
-    uint32_t t = (uint32_t)floor((bits - floor(bits)) * 65536.0 + 0.5);
+    uint32_t t = (uint32_t)floor((bits - floor(bits)) * 256.0 + 0.5);
     if (t < 1u) t = 1u;
-    if (t > 65535u) t = 65535u;
+    if (t > 255u) t = 255u;
     return t;
 }
 
@@ -159,10 +161,10 @@ uint32_t eden_oracle_coin_threshold(double bits)
 int eden_oracle_coin(uint64_t seed, uint64_t i, uint32_t threshold)
 {
     uint32_t w[4];
-    philox_stream(seed, 2u, i / 8u, w);
-    uint32_t word = w[(i % 8u) / 2u];
-    uint32_t half = (i % 2u) ? (word >> 16) : (word & 0xFFFFu);
-    return half < threshold;
+    philox_stream(seed, 2u, i / 16u, w);
+    uint32_t word = w[(i % 16u) / 4u];
+    uint32_t byte = (word >> (8u * (uint32_t)(i % 4u))) & 0xFFu;
+    return byte < threshold;
 }
 
 /* words of one client's message */
@@ -406,7 +408,6 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
     /* steps 4-6: z = eta r with eta = sqrt(D)/||y||, code, dot <r, Q(z)> */
     double eta = sqrt((double)D) / sqrt(N2);
     double dot = 0.0;
-    uint32_t extra_pos = 0;                        /* next free bit of the group's extra word */
     for (uint64_t i = 0; i < D; ++i) {
         double z = eta * y[i];
         if (!coin_thr) {
@@ -420,7 +421,6 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
             /* non-integer budget: 2^(W0+1) values if the coin is set, else 2^W0 */
             uint64_t g = i / 32u, l = i % 32u;
             uint32_t *grp = codes + g * W;
-            if (l == 0) extra_pos = 0;
             int coin = eden_oracle_coin(seed, i, coin_thr);
             uint32_t Wi = coin ? W0 + 1u : W0;
             uint32_t code = eden_oracle_quantise(z, Wi);
@@ -430,7 +430,7 @@ int eden_oracle_encode(const float *x, uint64_t d, double bits, uint64_t seed,
                 uint64_t b = l * W0 + j;
                 grp[b / 32u] |= ((field >> j) & 1u) << (b % 32u);
             }
-            if (coin) grp[W0] |= (code & 1u) << extra_pos++;
+            if (coin) grp[W0] |= (code & 1u) << l;
         }
         if (z_out) z_out[i] = z;
     }
@@ -465,18 +465,13 @@ int eden_oracle_decode(const uint32_t *codes, double S, double bits, uint64_t se
     if (!q) return -1;
 
     uint64_t received = 0;
-    uint32_t extra_pos = 0;
     for (uint64_t i = 0; i < D; ++i) {
         uint64_t pkt = i / EDEN_ORACLE_PACKET;
         int arrived = recv_mask ? (int)((recv_mask[pkt / 32u] >> (pkt % 32u)) & 1u) : 1;
         if (coin_thr) {
-            /* the position of a set coordinate's extra bit depends on the coins before it */
             uint64_t g = i / 32u, l = i % 32u;
             const uint32_t *grp = codes + g * W;
-            if (l == 0) extra_pos = 0;
             int coin = eden_oracle_coin(seed, i, coin_thr);
-            uint32_t my_pos = extra_pos;
-            if (coin) ++extra_pos;
             if (!arrived) continue;
             ++received;
             uint32_t field = 0;
@@ -484,7 +479,7 @@ int eden_oracle_decode(const uint32_t *codes, double S, double bits, uint64_t se
                 uint64_t b = l * W0 + j;
                 field |= ((grp[b / 32u] >> (b % 32u)) & 1u) << j;
             }
-            if (coin) q[i] = eden_oracle_value((field << 1) | ((grp[W0] >> my_pos) & 1u), W0 + 1u);
+            if (coin) q[i] = eden_oracle_value((field << 1) | ((grp[W0] >> l) & 1u), W0 + 1u);
             else q[i] = eden_oracle_value(field, W0);
             continue;
         }

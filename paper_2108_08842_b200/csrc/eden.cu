@@ -54,12 +54,12 @@ extern "C" uint32_t eden_code_width(double bits)
     return (uint32_t)std::floor(bits) + 1;     // non-integer: the wider of the two tables
 }
 
-// 0 for integer and sub-bit budgets, else round(frac(b) * 65536) clamped to [1, 65535]
+// 0 for integer and sub-bit budgets, else round(frac(b) * 256) clamped to [1, 255]
 static uint32_t coin_threshold(double bits)
 {
     if (bits <= 1.0 || bits == std::floor(bits)) return 0;
-    uint32_t t = (uint32_t)std::floor((bits - std::floor(bits)) * 65536.0 + 0.5);
-    return std::min(std::max(t, 1u), 65535u);
+    uint32_t t = (uint32_t)std::floor((bits - std::floor(bits)) * 256.0 + 0.5);
+    return std::min(std::max(t, 1u), 255u);
 }
 
 extern "C" uint64_t eden_code_bytes(uint64_t d, double bits)

@@ -20,7 +20,7 @@ struct ClientDesc {
     uint32_t L;              // log2 of the rotation dimension D
     uint32_t subbit;         // 1 if b < 1
     uint32_t index;          // position of this client in the caller's arrays
-    uint32_t coin_thr;       // non-integer b > 1: coin threshold round(frac * 65536); else 0
+    uint32_t coin_thr;       // non-integer b > 1: coin threshold round(frac * 256); else 0
     float delta;             // uniform-interval family (Section 4.3): interval width; else 0
     uint32_t recv_shift;     // log2 coordinates per bit of `recv`: 10 (packets), or 0 (one bit per coordinate, W = 1 only)
     uint32_t reserved;
@@ -82,15 +82,14 @@ __device__ __forceinline__ uint32_t sign_word(uint64_t seed, uint64_t g)
 
 // Coin of rotated coordinate i for a non-integer budget b > 1 (Section 4.1: the
 // coordinates that get the extra bit are picked by shared randomness): Philox stream 2,
-// call i/8 yields eight 16-bit numbers, coordinate i takes number i%8 (low half of word
-// 0, high half of word 0, ...); the coin is set iff the number is below the threshold.
+// call i/16 yields sixteen 8-bit numbers, coordinate i takes number i%16 (the bytes of word
+// 0 from the low one up, then word 1, ...); the coin is set iff the number is below the threshold.
 __device__ __forceinline__ bool coin_bit(uint64_t seed, uint64_t i, uint32_t threshold)
 {
-    const uint4 r = philox_stream(seed, 2u, i >> 3);
-    const uint32_t w = ((uint32_t)i >> 1) & 3u;
+    const uint4 r = philox_stream(seed, 2u, i >> 4);
+    const uint32_t w = ((uint32_t)i >> 2) & 3u;
     const uint32_t word = w == 0 ? r.x : w == 1 ? r.y : w == 2 ? r.z : r.w;
-    const uint32_t half = (i & 1u) ? word >> 16 : word & 0xFFFFu;
-    return half < threshold;
+    return ((word >> (8u * ((uint32_t)i & 3u))) & 0xFFu) < threshold;
 }
 
 // Uniform-interval family I_Delta (Section 4.3): magnitude index of |z| = the number of

@@ -624,6 +624,42 @@ __device__ __forceinline__ TreePairs load_tree_pairs()
     tp.w1 = pack2(__uint_as_float(unit), __uint_as_float(unit));
     return tp;
 }
+// One coordinate through the same search with the constants taken straight from constant
+// memory (no registers held): used where two tables are searched per coordinate
+// (non-integer budgets).  Returns the index itself.
+template <int W>
+__device__ __forceinline__ uint32_t fma_magnitude_one(float az, const float* tbn)
+{
+    static_assert(W >= 1 && W <= 8, "code widths of the Lloyd-Max tables");
+    if constexpr (W == 1) {
+        return 0u;
+    } else {
+        const FmaTree& tr = c_tree[W];
+        const float ir = fma_sat(az, tr.big, tr.k_root);
+        float m = ir;
+        if (W >= 3) {
+            const float i1 = fma_sat(az, tr.big, __fmaf_rz(ir, tr.a1, tr.b1));
+            m = fmaf(m, 2.f, i1);
+            if (W >= 4) {
+                const float t0 = __fmaf_rz(i1, __fmaf_rz(ir, tr.da, tr.a_lo), __fmaf_rz(ir, tr.db, tr.b_lo));
+                m = fmaf(m, 2.f, fma_sat(az, tr.big, t0));
+            }
+        }
+        // times a subnormal unit: the bit pattern is the integer (W >= 5: the byte offset of the octant)
+        m *= __uint_as_float(W >= 5 ? 4u << (W - 4) : 1u);
+        if constexpr (W >= 5) {
+            const char* base = reinterpret_cast<const char*>(tbn);
+#pragma unroll
+            for (int step = 1 << (W - 5); step >= 1; step >>= 1) {
+                const float b = *reinterpret_cast<const float*>(base + __float_as_uint(m) + 4 * (step - 1));
+                m = fmaf(fma_sat(az, tr.big, b), __uint_as_float(4u * (uint32_t)step), m);
+            }
+            return __float_as_uint(m) >> 2;
+        }
+        return __float_as_uint(m);
+    }
+}
+
 // `root`: the pair's indicators of the first level (for W = 2 they are the index itself)
 // Returns the magnitude indices (W <= 3) or four times them, the byte offsets into a table
 // of floats (W >= 4).  For W >= 5 the tree of constants finds the top three bits of the
@@ -789,27 +825,31 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
 
 // ---------------------------------------------------------------------------------
 // Non-integer budgets b > 1 (Section 4.1) on the row pass: the thread owns one group of 32
-// coordinates; W = floor(b) + 1 words per group: (W-1)-bit fields, then the lowest code
-// bit of the coordinates whose coin is set, packed in order.
+// coordinates; W = floor(b) + 1 words per group: (W-1)-bit fields, then one word whose bit l
+// is the lowest code bit of coordinate l if its coin is set.
 // ---------------------------------------------------------------------------------
-// coins of the 32 coordinates of group g: four Philox calls of eight 16-bit numbers each
+// coins of the 32 coordinates of group g: two Philox calls of sixteen 8-bit numbers each.
+// The four bytes of a word are compared with the threshold at once (one mask byte each) and
+// the four answers gathered into a nibble by one multiplication.
 __device__ __forceinline__ uint32_t group_coins(uint64_t seed, uint64_t g, uint32_t threshold)
 {
+    const uint32_t thr4 = threshold * 0x01010101u;
     uint32_t coins = 0u;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const uint4 r = philox_stream(seed, 2u, 4 * g + c);
+    for (int c = 0; c < 2; ++c) {
+        const uint4 r = philox_stream(seed, 2u, 2 * g + c);
         const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            coins |= ((w[j] & 0xFFFFu) < threshold ? 1u : 0u) << (8 * c + 2 * j);
-            coins |= ((w[j] >> 16) < threshold ? 1u : 0u) << (8 * c + 2 * j + 1);
+            const uint32_t lt = __vcmpltu4(w[j], thr4) & 0x01010101u;          // bit 8k: byte k is below the threshold
+            // bits 0, 8, 16, 24 -> bits 28..31 (the partial products below bit 28 cannot carry into them)
+            coins |= ((lt * 0x10204080u) >> 28) << (16 * c + 4 * j);
         }
     }
     return coins;
 }
 
-// tb_hi/tv_hi: positive boundaries and values of width W; tb_lo/tv_lo: of width W - 1
+// tb_hi/tv_hi: positive boundaries (held as -2^30 t) and values of width W; tb_lo/tv_lo: of width W - 1
 template <int W>
 __device__ __forceinline__ void quantise_pack_frac(const u64 (&v)[16], float inv_norm, bool live, uint32_t coins,
                                                    const float* tb_hi, const float* tv_hi,
@@ -819,7 +859,6 @@ __device__ __forceinline__ void quantise_pack_frac(const u64 (&v)[16], float inv
     constexpr int W0 = W - 1;
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = 0u;
-    uint32_t pos = 0u;
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
         float h[2];
@@ -828,33 +867,45 @@ __device__ __forceinline__ void quantise_pack_frac(const u64 (&v)[16], float inv
         for (int e = 0; e < 2; ++e) {
             const int l = 2 * k + e;
             const bool wide = (coins >> l) & 1u;
-            const int hw = wide ? (1 << W0) : (1 << W0) >> 1;       // half the number of values
-            const float* tb = wide ? tb_hi : tb_lo;
-            const float* tv = wide ? tv_hi : tv_lo;
-            const float z = h[e] * inv_norm;
-            const float az = fabsf(z);
-            int m = 0;
+            const uint32_t hw = wide ? (1u << W0) : (1u << W0) >> 1;   // half the number of values
+            const float az = fabsf(h[e]) * inv_norm;
+            uint32_t m;
+            if constexpr (W <= 3) {
+                // both tables are searched (a few multiply-adds, no branches); the coin picks the result
+                const uint32_t m_hi = fma_magnitude_one<W>(az, tb_hi), m_lo = fma_magnitude_one<W0>(az, tb_lo);
+                m = wide ? m_hi : m_lo;
+                dot = fmaf(az, wide ? tv_hi[m_hi] : tv_lo[m_lo], dot);
+            } else {
+                // one bisection in the coin's table (W0 levels for the wider table, the first of
+                // them idle for the narrower one): a load, a saturated multiply-add and a
+                // multiply-add per level, the index kept as a byte offset in a subnormal float
+                const char* tb = reinterpret_cast<const char*>(wide ? tb_hi : tb_lo);
+                const char* tv = reinterpret_cast<const char*>(wide ? tv_hi : tv_lo);
+                const float big = c_tree[2].big;
+                float mo = 0.f;
 #pragma unroll
-            for (int it = 0; it < W0; ++it) {
-                const int step = (1 << (W0 - 1)) >> it;
-                if (step < hw) m += (az > tb[m + step - 1]) ? step : 0;
+                for (int it = 0; it < W0; ++it) {
+                    const int step = (1 << (W0 - 1)) >> it;
+                    float ind = fma_sat(az, big, *reinterpret_cast<const float*>(tb + __float_as_uint(mo) + 4 * (step - 1)));
+                    if (it == 0) ind = wide ? ind : 0.f;
+                    mo = fmaf(ind, __uint_as_float(4u * (uint32_t)step), mo);
+                }
+                dot = fmaf(az, *reinterpret_cast<const float*>(tv + __float_as_uint(mo)), dot);
+                m = __float_as_uint(mo) >> 2;
             }
-            dot = fmaf(fabsf(h[e]), tv[m], dot);
-            const uint32_t code = (uint32_t)m ^ (z < 0.f ? (uint32_t)hw - 1u : (uint32_t)hw);
+            const uint32_t code = m ^ (__float_as_uint(h[e]) >> 31 ? hw - 1u : hw);
             const uint32_t field = wide ? code >> 1 : code;
             const int a = (l * W0) >> 5, off = (l * W0) & 31;
             words[a] |= field << off;
             if (off + W0 > 32) words[a + 1] |= field >> (32 - off);
-            if (wide) {
-                words[W0] |= (code & 1u) << pos;
-                ++pos;
-            }
+            words[W0] |= (wide ? code & 1u : 0u) << l;          // bit l of the group's last word
         }
     }
     if (!live) {
 #pragma unroll
         for (int j = 0; j < W; ++j) words[j] = 0u;
     }
+    dot = live ? dot * __frcp_rn(inv_norm) : 0.f;      // summed as |z| Q(|z|): back to the units of h
 }
 
 // Uniform-interval family (Section 4.3) on the row pass: one signed byte per coordinate
@@ -903,14 +954,14 @@ struct EncTables {
     __device__ __forceinline__ void fill(int t)
     {
         constexpr int half = 1 << (W - 1);
-        // integer budgets search with saturated multiply-adds: boundaries are held as -2^30 t
+        // the searches work with saturated multiply-adds: boundaries are held as -2^30 t
         for (int j = t; j < half; j += kFastThreads) {
-            tb[j] = (FRAC ? 1.f : -1073741824.f) * c_pos_boundary[table_offset(W) + j];
+            tb[j] = -1073741824.f * c_pos_boundary[table_offset(W) + j];
             tv[j] = c_pos_value[table_offset(W) + j];
         }
         if (FRAC)
             for (int j = t; j < (half >> 1); j += kFastThreads) {
-                tb0[j] = c_pos_boundary[table_offset(W > 1 ? W - 1 : 1) + j];
+                tb0[j] = -1073741824.f * c_pos_boundary[table_offset(W > 1 ? W - 1 : 1) + j];
                 tv0[j] = c_pos_value[table_offset(W > 1 ? W - 1 : 1) + j];
             }
     }
@@ -1234,7 +1285,6 @@ k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0)
         constexpr int W0 = W - 1;
         const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
         const float* tbl0 = s_val0 + (arrived ? 0 : (1 << W0));
-        uint32_t pos = 0u;
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             float q[2];
@@ -1246,9 +1296,8 @@ k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0)
                 if (off + W0 > 32) field |= words[a + 1] << (32 - off);
                 field &= (1u << W0) - 1u;
                 const bool wide = (coins >> l) & 1u;
-                const uint32_t code = (field << 1) | ((words[W0] >> pos) & 1u);
+                const uint32_t code = (field << 1) | ((words[W0] >> l) & 1u);
                 q[e] = wide ? tbl[code] : tbl0[field];
-                pos += wide ? 1u : 0u;
             }
             v[k] = pack2(q[0], q[1]);
         }

@@ -235,10 +235,8 @@ k_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
             if (lane == j) mine = word;
         }
         if (frac) {
-            // the lowest code bit of the coordinates whose coin is set, packed in order
-            const uint32_t coins = __ballot_sync(0xffffffffu, coin);
-            const int rank = __popc(coins & ((1u << lane) - 1u));
-            const uint32_t word = __reduce_or_sync(0xffffffffu, coin ? (code & 1u) << rank : 0u);
+            // last word of the group: bit l = lowest code bit of coordinate l if its coin is set
+            const uint32_t word = __ballot_sync(0xffffffffu, coin && (code & 1u));
             if (lane == Wf) mine = word;
         }
         const uint64_t widx = ((base + e) >> 5) * W + lane;
@@ -322,7 +320,6 @@ __device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i
     const int W = (int)cd.W;
     const bool frac = cd.coin_thr != 0u;
     const bool coin = frac && valid && coin_bit(cd.seed, i, cd.coin_thr);
-    const uint32_t coins = frac ? __ballot_sync(0xffffffffu, coin) : 0u;
     if (!valid) return 0.f;
     if (cd.recv) {
         const uint64_t pkt = i >> cd.recv_shift;
@@ -338,8 +335,8 @@ __device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i
         if (cd.utable) return uniform_byte_value(code, tv);
         return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
     }
-    // non-integer budget: groups of 32 coordinates, W words each: (W-1)-bit fields, then the
-    // extra bits of the coordinates whose coin is set
+    // non-integer budget: groups of 32 coordinates, W words each: (W-1)-bit fields, then one
+    // word whose bit l is the extra bit of coordinate l (if its coin is set)
     const int W0 = W - 1;
     const uint32_t l = (uint32_t)(i & 31);
     const uint32_t* grp = cd.codes + (i >> 5) * W;
@@ -348,8 +345,7 @@ __device__ __forceinline__ float received_value(const ClientDesc& cd, uint64_t i
     if (off + W0 > 32) field |= grp[(bit >> 5) + 1] << (32 - off);
     field &= (1u << W0) - 1u;
     if (coin) {
-        const int rank = __popc(coins & ((1u << l) - 1u));
-        const uint32_t code = (field << 1) | ((grp[W0] >> rank) & 1u);
+        const uint32_t code = (field << 1) | ((grp[W0] >> l) & 1u);
         const int half = 1 << (W - 1);
         return code >= (uint32_t)half ? tv[code - half] : -tv[half - 1 - code];
     }

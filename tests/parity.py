@@ -28,7 +28,6 @@ def unpack_fractional(words: np.ndarray, D: int, W0: int, coins: np.ndarray) -> 
     codes = np.zeros(D, dtype=np.int64)
     for g in range((D + 31) // 32):
         grp = words[g * (W0 + 1):(g + 1) * (W0 + 1)]
-        pos = 0
         for l in range(min(32, D - 32 * g)):
             i = 32 * g + l
             field = 0
@@ -36,8 +35,7 @@ def unpack_fractional(words: np.ndarray, D: int, W0: int, coins: np.ndarray) -> 
                 b = l * W0 + j
                 field |= ((int(grp[b // 32]) >> (b % 32)) & 1) << j
             if coins[i]:
-                codes[i] = (field << 1) | ((int(grp[W0]) >> pos) & 1)
-                pos += 1
+                codes[i] = (field << 1) | ((int(grp[W0]) >> l) & 1)     # bit l of the group's last word
             else:
                 codes[i] = field
     return codes

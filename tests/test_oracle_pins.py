@@ -570,17 +570,17 @@ def test_nmse_of_mean_with_unequal_budgets_and_norms_follows_lemma_2_2():
 
 # ----------------------------------------------------------------------------- non-integer budgets b > 1
 def _coins_from_raw_philox(seed, D, bits):
-    thr = int(math.floor((bits - math.floor(bits)) * 65536 + 0.5))
+    thr = int(math.floor((bits - math.floor(bits)) * 256 + 0.5))
     key = [seed & 0xFFFFFFFF, seed >> 32]
     out = np.zeros(D, dtype=bool)
-    for t in range((D + 7) // 8):
+    for t in range((D + 15) // 16):
         w = O.philox4x32_10([t, 0, 2, 0], key)
-        halves = []
+        numbers = []
         for v in w:
-            halves += [int(v) & 0xFFFF, int(v) >> 16]
-        for j in range(8):
-            if 8 * t + j < D:
-                out[8 * t + j] = halves[j] < thr
+            numbers += [(int(v) >> (8 * j)) & 0xFF for j in range(4)]
+        for j in range(16):
+            if 16 * t + j < D:
+                out[16 * t + j] = numbers[j] < thr
     return out
 
 
@@ -588,7 +588,6 @@ def _unpack_fractional(words, D, W0, coins):
     codes = np.zeros(D, dtype=np.int64)
     for g in range((D + 31) // 32):
         grp = words[g * (W0 + 1):(g + 1) * (W0 + 1)]
-        pos = 0
         for l in range(min(32, D - 32 * g)):
             i = 32 * g + l
             field = 0
@@ -596,8 +595,7 @@ def _unpack_fractional(words, D, W0, coins):
                 b = l * W0 + j
                 field |= ((int(grp[b // 32]) >> (b % 32)) & 1) << j
             if coins[i]:
-                codes[i] = (field << 1) | ((int(grp[W0]) >> pos) & 1)
-                pos += 1
+                codes[i] = (field << 1) | ((int(grp[W0]) >> l) & 1)     # bit l of the group's last word
             else:
                 codes[i] = field
     return codes
@@ -609,7 +607,7 @@ def test_fractional_budget_against_dense_reference(d, bits):
     x = rng.standard_normal(d).astype(np.float32)
     seed = int(rng.integers(1, 2 ** 63))
     D, W0 = O.rot_dim(d, bits), int(math.floor(bits))
-    assert O.code_width(bits) == W0 + 1 and O.coin_threshold(bits) == round((bits - W0) * 65536)
+    assert O.code_width(bits) == W0 + 1 and O.coin_threshold(bits) == round((bits - W0) * 256)
     coins = _coins_from_raw_philox(seed, D, bits)
     assert all(O.coin(seed, i, O.coin_threshold(bits)) == coins[i] for i in range(D))
     # independent dense route: rotate, per-coordinate nearest value in its own table (Section 4.1)
