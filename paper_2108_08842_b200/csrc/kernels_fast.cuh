@@ -857,6 +857,35 @@ __device__ __forceinline__ void quantise_pack_frac(const u64 (&v)[16], float inv
                                                    uint32_t (&words)[W], float& dot)
 {
     constexpr int W0 = W - 1;
+    if constexpr (W == 2) {
+        // 1 < b < 2 (the paper's own example is b = 1.5): one-bit codes, two-bit codes where the
+        // coin is set.  The first word is the "not negative" bits either way (the upper bit of a
+        // two-bit code is that bit too); the second holds index XOR sign of the coordinates with
+        // a coin.  Signs and indices are gathered into words by funnel shifts and combined once
+        // per thread; the value is c1 + coin * ((v0 - c1) + index * (v1 - v0)) by multiply-adds.
+        const FmaTree& tr = c_tree[2];
+        const float c1 = c_pos_value[0], lift = tr.v0 - c1;
+        uint32_t negs = 0u, idx = 0u;
+#pragma unroll
+        for (int k = 15; k >= 0; --k) {
+            float h[2];
+            unpack2(v[k], h[0], h[1]);
+#pragma unroll
+            for (int e = 1; e >= 0; --e) {
+                const int l = 2 * k + e;
+                const float az = fabsf(h[e]) * inv_norm;
+                const float ind = fma_sat(az, tr.big, tr.k_root);
+                negs = __funnelshift_l(__float_as_uint(h[e]), negs, 1);
+                idx = __funnelshift_l(__float_as_uint(fmaf(ind, -2.f, 0.5f)), idx, 1);     // its sign bit is the index
+                const float coin = __uint_as_float((uint32_t)((int)(coins << (31 - l)) >> 31) & 0x3F800000u);
+                dot = fmaf(az, fmaf(coin, fmaf(ind, tr.dv, lift), c1), dot);
+            }
+        }
+        words[0] = live ? ~negs : 0u;
+        words[1] = live ? (idx ^ negs) & coins : 0u;
+        dot = live ? dot * __frcp_rn(inv_norm) : 0.f;
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < W; ++j) words[j] = 0u;
 #pragma unroll
@@ -1284,7 +1313,12 @@ k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0)
         // non-integer budget: (W-1)-bit fields, then the extra bits of the coordinates whose coin is set
         constexpr int W0 = W - 1;
         const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
-        const float* tbl0 = s_val0 + (arrived ? 0 : (1 << W0));
+        // One load per coordinate, no branches: the shared-memory address of the value in the
+        // wider table (field and extra bit) and in the narrower one (field alone) are both
+        // formed, the coin's mask picks one.  Both include the offset of the zero half for
+        // a lost packet.
+        const uint32_t hi_addr = smem_addr(s_val) + (arrived ? 0u : (4u << W));
+        const uint32_t lo_addr = smem_addr(s_val0) + (arrived ? 0u : (4u << W0));
 #pragma unroll
         for (int k = 0; k < 16; ++k) {
             float q[2];
@@ -1292,12 +1326,15 @@ k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0)
             for (int e = 0; e < 2; ++e) {
                 const int l = 2 * k + e;
                 const int a = (l * W0) >> 5, off = (l * W0) & 31;
-                uint32_t field = words[a] >> off;
-                if (off + W0 > 32) field |= words[a + 1] << (32 - off);
-                field &= (1u << W0) - 1u;
-                const bool wide = (coins >> l) & 1u;
-                const uint32_t code = (field << 1) | ((words[W0] >> l) & 1u);
-                q[e] = wide ? tbl[code] : tbl0[field];
+                uint32_t x;                                     // the field at bits [2, W0 + 2): its byte offset
+                if (off >= 2) x = off + W0 > 32 ? __funnelshift_r(words[a], words[a + 1 < W ? a + 1 : a], off - 2)
+                                                : words[a] >> (off - 2);
+                else x = words[a] << (2 - off);
+                const uint32_t fb = x & (((1u << W0) - 1u) << 2);
+                const uint32_t eb = (l >= 2 ? words[W0] >> (l - 2) : words[W0] << (2 - l)) & 4u;   // the extra bit, times four
+                const uint32_t wide = (uint32_t)((int)(coins << (31 - l)) >> 31);                  // all ones if the coin is set
+                const uint32_t addr = ((hi_addr + 2u * fb + eb) & wide) | ((lo_addr + fb) & ~wide);
+                asm("ld.shared.f32 %0, [%1];" : "=f"(q[e]) : "r"(addr));
             }
             v[k] = pack2(q[0], q[1]);
         }
