@@ -939,8 +939,9 @@ struct SlabStreams {
 
 // Sender passes of one group on the register-blocked path.
 // `h_descs`: the host copy of the group's descriptors (d_descs is the same array on the device).
+// `fold_scales`: small rounds: the row pass writes the scales itself (no k_enc_scale); else nullptr.
 int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g, const ClientDesc* h_descs,
-                      ClientDesc* d_descs, ClientState* d_states, uint64_t d, uint32_t* d_status)
+                      ClientDesc* d_descs, ClientState* d_states, uint64_t d, uint32_t* d_status, float* fold_scales)
 {
     const uint32_t gn = (uint32_t)g.members.size();
     const double D = (double)(1ull << g.L);
@@ -996,7 +997,7 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
                     EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_W(r.W,
                         LAUNCH_CL(ctx, "f_enc_last", cn * (4.0 + r.W / 8.0) * 8192.0 * tn, (k_f_enc_last<W_, 0, FRAC_>),
                                   dim3(tn, cn), dim3(kFastThreads), 0, dd, ds,
-                                  (const float*)h_descs[r.first + c0].work, g.L, inv_ready, t0)));
+                                  (const float*)h_descs[r.first + c0].work, g.L, inv_ready, t0, fold_scales, d_status)));
                 }
             }
         }
@@ -1006,7 +1007,7 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
         if (g.uniform) {
             LAUNCH(ctx, "f_enc_last", r.count * 5.0 * D, (k_f_enc_last<8, 0, false, true>), dim3(tiles, r.count),
                    kFastThreads, 0, (const ClientDesc*)(d_descs + r.first), d_states + r.first,
-                   (const float*)h_descs[r.first].work, g.L, inv_ready, 0u);
+                   (const float*)h_descs[r.first].work, g.L, inv_ready, 0u, fold_scales, d_status);
             continue;
         }
         if (ctx->row_staging && pl.row_lc == 0) {
@@ -1026,17 +1027,19 @@ int fast_encode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
             LAUNCH_CL(ctx, "f_enc_last", r.count * (4.0 + r.W / 8.0) * D, (k_f_enc_last<W_, LC_, FRAC_>),
                       dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
                       (const ClientDesc*)(d_descs + r.first), d_states + r.first,
-                      (const float*)h_descs[r.first].work, g.L, inv_ready, 0u))));
+                      (const float*)h_descs[r.first].work, g.L, inv_ready, 0u, fold_scales, d_status))));
     }
     return EDEN_OK;
 }
 
 // Receiver passes of one group on the register-blocked path.
 // `part`/`part_bytes`: free workspace behind the group's work buffers, for partial sums.
+// `fold_scales`: small rounds: the row pass does k_dec_prep's work from these scales; else nullptr.
 int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const Group& g,
                       ClientDesc* d_descs, ClientState* d_states, float* out, uint64_t d, int mode,
-                      float* part, uint64_t part_bytes)
+                      float* part, uint64_t part_bytes, const float* fold_scales, uint32_t* d_status)
 {
+    ClientState* const fold_states = fold_scales ? d_states : nullptr;
     const uint32_t gn = (uint32_t)g.members.size();
     const double D = (double)(1ull << g.L);
     const unsigned tiles = (unsigned)((1ull << g.L) >> kFastTileLog);
@@ -1064,7 +1067,8 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
                     fork.use(slab++);
                     EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_W(r.W,
                         LAUNCH_CL(ctx, "f_dec_first", cn * (4.0 + r.W / 8.0) * 8192.0 * tn, (k_f_dec_first<W_, 0, FRAC_>),
-                                  dim3(tn, cn), dim3(kFastThreads), 0, dd, t0)));
+                                  dim3(tn, cn), dim3(kFastThreads), 0, dd, t0,
+                                  fold_states ? fold_states + r.first + c0 : nullptr, fold_scales, d_status)));
                     EDEN_DISPATCH_LR(ps.lr,
                         LAUNCH_CL(ctx, "f_mid", cn * 8.0 * 8192.0 * tn, (k_f_col<LR_, 0, false>), dim3(tn, cn),
                                   dim3(kFastThreads), 0, dd, d_states + r.first + c0, ps.lo, 0, t0));
@@ -1076,7 +1080,8 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
             EDEN_DISPATCH_FRAC(g.fractional, EDEN_DISPATCH_LC(pl.row_lc, EDEN_DISPATCH_W(r.W,
                 LAUNCH_CL(ctx, "f_dec_first", r.count * (4.0 + r.W / 8.0) * D, (k_f_dec_first<W_, LC_, FRAC_>),
                           dim3(tiles, r.count), dim3(kFastThreads), pl.row_lc,
-                          (const ClientDesc*)(d_descs + r.first), 0u))));
+                          (const ClientDesc*)(d_descs + r.first), 0u,
+                          fold_states ? fold_states + r.first : nullptr, fold_scales, d_status))));
         }
     }
     // the receiver walks the column ranges bottom-up so that the top range comes last
@@ -1122,6 +1127,11 @@ int fast_decode_group(eden_ctx* ctx, const std::vector<ClientPlan>& plan, const 
     }
     return EDEN_OK;
 }
+
+// rounds of at most this many row-pass tiles (2^25 coordinates) fold their small kernels into the row pass
+// (at 2^28 the fence per tile already costs the sender's row pass 7 %)
+constexpr uint64_t kFoldMaxTiles = 4096;
+constexpr uint64_t kFoldMaxMaskWords = 256;    // ... if a client's received-bitmap is at most this long
 
 bool fast_eligible(const eden_ctx* ctx, const Group& g)
 {
@@ -1343,6 +1353,16 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
     rc = upload_descs_and_clear_states(ctx, lay, descs);
     if (rc) return rc;
 
+    // Small rounds (the paper's federated-learning sizes) are a handful of launches of a few
+    // microseconds each: there the row pass writes the scales itself and k_enc_scale is not
+    // launched.  Needs every group on the register-blocked path.
+    bool fold = !ctx->row_staging;
+    uint64_t fold_tiles = 0;
+    for (const Group& g : groups) {
+        fold = fold && fast_eligible(ctx, g) && (x_aligned || g.subbit);
+        fold_tiles += (uint64_t)g.members.size() << (g.L > kFastTileLog ? g.L - kFastTileLog : 0);
+    }
+    fold = fold && fold_tiles <= kFoldMaxTiles;
     for (size_t gi = 0; gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
         const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
@@ -1372,7 +1392,8 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
                        dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
         }
         if (fast_eligible(ctx, g) && (x_aligned || g.subbit)) {
-            rc = fast_encode_group(ctx, plan, g, descs.data() + first, d_descs + first, d_states + first, d, d_status);
+            rc = fast_encode_group(ctx, plan, g, descs.data() + first, d_descs + first, d_states + first, d, d_status,
+                                   fold ? scales : nullptr);
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);
@@ -1397,7 +1418,8 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
                    sizeof(float) << lc, d_descs + first, d_states + first, rg);
         }
     }
-    LAUNCH(ctx, "enc_scale", n * 20.0, k_enc_scale, (n + 127) / 128, 128, 0, d_descs, d_states, scales, n, d_status);
+    if (!fold)
+        LAUNCH(ctx, "enc_scale", n * 20.0, k_enc_scale, (n + 127) / 128, 128, 0, d_descs, d_states, scales, n, d_status);
     return EDEN_OK;
 }
 
@@ -1493,7 +1515,17 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
     }
     rc = upload_descs_and_clear_states(ctx, lay, descs);
     if (rc) return rc;
-    LAUNCH(ctx, "dec_prep", n * 8.0, k_dec_prep, n, 256, 0, d_descs, d_states, scales, d_status);
+    // small rounds: the receiver's row pass computes p and the factor itself (see encode_common)
+    bool fold = true;
+    uint64_t fold_tiles = 0;
+    for (const Group& g : groups) {
+        fold = fold && fast_eligible(ctx, g) && (out_aligned || g.subbit) &&
+               ((1ull << g.L) >> recv_shift) <= 32ull * kFoldMaxMaskWords;
+        fold_tiles += (uint64_t)g.members.size() << (g.L > kFastTileLog ? g.L - kFastTileLog : 0);
+    }
+    fold = fold && fold_tiles <= kFoldMaxTiles;
+    if (!fold)
+        LAUNCH(ctx, "dec_prep", n * 8.0, k_dec_prep, n, 256, 0, d_descs, d_states, scales, d_status);
 
     // the first group with b >= 1 covers every output coordinate, so for the mean it may
     // overwrite; everything after it accumulates
@@ -1532,7 +1564,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         if (fast_eligible(ctx, g) && (out_aligned || g.subbit)) {
             rc = fast_decode_group(ctx, plan, g, d_descs + first, d_states + first, out, d, mode,
                                    (float*)(ctx->ws + lay.work_off + group_work_end[gi]),
-                                   lay.work_bytes - group_work_end[gi]);
+                                   lay.work_bytes - group_work_end[gi], fold ? scales : nullptr, d_status);
             if (rc) return rc;
         } else if (g.L <= kGenericTileLog) {
             const PassGeom rg = row_geom(g.L);

@@ -36,6 +36,8 @@ struct ClientState {
     double received;         // fraction of coordinates received
     float factor;            // decode: S / (p sqrt D) * mean_scale
     uint32_t flags;
+    uint32_t tiles_done;     // encode, small rounds: tiles of the last pass that have added their part of `dot`
+    uint32_t reserved;
 };
 
 // Result of the exact-size mask selection for one (seed, d, k): coordinate i is kept

@@ -1074,7 +1074,9 @@ template <int W, int LC, bool FRAC, bool UNI = false>
 #endif
 __global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : EDEN_ENC_LAST_BLOCKS))
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L,
-             int inv_ready, uint32_t tile0)
+             int inv_ready, uint32_t tile0,
+             float* __restrict__ scales /* small rounds: the block that finishes a client writes its scale S; else nullptr */,
+             uint32_t* __restrict__ status)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ float s_warp_dot[kFastThreads / 32];
@@ -1128,7 +1130,28 @@ k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ sta
         float tot = 0.f;
 #pragma unroll
         for (int j = 0; j < kFastThreads / 32; ++j) tot += s_warp_dot[j];
-        atomicAdd(&states[blockIdx.y].dot, (double)tot);
+        ClientState* st = &states[blockIdx.y];
+        atomicAdd(&st->dot, (double)tot);
+        if (scales) {
+            // Small rounds save a launch: every tile counts itself in after its sum has gone out
+            // (the fence orders the two), and the tile that counts last has all sums before it
+            // and forms S = ||y||^2 sqrt(D) / sum h Q (Section 2.3) like k_enc_scale.  An
+            // arrival counter, nobody waits.  (Large rounds keep the separate kernel: a fence
+            // per tile costs them more than one launch.)
+            __threadfence();
+            if (atomicAdd(&st->tiles_done, 1u) == (1u << (L - kFastTileLog)) - 1u) {
+                __threadfence();
+                const double dot_all = atomicAdd(&st->dot, 0.0), n2 = st->norm2;
+                uint32_t flags = 0;
+                double S = 0.0;
+                if (!(n2 < INFINITY)) flags |= 0x2u;
+                else if (n2 == 0.0) flags |= 0x1u;
+                else S = cd.extra_scale * n2 * sqrt((double)(1ull << L)) / dot_all;
+                scales[cd.index] = (float)S;
+                st->flags = flags;
+                if (flags) atomicOr(status, flags);
+            }
+        }
     }
 }
 
@@ -1250,7 +1273,9 @@ k_f_enc_last_staged(const ClientDesc* __restrict__ descs, ClientState* __restric
 // =================================================================================
 template <int W, int LC, bool FRAC>
 __global__ void __launch_bounds__(kFastThreads, 4)
-k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0)
+k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0,
+              ClientState* __restrict__ states /* small rounds: tile 0 of a client does k_dec_prep's work; else nullptr */,
+              const float* __restrict__ scales, uint32_t* __restrict__ status)
 {
     __shared__ __align__(16) u64 s[kRowSmemUnits];
     __shared__ float s_val[2 << W];                    // the 2^W values by code, then 2^W zeros
@@ -1275,6 +1300,34 @@ k_f_dec_first(const ClientDesc* __restrict__ descs, uint32_t tile0)
                                                 : -c_pos_value[table_offset(W > 1 ? W - 1 : 1) + h0 - 1 - j];
             s_val0[j] = c;
         }
+    if (states && blockIdx.x + tile0 == 0u && t < 32) {
+        // received fraction p and the factor S / (p sqrt D) of this client (Section 4.2), for
+        // the last pass: one warp counts the bitmap (small rounds only: a few words)
+        const uint64_t D = 1ull << cd.L;
+        const uint64_t bits = (D + (1ull << cd.recv_shift) - 1) >> cd.recv_shift;
+        uint32_t cnt = 0u;
+        if (cd.recv) {
+            for (uint64_t w = t; w < (bits + 31) >> 5; w += 32) {
+                uint32_t word = cd.recv[w];
+                const uint64_t left = bits - (w << 5);
+                if (left < 32) word &= (1u << left) - 1u;
+                cnt += (uint32_t)__popc(word);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        }
+        if (t == 0) {
+            const double got = cd.recv ? (double)cnt : (double)bits;
+            const double coords = D >= (1ull << cd.recv_shift) ? got * (double)(1ull << cd.recv_shift) : got * (double)D;
+            const double p = coords / (double)D;
+            ClientState* st = &states[blockIdx.y];
+            const uint32_t flags = coords == 0.0 ? 0x4u : 0u;
+            st->received = p;
+            st->factor = flags ? 0.f : (float)((double)scales[cd.index] / (p * sqrt((double)D)) * cd.mean_scale);
+            st->flags = flags;
+            if (flags) atomicOr(status, flags);
+        }
+    }
     __syncthreads();
     const uint64_t base = (uint64_t)(blockIdx.x + tile0) << kFastTileLog;
     // the tile is 8 packets of 1024 coordinates; this thread's 32 coordinates lie in one.

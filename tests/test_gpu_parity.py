@@ -374,8 +374,9 @@ def test_unaligned_input_rows_take_the_generic_path(E):
     ctx.close()
 
 
-def test_zero_vector_and_status_word(E):
-    d, n = 5000, 3
+@pytest.mark.parametrize("d", [5000, 40000])     # one block per client; the multi-pass kernels (whose row pass writes the scales of a small round itself)
+def test_zero_vector_and_status_word(E, d):
+    n = 3
     xs = np.random.default_rng(1).standard_normal((n, d)).astype(np.float32)
     xs[1] = 0.0
     ctx = _ctx(E, d, n)
@@ -400,13 +401,14 @@ def test_zero_vector_and_status_word(E):
     ctx.close()
 
 
-def test_all_packets_lost_is_reported_not_fatal(E):
-    d, n = 4096, 2
+@pytest.mark.parametrize("d", [4096, 1 << 15])    # 4 packets, one block per client; 32 packets, multi-pass kernels
+def test_all_packets_lost_is_reported_not_fatal(E, d):
+    n = 2
     xs = np.random.default_rng(2).standard_normal((n, d)).astype(np.float32)
     ctx = _ctx(E, d, n)
     codes, scales = ctx.encode(torch.from_numpy(xs).cuda(), [1.0, 1.0], [5, 6])
     none = torch.zeros(1, dtype=torch.int32, device="cuda")
-    full = torch.full((1,), 0xF, dtype=torch.int32, device="cuda")
+    full = torch.full((1,), -1 if d > 4096 else 0xF, dtype=torch.int32, device="cuda")
     mean = ctx.mean(codes, scales, [1.0, 1.0], [5, 6], d, [none, full]).cpu().numpy()
     assert ctx.status() == E.STATUS_NO_DATA
     stats = ctx.client_stats(n)
