@@ -304,7 +304,8 @@ def test_mask_threshold_on_a_pair_of_equal_keys(E, which, extra, rounds):
     run_workload(E, work, options=[(E.OPT_SEL_ROUNDS, rounds)])
 
 
-@pytest.mark.parametrize("bits,d", [(1.5, 100), (1.5, 40000), (2.25, 5000), (7.5, 3000), (3.75, 300000)])
+@pytest.mark.parametrize("bits,d", [(1.5, 100), (1.5, 40000), (2.25, 5000), (7.5, 3000), (3.75, 300000),
+                                    (1.5, (1 << 22) + 5), (2.5, 1 << 21), (4.75, 70000), (5.5, 40000)])
 def test_non_integer_budgets(E, bits, d):
     # Section 4.1: a shared coin per coordinate picks 2^floor(b) or 2^(floor(b)+1) values
     n = 3

@@ -92,6 +92,22 @@ def test_vnmse_follows_lemma_4_3_at_2_pow_22(E):
     assert abs(nmse - expect) < 0.05 * expect
 
 
+def test_zero_vector_is_reported_and_decodes_to_zero(E):
+    d = 20000
+    xs = np.zeros((2, d), dtype=np.float32)
+    xs[1] = np.random.default_rng(5).standard_normal(d).astype(np.float32)
+    seeds, bits = [41, 42], [0.5, 0.5]
+    ctx = E.Context(0, workspace_bytes_=E.after_workspace_bytes(d, 2))
+    codes, scales = ctx.encode_sparsify_after(torch.from_numpy(xs).cuda(), bits, seeds)
+    assert ctx.status() == E.STATUS_ZERO_VECTOR
+    assert float(scales[0]) == 0.0 and not codes[0].any()
+    got = ctx.mean_sparsify_after(codes, scales, bits, seeds, d).cpu().numpy()
+    e = O.encode_after(xs[1], 0.5, 42)
+    want = O.decode_after(e["codes"], float(np.float32(e["scale"])), 0.5, 42, d) / 2
+    assert np.max(np.abs(got - want)) <= 1e-3 * np.max(np.abs(want))
+    ctx.close()
+
+
 def test_budgets_outside_the_sub_bit_range_are_refused(E):
     ctx = E.Context(0, workspace_bytes_=E.after_workspace_bytes(1000, 1))
     x = torch.zeros((1, 1000), dtype=torch.float32, device="cuda")

@@ -53,6 +53,22 @@ def test_size_rules_match_oracle(lib):
             assert cb % 16 == 0 and 4 * words <= cb < 4 * words + 16
     for bad in (0.0, -1.0, 8.5, 9.0, float("nan")):
         assert lib.eden_code_width(bad) == 0
+    # sparsification after the rotation: the kept count is taken over the rotated coordinates
+    lib.eden_after_kept_count.restype = ctypes.c_uint64
+    lib.eden_after_code_bytes.restype = ctypes.c_uint64
+    lib.eden_after_workspace_bytes.restype = ctypes.c_uint64
+    lib.eden_workspace_bytes.restype = ctypes.c_uint64
+    for f in (lib.eden_after_kept_count, lib.eden_after_code_bytes):
+        f.argtypes = [ctypes.c_uint64, ctypes.c_double]
+    lib.eden_after_workspace_bytes.argtypes = [ctypes.c_uint64, ctypes.c_uint32]
+    lib.eden_workspace_bytes.argtypes = [ctypes.c_uint64, ctypes.c_uint32]
+    for d in (1, 33, 1000, 1025, 10 ** 6, 2 ** 23):
+        for bits in (0.001, 0.1, 0.5, 0.999):
+            k = O.after_kept_count(d, bits)
+            assert lib.eden_after_kept_count(d, bits) == k and 1 <= k <= O.rot_dim(d, 1.0)
+            cb = lib.eden_after_code_bytes(d, bits)
+            assert cb % 16 == 0 and (k + 31) // 32 * 4 <= cb < (k + 31) // 32 * 4 + 16
+        assert lib.eden_after_workspace_bytes(d, 3) > lib.eden_workspace_bytes(d, 3)
 
 
 def test_library_tables_match_oracle_tables(lib):
