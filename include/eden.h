@@ -122,8 +122,9 @@ int eden_table(uint32_t W, float* centroids, float* boundaries);
 
 /* Host only.  The kernels search the intervals of code widths 2..4 with multiply-adds whose
  * constants are derived from the table above; EDEN_OK if every boundary that search can
- * form is bit-identical to the table's fp32 boundary (it is, for the tables of Section 3;
- * eden_create refuses to run otherwise). */
+ * form is bit-identical to the table's fp32 boundary and no boundary is too small for the
+ * kernels' exact comparison (both hold for the tables of Section 3; eden_create refuses
+ * to run otherwise). */
 int eden_self_check(void);
 
 /* ---- context ---------------------------------------------------------------------- */

@@ -191,6 +191,9 @@ const Tables& tables()
         std::memset(t.tree, 0, sizeof(t.tree));
         for (int W = 2; W <= 8; ++W) {
             const int off = (1 << (W - 1)) - 1;
+            // the saturated multiply-adds need one unit in the last place of any boundary,
+            // times 2^30, to be at least 1: no boundary below 2^-7
+            t.tree_exact = t.tree_exact && t.pos_boundary[off] >= 0.0078125f;
             if (W <= 4) {
                 t.tree_exact = build_fma_tree(W, t.pos_boundary + off, t.pos_value + off, t.tree[W]) && t.tree_exact;
             } else {

@@ -573,8 +573,9 @@ __device__ __forceinline__ void row_step_inner(u64 (&v)[16])
 // instead of compares and selects on the half-rate ALU pipe.
 // With a boundary t held as T = -2^30 t, the saturated multiply-add sat(az 2^30 + T) is
 // exactly 1 if az > t and exactly 0 otherwise: az - t is zero or at least one unit in the
-// last place of the smaller operand (2^-26 for the smallest boundary), which the factor
-// 2^30 lifts above 1, and the multiply-add rounds once.  The boundary of the next level is
+// last place of t (2^-25 for the smallest boundary of the four-bit table, 2^-29 for that of
+// the eight-bit one: the host checks that no boundary lies below 2^-7), which the factor
+// 2^30 lifts to 1 or more, and the multiply-add rounds once.  The boundary of the next level is
 // itself a multiply-add of that indicator (constants chosen on the host so that, rounded
 // towards zero, it lands exactly on the fp32 boundary), and the index is the sum of the
 // indicators (as a float 0..7) times the subnormal number 2^-149, whose bit pattern is the
@@ -1065,14 +1066,11 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
 // one another 2^L floats apart, so a block's tile address needs no descriptor and its loads
 // start at once.
 template <int W, int LC, bool FRAC, bool UNI = false>
-// Five resident blocks per SM for integer budgets (51 registers; at most a few words
-// spilled): cfg5's shape 3240 -> 3370 GB/s, cfg4's 5000 -> 5090 GB/s.  Six fit as well but
-// run slower (2940 / 4310 GB/s, with or without L1 allocation of the tile loads).  The
-// non-integer budgets keep four (their coins cost registers).
-#ifndef EDEN_ENC_LAST_BLOCKS
-#define EDEN_ENC_LAST_BLOCKS (W >= 3 ? 4 : 5)
-#endif
-__global__ void __launch_bounds__(kFastThreads, (FRAC ? 4 : EDEN_ENC_LAST_BLOCKS))
+// Resident blocks per SM: five for one- and two-bit codes (48 registers, a few words spilled:
+// 5580 -> 5870 GB/s at W = 1 against four); four from three bits on and for non-integer
+// budgets, whose search constants and coins want the 64 registers (W = 4: 4140 GB/s with
+// four blocks and no spills, 3960 with five and 68 bytes spilled).  Six run slower at every width.
+__global__ void __launch_bounds__(kFastThreads, (FRAC || W >= 3 ? 4 : 5))
 k_f_enc_last(const ClientDesc* __restrict__ descs, ClientState* __restrict__ states, const float* __restrict__ work0, int L,
              int inv_ready, uint32_t tile0,
              float* __restrict__ scales /* small rounds: the block that finishes a client writes its scale S; else nullptr */,

@@ -420,6 +420,16 @@ def test_all_packets_lost_is_reported_not_fatal(E, d):
     ctx.close()
 
 
+def test_options_are_checked(E):
+    ctx = _ctx(E, 1024, 1)
+    for opt, bad in ((E.OPT_PLAN_VARIANT, 4), (E.OPT_ROW_STAGING, 2), (E.OPT_SEL_ROUNDS, 1), (E.OPT_SLAB_MIB, -1),
+                     (E.OPT_SLAB_STREAMS, 0), (E.OPT_SLAB_SIDES, 4), (99, 0)):
+        with pytest.raises(E.EdenError) as e:
+            ctx.set_option(opt, bad)
+        assert e.value.code == -1
+    ctx.close()
+
+
 def test_bad_arguments(E):
     ctx = _ctx(E, 1024, 2)
     x = torch.zeros(2, 1024, device="cuda")
