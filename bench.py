@@ -258,6 +258,10 @@ def run_gpu(args):
         masks_np = [work.recv_mask(c, eden.num_packets(d, float(bits[c]))) for c in range(n)]
         masks_gpu = [torch.from_numpy(m.view(np.int32)).to(dev) for m in masks_np]
     ctx = eden.Context(local_rank, d_max=d, n_batch=n, host_staging=True)
+    if args.sel_rounds:
+        ctx.set_option(eden.OPT_SEL_ROUNDS, args.sel_rounds)
+    if args.sel_inline:
+        ctx.set_option(eden.OPT_SEL_AHEAD, 0)
     if args.slab_mib:
         ctx.set_option(eden.OPT_SLAB_MIB, args.slab_mib)
         ctx.set_option(eden.OPT_SLAB_STREAMS, args.slab_streams)
@@ -373,6 +377,7 @@ def run_gpu(args):
         achieved = top["bytes"] / top["launches"] / (top["ms"] / top["launches"] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": top_name, "achieved": achieved, "peak": peak,
                     "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                    "frac_of_nominal_8000": achieved / 8000.0,
                     "traffic": (traffic_table[top_name] * n * float(eden.rot_dim(d, float(bits[0])))
                                 if top_name in traffic_table and len(set(map(float, bits))) == 1 else None),
                     "traffic_source": "ncu dram__bytes_read+write, one client, scaled by clients per launch "
@@ -435,8 +440,19 @@ def run_gpu(args):
         sample = synth.make(args.workload, d=d, n=threads, seed=rank)
         if args.bits is not None:
             sample.bits = np.full(sample.n, float(args.bits))
-        dt, nbytes, _ = oracle_sample(sample, list(range(threads)), threads)
+        dt, nbytes, o_mean = oracle_sample(sample, list(range(threads)), threads)
+        # the oracle's own accuracy on its sample (NMSE of its mean against the sample's true mean)
+        o_true = np.zeros(d, dtype=np.float64)
+        o_energy = 0.0
+        for c in range(threads):
+            xc = sample.vector(c).astype(np.float64)
+            o_true += xc
+            o_energy += float(np.dot(xc, xc))
+        o_true /= threads
+        o_nmse = float(np.sum((o_mean - o_true) ** 2) / (o_energy / threads))
+        del o_true
         cpu = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "nmse_vs_true_mean_of_sample": o_nmse,
                "sample": "%d of the %d clients of %s at its own dimension (%d coordinates, rotation of %d), "
                          "encode + decode+mean, %d threads, %.1f s" %
                          (threads, n, work.name, d, eden.rot_dim(d, float(bits[0])), threads, dt)}
@@ -546,6 +562,10 @@ def main():
                          "Lloyd-Max tables; device-resident timing only (no end-to-end or CPU leg)")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="experiment: no per-kernel event bracketing in the timed region (no kernel table, no roofline)")
+    ap.add_argument("--sel-rounds", type=int, default=0,
+                    help="experiment: form of the b < 1 mask selection (EDEN_OPT_SEL_ROUNDS; 0 keeps the default)")
+    ap.add_argument("--sel-inline", action="store_true",
+                    help="experiment: select the b < 1 masks in line instead of ahead on a side stream (EDEN_OPT_SEL_AHEAD 0)")
     ap.add_argument("--slab-streams", type=int, default=1)
     ap.add_argument("--slab-sides", type=int, default=3)
     ap.add_argument("--slab-mib", type=int, default=0,

@@ -341,9 +341,16 @@ int eden_force_generic_kernels(eden_ctx* ctx, int on);
  *                          saves one sweep over HBM for 2^24..2^27 coordinates.
  *   EDEN_OPT_ROW_STAGING   1: the sender's last pass runs as a persistent kernel whose
  *                          tiles are staged in shared memory by bulk asynchronous copies.
- *   EDEN_OPT_SEL_ROUNDS    2 (default): the threshold of a b < 1 mask is found in two passes
- *                          over the keys where the candidate list holds them; 3: always in
- *                          three histogram rounds (the form very long vectors use).
+ *   EDEN_OPT_SEL_ROUNDS    How the threshold of a b < 1 mask (the k-th smallest key) is found.
+ *                          1 (default): in one pass over the keys, which keeps the keys inside
+ *                          a band predicted from k/d as candidates; a job whose threshold
+ *                          turns out to lie outside its band is redone by form 2 (the mask is
+ *                          the same either way).  2: a histogram pass, then the candidate
+ *                          pass.  3: three histogram rounds (the form vectors too long for
+ *                          the candidate list use whatever this option says).
+ *   EDEN_OPT_SEL_BAND      Half-width of form 1's band in tenths of a standard deviation of
+ *                          the k-th smallest of d uniform keys, 0..120 (default 40).  0 leaves
+ *                          the band empty, so every job is redone: for tests.
  *   EDEN_OPT_SLAB_MIB      0 (default): every pass of the transform is one launch over all
  *                          clients of a group; m > 0: vectors that take three sweeps run
  *                          their middle and last (receiver: first and middle) pass slab by
@@ -354,6 +361,10 @@ int eden_force_generic_kernels(eden_ctx* ctx, int on);
 #define EDEN_OPT_SEL_ROUNDS   3
 #define EDEN_OPT_SLAB_MIB     4
 #define EDEN_OPT_SLAB_SIDES   6   /* 1: sender only, 2: receiver only, 3 (default): both */
+#define EDEN_OPT_SEL_BAND     7
+#define EDEN_OPT_SEL_AHEAD    8   /* 1 (default): in a call that mixes budgets below and above one bit, the masks of the
+                                     b < 1 senders are selected on a side stream while the other senders' passes run on
+                                     the context's stream, which waits for them where it needs them; 0: in line */
 #define EDEN_OPT_SLAB_STREAMS 5   /* 1 (default)..4: slabs are dealt round-robin to this many streams, so that
                                      one slab's second pass can overlap the next slab's first */
 int eden_set_option(eden_ctx* ctx, int option, int value);

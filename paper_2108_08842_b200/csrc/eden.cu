@@ -324,6 +324,10 @@ struct eden_ctx {
     int plan_variant;
     int row_staging;                 // 1: the sender's row pass runs in its persistent, bulk-copy-staged form
     int sel_rounds;                  // 3: the b < 1 mask threshold is found in three histogram rounds at every size
+    int sel_band;                    // half-width of the predicted band of the one-pass selection, tenths of a standard deviation
+    int sel_ahead;                   // 1: the masks of a call's b < 1 clients are selected on a side stream while the b >= 1 groups run
+    cudaStream_t sel_stream;         // that side stream (created on first use)
+    std::vector<cudaEvent_t> sel_events;   // fork (0), join (1) and one per b < 1 group (2 + ...)
     int slab_mib;                    // > 0: middle and row pass are launched slab by slab (MiB of intermediate per slab)
     int slab_streams;                // slabs are dealt round-robin to this many streams (1 = the context's own)
     int slab_sides;                  // bit 0: the sender uses the slab order, bit 1: the receiver
@@ -404,7 +408,10 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
     ctx->force_generic = false;
     ctx->plan_variant = 0;
     ctx->row_staging = 0;
-    ctx->sel_rounds = 2;
+    ctx->sel_rounds = 1;
+    ctx->sel_band = 40;
+    ctx->sel_ahead = 1;
+    ctx->sel_stream = nullptr;
     ctx->slab_mib = 0;
     ctx->slab_streams = 1;
     ctx->slab_sides = 3;
@@ -441,6 +448,8 @@ extern "C" int eden_destroy(eden_ctx* ctx)
     for (cudaEvent_t e : ctx->sync_events) cudaEventDestroy(e);
     for (cudaStream_t st : ctx->side) cudaStreamDestroy(st);
     for (cudaEvent_t e : ctx->slab_events) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->sel_events) cudaEventDestroy(e);
+    if (ctx->sel_stream) cudaStreamDestroy(ctx->sel_stream);
     if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
     if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
     delete ctx;
@@ -469,8 +478,16 @@ extern "C" int eden_set_option(eden_ctx* ctx, int option, int value)
             ctx->row_staging = value;
             return EDEN_OK;
         case EDEN_OPT_SEL_ROUNDS:
-            if (value != 2 && value != 3) return EDEN_ERR_INVALID_ARG;
+            if (value < 1 || value > 3) return EDEN_ERR_INVALID_ARG;
             ctx->sel_rounds = value;
+            return EDEN_OK;
+        case EDEN_OPT_SEL_BAND:
+            if (value < 0 || value > 120) return EDEN_ERR_INVALID_ARG;
+            ctx->sel_band = value;
+            return EDEN_OK;
+        case EDEN_OPT_SEL_AHEAD:
+            if (value != 0 && value != 1) return EDEN_ERR_INVALID_ARG;
+            ctx->sel_ahead = value;
             return EDEN_OK;
         case EDEN_OPT_SLAB_MIB:
             if (value < 0 || value > 4096) return EDEN_ERR_INVALID_ARG;
@@ -661,6 +678,34 @@ bool two_pass_selection(const eden_ctx* ctx, uint64_t d)
     return mean + 12.0 * std::sqrt(mean) + 64.0 <= (double)kSelCandCap;
 }
 
+// One-pass selection: the keys are independent uniform 32-bit words, so the k-th smallest
+// of d lies near (k/d)*2^32 with a standard deviation of sqrt(p(1-p)/d)*2^32.  The band is
+// that centre plus or minus `tenths`/10 standard deviations, narrowed where the keys it is
+// expected to hold would not fit the candidate list; below three standard deviations the
+// prediction is not worth a pass and the band is left empty (lo > hi), which sends the job
+// to the histogram round.  A wrong prediction costs time, never the result.
+void predicted_band(uint64_t d, uint64_t k, int tenths, uint32_t* lo, uint32_t* hi)
+{
+    *lo = 1u;
+    *hi = 0u;
+    if (d == 0 || k == 0 || k > d || tenths <= 0) return;
+    const double two32 = 4294967296.0;
+    const double p = (double)k / (double)d;
+    const double sd = std::sqrt(p * (1.0 - p) / (double)d) * two32;
+    double half = 0.1 * tenths * sd + 2.0;
+    // expected candidates d * (2 half + 1) / 2^32, kept six of its own deviations under the cap
+    const double room = (double)kSelCandCap - 6.0 * std::sqrt((double)kSelCandCap) - 64.0;
+    const double half_max = (room * two32 / (double)d - 1.0) / 2.0;
+    if (half > half_max) {
+        half = half_max;
+        if (half < 3.0 * sd) return;
+    }
+    const double centre = p * two32;
+    const double a = std::floor(centre - half), b = std::ceil(centre + half);
+    *lo = a < 0.0 ? 0u : (uint32_t)a;
+    *hi = b > two32 - 1.0 ? 0xFFFFFFFFu : (uint32_t)b;
+}
+
 // mask bitmap of one job: 32 words per chunk of 1024 coordinates
 uint64_t keep_bitmap_bytes(uint64_t d)
 {
@@ -678,8 +723,9 @@ uint64_t sel_scratch_bytes(const eden_ctx* ctx, uint64_t d)
 // b < 1) are launched together, split so that each group's work buffers and selection
 // scratch fit the workspace.  Larger dimensions first, so that for the mean a group with
 // b >= 1, which covers every output coordinate, comes before any b < 1 group.
+// `scratch_outside`: the selection scratch of the b < 1 clients lives elsewhere (SelectionAhead).
 int make_groups(const eden_ctx* ctx, const std::vector<ClientPlan>& plan, uint64_t d, uint64_t work_bytes,
-                std::vector<Group>& groups)
+                std::vector<Group>& groups, bool scratch_outside = false)
 {
     std::vector<uint32_t> idx(plan.size());
     for (uint32_t c = 0; c < plan.size(); ++c) idx[c] = c;
@@ -697,7 +743,7 @@ int make_groups(const eden_ctx* ctx, const std::vector<ClientPlan>& plan, uint64
         g.fractional = plan[idx[i]].coin_thr != 0;
         g.uniform = plan[idx[i]].delta > 0.0;
         const uint64_t need = (plan[idx[i]].needs_work ? work_buffer_bytes(plan[idx[i]].D) : 0) +
-                              (g.subbit ? sel_scratch_bytes(ctx, d) : 0);
+                              (g.subbit && !scratch_outside ? sel_scratch_bytes(ctx, d) : 0);
         if (need > work_bytes) return EDEN_ERR_WORKSPACE;
         uint64_t used = 0;
         while (i < idx.size() && plan[idx[i]].L == g.L && plan[idx[i]].subbit == g.subbit &&
@@ -1203,17 +1249,31 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
     batch.grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
     const unsigned hist_grid = (unsigned)(((d + 3) / 4 + (uint64_t)kSelThreads * kSelCallsPerThread - 1) /
                                           ((uint64_t)kSelThreads * kSelCallsPerThread));
+    const bool predict = two_pass && ctx->sel_rounds == 1;
+    if (predict)
+        for (uint32_t j = 0; j < n; ++j) predicted_band(jobs[j].d, jobs[j].k, ctx->sel_band, &jobs[j].lo, &jobs[j].hi);
     CUDA_OK(cudaMemcpyAsync(batch.d_jobs, jobs.data(), sizeof(SelJob) * n, cudaMemcpyHostToDevice, ctx->stream));
-    CUDA_OK(cudaMemsetAsync(hist_base, 0, kBatchHistBytes * n, ctx->stream));
+    // the MaskSelect slots (the fallback flags) and the histograms are contiguous
+    CUDA_OK(cudaMemsetAsync(sel_base, 0, (256ull + kBatchHistBytes) * n, ctx->stream));
     const double keys = (double)n * (double)d;
     if (two_pass) {
         uint32_t* d_status = (uint32_t*)(ctx->ws + fixed_layout(1).status);
-        LAUNCH(ctx, "sel_hist", 0, k_selc_hist, dim3(hist_grid, n), kSelThreads, 0, (const SelJob*)batch.d_jobs);
-        LAUNCH(ctx, "sel_find", n * (double)kSelBins * 4, k_selb_find, n, 1024, 0, (const SelJob*)batch.d_jobs, 0);
-        LAUNCH(ctx, "sel_collect", keys / 128.0, k_selc_collect, dim3(batch.grid, n), kSelThreads, 0,
-               (const SelJob*)batch.d_jobs);
-        LAUNCH(ctx, "sel_resolve", keys / 64.0, k_selc_resolve, n, 1024, 0, (const SelJob*)batch.d_jobs, d_status,
-               (uint64_t)batch.grid);
+        const SelJob* dj = (const SelJob*)batch.d_jobs;
+        const uint64_t n_chunks64 = batch.grid;
+        const unsigned collect_grid = (batch.grid + kSelThreads / 32 - 1) / (kSelThreads / 32);
+        if (predict) {
+            // one pass over the keys; k_selc_redo only does the jobs whose threshold fell outside their band
+            LAUNCH(ctx, "sel_collect", keys / 128.0, k_selc_collect<true>, dim3(collect_grid, n), kSelThreads, 0,
+                   dj, n_chunks64);
+            LAUNCH(ctx, "sel_resolve", keys / 64.0, k_selc_resolve<true>, n, 1024, 0, dj, d_status, n_chunks64);
+            LAUNCH(ctx, "sel_redo", 0, k_selc_redo, n, 1024, 0, dj, d_status, n_chunks64);
+            return EDEN_OK;
+        }
+        LAUNCH(ctx, "sel_hist", 0, k_selc_hist, dim3(hist_grid, n), kSelThreads, 0, dj);
+        LAUNCH(ctx, "sel_find", n * (double)kSelBins * 4, k_selb_find, n, 1024, 0, dj, 0);
+        LAUNCH(ctx, "sel_collect", keys / 128.0, k_selc_collect<false>, dim3(collect_grid, n), kSelThreads, 0,
+               dj, n_chunks64);
+        LAUNCH(ctx, "sel_resolve", keys / 64.0, k_selc_resolve<false>, n, 1024, 0, dj, d_status, n_chunks64);
         return EDEN_OK;
     }
     for (int round = 0; round < 3; ++round) {
@@ -1226,6 +1286,86 @@ int start_selection_batch(eden_ctx* ctx, char* region, uint64_t d, const std::ve
            (uint64_t)batch.grid);
     return EDEN_OK;
 }
+
+// Selection ahead of its use.  The masks of a call's b < 1 clients depend on nothing but
+// (seed, d, k), and finding them is integer arithmetic (the Philox keys) with next to no
+// memory traffic, while the transform passes of the b >= 1 groups, which come first in the
+// processing order, are bound by HBM.  So the selections of all b < 1 groups are enqueued on
+// a side stream when the call starts, with their scratch in an arena at the end of the work
+// region, and the main stream waits for a group's event only when it reaches that group.
+// The launch macros follow ctx->stream, which begin() points at the side stream and end()
+// puts back; the destructor joins the side stream into the main one whatever happened.
+struct SelectionAhead {
+    eden_ctx* ctx;
+    cudaStream_t main;
+    bool on, forked;
+    uint64_t arena_off, arena_bytes;
+    std::vector<SelBatch> batches;       // by group index (empty entries for b >= 1 groups)
+    std::vector<int> event_of;           // by group index: its event in ctx->sel_events, -1 if none
+
+    explicit SelectionAhead(eden_ctx* c) : ctx(c), main(c->stream), on(false), forked(false), arena_off(0), arena_bytes(0) {}
+
+    // Decides whether this call selects ahead and shrinks the work region by the arena.
+    void plan_arena(const std::vector<ClientPlan>& plan, uint64_t d, CallLayout& lay)
+    {
+        uint64_t n_sub = 0;
+        for (const ClientPlan& p : plan) n_sub += p.subbit ? 1 : 0;
+        if (!ctx->sel_ahead || n_sub == 0 || n_sub == plan.size()) return;
+        const uint64_t bytes = n_sub * sel_scratch_bytes(ctx, d);
+        if (bytes >= lay.work_bytes / 2) return;
+        on = true;
+        arena_bytes = bytes;
+        lay.work_bytes -= bytes;
+        arena_off = lay.work_off + lay.work_bytes;
+    }
+    void cancel(CallLayout& lay)
+    {
+        if (!on) return;
+        on = false;
+        lay.work_bytes += arena_bytes;
+    }
+    int begin(size_t n_groups)
+    {
+        batches.assign(n_groups, SelBatch{nullptr, 0, 0, false, {}});
+        event_of.assign(n_groups, -1);
+        if (!ctx->sel_stream && cudaStreamCreateWithFlags(&ctx->sel_stream, cudaStreamNonBlocking) != cudaSuccess) {
+            ctx->sel_stream = nullptr;
+            return EDEN_ERR_CUDA;
+        }
+        while (ctx->sel_events.size() < 2 + n_groups) {
+            cudaEvent_t e;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return EDEN_ERR_CUDA;
+            ctx->sel_events.push_back(e);
+        }
+        // the arena may still be in use by earlier work on the main stream
+        if (cudaEventRecord(ctx->sel_events[0], main) != cudaSuccess ||
+            cudaStreamWaitEvent(ctx->sel_stream, ctx->sel_events[0], 0) != cudaSuccess)
+            return EDEN_ERR_CUDA;
+        forked = true;
+        ctx->stream = ctx->sel_stream;
+        return EDEN_OK;
+    }
+    // group gi's selection has been enqueued
+    int mark(size_t gi)
+    {
+        event_of[gi] = (int)(2 + gi);
+        return cudaEventRecord(ctx->sel_events[2 + gi], ctx->sel_stream) == cudaSuccess ? EDEN_OK : EDEN_ERR_CUDA;
+    }
+    void end() { ctx->stream = main; }
+    // the main stream is about to use group gi's masks
+    int wait(size_t gi)
+    {
+        if (event_of[gi] < 0) return EDEN_ERR_INVALID_ARG;
+        return cudaStreamWaitEvent(main, ctx->sel_events[event_of[gi]], 0) == cudaSuccess ? EDEN_OK : EDEN_ERR_CUDA;
+    }
+    ~SelectionAhead()
+    {
+        ctx->stream = main;
+        if (!forked) return;
+        cudaEventRecord(ctx->sel_events[1], ctx->sel_stream);
+        cudaStreamWaitEvent(main, ctx->sel_events[1], 0);
+    }
+};
 
 }  // namespace
 
@@ -1308,7 +1448,14 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
     rc = carve(ctx, d, n, delta != nullptr, lay);
     if (rc) return rc;
     std::vector<Group> groups;
-    rc = make_groups(ctx, plan, d, lay.work_bytes, groups);
+    SelectionAhead ahead(ctx);
+    ahead.plan_arena(plan, d, lay);
+    rc = make_groups(ctx, plan, d, lay.work_bytes, groups, ahead.on);
+    if (rc == EDEN_ERR_WORKSPACE && ahead.on) {
+        ahead.cancel(lay);
+        groups.clear();
+        rc = make_groups(ctx, plan, d, lay.work_bytes, groups);
+    }
     if (rc) return rc;
     const FixedLayout f = fixed_layout(d);
     const bool x_aligned = ((uintptr_t)x & 15u) == 0 && (ld_x & 3u) == 0;
@@ -1366,26 +1513,55 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
         fold_tiles += (uint64_t)g.members.size() << (g.L > kFastTileLog ? g.L - kFastTileLog : 0);
     }
     fold = fold && fold_tiles <= kFoldMaxTiles;
+    // selection jobs of a b < 1 group; *work_end gets the bytes its work buffers take
+    auto selection_jobs = [&](size_t gi, std::vector<SelJob>& jobs, uint64_t* work_end, uint64_t* kept) {
+        const Group& g = groups[gi];
+        const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
+        jobs.resize(gn);
+        *work_end = 0;
+        *kept = 0;
+        for (uint32_t j = 0; j < gn; ++j) {
+            const ClientPlan& p = plan[g.members[j]];
+            std::memset(&jobs[j], 0, sizeof(SelJob));
+            jobs[j].seed = seeds[p.index];
+            jobs[j].d = d;
+            jobs[j].k = p.k;
+            jobs[j].in = x + (uint64_t)p.index * ld_x;
+            jobs[j].out = descs[first + j].work;
+            *work_end += work_buffer_bytes(p.D);
+            *kept += p.k;
+        }
+    };
+    if (ahead.on) {
+        rc = ahead.begin(groups.size());
+        uint64_t off = ahead.arena_off;
+        for (size_t gi = 0; gi < groups.size() && rc == EDEN_OK; ++gi) {
+            if (!groups[gi].subbit) continue;
+            std::vector<SelJob> jobs;
+            uint64_t work_end, kept;
+            selection_jobs(gi, jobs, &work_end, &kept);
+            rc = start_selection_batch(ctx, ctx->ws + off, d, jobs, ahead.batches[gi]);
+            if (rc == EDEN_OK) rc = ahead.mark(gi);
+            off += groups[gi].members.size() * sel_scratch_bytes(ctx, d);
+        }
+        ahead.end();
+        if (rc) return rc;
+    }
     for (size_t gi = 0; gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
         const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
         if (g.subbit) {
             // exact-size masks of all members, then gather their kept coordinates
-            std::vector<SelJob> jobs(gn);
-            uint64_t work_end = 0, kept = 0;
-            for (uint32_t j = 0; j < gn; ++j) {
-                const ClientPlan& p = plan[g.members[j]];
-                std::memset(&jobs[j], 0, sizeof(SelJob));
-                jobs[j].seed = seeds[p.index];
-                jobs[j].d = d;
-                jobs[j].k = p.k;
-                jobs[j].in = x + (uint64_t)p.index * ld_x;
-                jobs[j].out = descs[first + j].work;
-                work_end += work_buffer_bytes(p.D);
-                kept += p.k;
-            }
+            std::vector<SelJob> jobs;
+            uint64_t work_end, kept;
+            selection_jobs(gi, jobs, &work_end, &kept);
             SelBatch batch;
-            rc = start_selection_batch(ctx, ctx->ws + lay.work_off + work_end, d, jobs, batch);
+            if (ahead.on) {
+                rc = ahead.wait(gi);
+                batch = ahead.batches[gi];
+            } else {
+                rc = start_selection_batch(ctx, ctx->ws + lay.work_off + work_end, d, jobs, batch);
+            }
             if (rc) return rc;
             if (batch.two_pass)
                 LAUNCH(ctx, "sel_compact", 4.0 * gn * (double)d + 4.0 * (double)kept, k_selc_compact,
@@ -1467,7 +1643,14 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
     rc = carve(ctx, d, n, delta != nullptr, lay);
     if (rc) return rc;
     std::vector<Group> groups;
-    rc = make_groups(ctx, plan, d, lay.work_bytes, groups);
+    SelectionAhead ahead(ctx);
+    ahead.plan_arena(plan, d, lay);
+    rc = make_groups(ctx, plan, d, lay.work_bytes, groups, ahead.on);
+    if (rc == EDEN_ERR_WORKSPACE && ahead.on) {
+        ahead.cancel(lay);
+        groups.clear();
+        rc = make_groups(ctx, plan, d, lay.work_bytes, groups);
+    }
     if (rc) return rc;
     const FixedLayout f = fixed_layout(d);
     // the register-blocked last pass moves `out` 16 bytes at a time; a vector that is not
@@ -1537,6 +1720,39 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         CUDA_OK(cudaMemsetAsync(out, 0, d * sizeof(float), ctx->stream));
         written = true;
     }
+    // selection jobs of a b < 1 group; *work_end gets the bytes its work buffers take
+    auto selection_jobs = [&](size_t gi, std::vector<SelJob>& jobs, uint64_t* work_end, uint64_t* kept) {
+        const Group& g = groups[gi];
+        const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
+        jobs.resize(gn);
+        *work_end = 0;
+        *kept = 0;
+        for (uint32_t j = 0; j < gn; ++j) {
+            const ClientPlan& p = plan[g.members[j]];
+            std::memset(&jobs[j], 0, sizeof(SelJob));
+            jobs[j].seed = seeds[p.index];
+            jobs[j].d = d;
+            jobs[j].k = p.k;
+            jobs[j].in = descs[first + j].work;
+            *work_end += work_buffer_bytes(p.D);
+            *kept += p.k;
+        }
+    };
+    if (ahead.on) {
+        rc = ahead.begin(groups.size());
+        uint64_t off = ahead.arena_off;
+        for (size_t gi = 0; gi < groups.size() && rc == EDEN_OK; ++gi) {
+            if (!groups[gi].subbit) continue;
+            std::vector<SelJob> jobs;
+            uint64_t work_end, kept;
+            selection_jobs(gi, jobs, &work_end, &kept);
+            rc = start_selection_batch(ctx, ctx->ws + off, d, jobs, ahead.batches[gi]);
+            if (rc == EDEN_OK) rc = ahead.mark(gi);
+            off += groups[gi].members.size() * sel_scratch_bytes(ctx, d);
+        }
+        ahead.end();
+        if (rc) return rc;
+    }
     for (size_t gi = 0; gi < groups.size(); ++gi) {
         const Group& g = groups[gi];
         const uint32_t first = group_start[gi], gn = (uint32_t)g.members.size();
@@ -1546,19 +1762,15 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         if (g.subbit) {
             // exact-size masks of all members (the estimates of their kept coordinates will
             // be written to their work buffers and scattered from there)
-            std::vector<SelJob> jobs(gn);
-            uint64_t work_end = 0;
-            for (uint32_t j = 0; j < gn; ++j) {
-                const ClientPlan& p = plan[g.members[j]];
-                std::memset(&jobs[j], 0, sizeof(SelJob));
-                jobs[j].seed = seeds[p.index];
-                jobs[j].d = d;
-                jobs[j].k = p.k;
-                jobs[j].in = descs[first + j].work;
-                work_end += work_buffer_bytes(p.D);
-                kept += p.k;
+            std::vector<SelJob> jobs;
+            uint64_t work_end;
+            selection_jobs(gi, jobs, &work_end, &kept);
+            if (ahead.on) {
+                rc = ahead.wait(gi);
+                batch = ahead.batches[gi];
+            } else {
+                rc = start_selection_batch(ctx, ctx->ws + lay.work_off + work_end, d, jobs, batch);
             }
-            rc = start_selection_batch(ctx, ctx->ws + lay.work_off + work_end, d, jobs, batch);
             if (rc) return rc;
         }
         // with OUT_YHAT every member writes its own estimate: one block row per member

@@ -48,7 +48,8 @@ struct MaskSelect {
     uint32_t tau;
     uint32_t rem;
     uint32_t below;          // keys < tau
-    uint32_t pad[3];
+    uint32_t fallback;       // one-pass selection: tau was outside the predicted band, redo with the histogram round
+    uint32_t pad[2];
 };
 
 // ----------------------------------------------------------------------------------

@@ -9,7 +9,8 @@
 // 1024-coordinate chunk counts, a scan of the chunk counts, and a scan inside each chunk.
 // Three forms: single-job kernels with two 16-bit histogram rounds (the mask entry points),
 // batched kernels with three digit rounds over all keys (long vectors), and the batched
-// two-pass form with a candidate list and a mask bitmap (the default).
+// form with a candidate list and a mask bitmap (the default), which reads the keys once
+// where the threshold falls inside the band predicted for it and twice otherwise.
 #pragma once
 #include "eden_device.cuh"
 
@@ -218,6 +219,7 @@ struct SelJob {
     float* out;                      // compact: the compacted vector
     uint2* cand;                     // two-pass selection: (key, coordinate) of the keys that share tau's first digit
     uint32_t* keep;                  // two-pass selection: the mask as a bitmap (bit i % 32 of word i / 32)
+    uint32_t lo, hi;                 // one-pass selection: the band of keys predicted to hold tau (empty if lo > hi)
 };
 
 // Batched selection finds the k-th smallest key in three digit rounds of 10, 11 and 11
@@ -368,21 +370,29 @@ k_selb_chunk_scan(const SelJob* __restrict__ jobs, uint64_t n_chunks)
 }
 
 // ---------------------------------------------------------------------------------
-// Two-pass selection (vectors short enough for the candidate list, kSelCandCap).  The
-// first digit of tau, the top 11 bits, comes from one histogram round as above.  The second
-// pass over the keys does two things at once: it counts, per chunk of 1024 coordinates, the
-// keys whose first digit is smaller (they are below tau whatever its other bits are), and it
-// appends the keys that share the digit, about one in 2048, to the job's candidate list with
-// their coordinates; the coordinates of the first kind are also marked in the job's mask
-// bitmap.  One block per job then finds tau's remaining 21 bits among the candidates alone
-// and, for each candidate that is kept (below tau, or equal to it and among the first `rem`
-// such coordinates), sets its bit and adds it to its chunk's count.  Compaction and scatter
-// read the bitmap, so the keys are generated twice per side (histogram, this pass) instead
-// of five times.  job.hist[kSelBins] counts the candidates (zeroed with the histograms).
+// Selection with a candidate list (vectors short enough for it, kSelCandCap).
+//
+// Keys below a band [lo, hi] that is known to hold tau are kept whatever tau's exact value
+// is: one pass over the keys counts them per chunk of 1024 coordinates and marks them in
+// the job's mask bitmap, and appends the keys inside the band to the job's candidate list
+// with their coordinates.  One block per job then finds tau among the candidates alone and,
+// for each candidate that is kept (below tau, or equal to it and among the first `rem` such
+// coordinates), sets its bit and adds it to its chunk's count.  Compaction and scatter read
+// the bitmap.  job.hist[kSelBins] counts the candidates (zeroed with the histograms).
+//
+// Where the band comes from:
+//  * predicted (the default): the keys are uniform, so the k-th smallest of d is close to
+//    (k/d) 2^32; the host puts a band of a few standard deviations around it and the keys
+//    are generated once per side.  If tau turns out to lie outside (or the list overflows)
+//    the job is flagged and k_selc_redo does it again the second way, one block per job:
+//    slow, but it runs about once in 10^4 jobs, and the mask is the same either way.
+//  * from a histogram round: the bin of tau's top 11 bits (one key in 2048 is a candidate);
+//    the keys are generated twice per side.
 // ---------------------------------------------------------------------------------
 constexpr int kSelFirstShift = 21;                     // first digit = key >> 21 (11 bits, kSelBins bins)
 constexpr uint32_t kSelCandCap = 61440;                // candidates a job can hold (480 KB)
 constexpr uint32_t kStatusScratch = 0x10u;             // EDEN_STATUS_SCRATCH
+constexpr int kSelDigitBins = 4096;                    // bins of a digit round among the candidates
 
 __global__ void __launch_bounds__(kSelThreads)
 k_selc_hist(const SelJob* __restrict__ jobs)
@@ -408,118 +418,186 @@ k_selc_hist(const SelJob* __restrict__ jobs)
         if (s_hist[b]) atomicAdd(&job.hist[b], s_hist[b]);
 }
 
-__global__ void __launch_bounds__(kSelThreads)
-k_selc_collect(const SelJob* __restrict__ jobs)
+// One warp, one chunk of 1024 coordinates: lane l takes the eight Philox calls of the
+// chunk's bitmap word l, builds the word in a register, and the warp adds up the counts;
+// nothing goes through shared memory or a block barrier.
+__device__ __forceinline__ void collect_chunk(const SelJob& job, uint64_t chunk, uint32_t lo, uint32_t hi)
 {
-    __shared__ unsigned long long scratch[33];
-    const SelJob job = jobs[blockIdx.y];
-    const uint32_t digit = job.sel->bin_hi;
-    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const uint4 k4 = mask_keys(job.seed, t);
-    const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
-    unsigned long long mine = 0;
-    uint32_t nibble = 0u;
+    const uint32_t lane = threadIdx.x & 31u;
+    const bool empty = lo > hi;
+    uint32_t word = 0u;
+    const uint64_t t0 = chunk * (kSelChunk / 4) + lane * 8u;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const uint64_t i = t * 4 + j;
-        if (i >= job.d) break;
-        const uint32_t top = keys[j] >> kSelFirstShift;
-        if (top < digit) {
-            ++mine;
-            nibble |= 1u << j;
-        } else if (top == digit) {
-            const uint32_t slot = atomicAdd(&job.hist[kSelBins], 1u);
-            if (slot < kSelCandCap) job.cand[slot] = make_uint2(keys[j], (uint32_t)i);
+    for (int c = 0; c < 8; ++c) {
+        const uint64_t t = t0 + c;
+        if (t * 4 >= job.d) break;
+        const uint4 k4 = mask_keys(job.seed, t);
+        const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint64_t i = t * 4 + j;
+            if (i >= job.d) break;
+            if (keys[j] < lo) {
+                word |= 1u << (4 * c + j);
+            } else if (keys[j] <= hi && !empty) {
+                const uint32_t slot = atomicAdd(&job.hist[kSelBins], 1u);
+                if (slot < kSelCandCap) job.cand[slot] = make_uint2(keys[j], (uint32_t)i);
+            }
         }
     }
-    // eight threads hold the 32 coordinates of one bitmap word
-    uint32_t word = nibble << (4 * (threadIdx.x & 7));
-    word |= __shfl_xor_sync(0xffffffffu, word, 1);
-    word |= __shfl_xor_sync(0xffffffffu, word, 2);
-    word |= __shfl_xor_sync(0xffffffffu, word, 4);
-    if ((threadIdx.x & 7) == 0) job.keep[t >> 3] = word;
-    unsigned long long total;
-    block_exclusive_scan(mine, scratch, &total);
-    if (threadIdx.x == 0) job.chunks[blockIdx.x] = total;
+    job.keep[chunk * 32u + lane] = word;
+    const uint32_t count = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(word));
+    if (lane == 0) job.chunks[chunk] = count;
 }
 
-// One block of 1024 threads per job; ends with the exclusive scan of the job's chunk counts
-// (the positions compaction and scatter start from).
-__global__ void __launch_bounds__(1024)
-k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status, uint64_t n_chunks)
+// PREDICTED: the band is job.lo .. job.hi; otherwise the bin of the digit in sel->bin_hi.
+template <bool PREDICTED>
+__global__ void __launch_bounds__(kSelThreads)
+k_selc_collect(const SelJob* __restrict__ jobs, uint64_t n_chunks)
 {
-    __shared__ uint32_t s_hist[kSelBins];
-    __shared__ unsigned long long scratch[33];
-    __shared__ uint32_t s_bin, s_before;
-    const SelJob job = jobs[blockIdx.x];
+    const SelJob job = jobs[blockIdx.y];
+    const uint64_t chunk = (uint64_t)blockIdx.x * (kSelThreads / 32) + (threadIdx.x >> 5);
+    if (chunk >= n_chunks) return;
+    const uint32_t lo = PREDICTED ? job.lo : job.sel->bin_hi << kSelFirstShift;
+    const uint32_t hi = PREDICTED ? job.hi : lo | ((1u << kSelFirstShift) - 1u);
+    collect_chunk(job, chunk, lo, hi);
+}
+
+// A block's walk over a job's candidate list, eight loads in flight per thread (one block
+// per job: the walk is bound by the latency of the loads, not by their number).
+template <class F>
+__device__ __forceinline__ void for_each_candidate(const SelJob& job, uint32_t n, F f)
+{
+    for (uint32_t c0 = threadIdx.x; c0 < n; c0 += 8u * blockDim.x) {
+        uint2 kc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t c = c0 + u * blockDim.x;
+            kc[u] = c < n ? __ldcg(&job.cand[c]) : make_uint2(0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (c0 + u * blockDim.x < n) f(kc[u]);
+    }
+}
+
+// Sum of the job's chunk counts (SCAN: replaced in place by their exclusive prefix sums),
+// thread t taking a contiguous run, eight loads in flight.  Whole block.
+template <bool SCAN>
+__device__ __forceinline__ unsigned long long chunk_counts_sum(const SelJob& job, uint64_t n_chunks,
+                                                               unsigned long long* scan_scratch)
+{
+    const uint64_t per = (n_chunks + blockDim.x - 1) / blockDim.x;
+    const uint64_t c0 = min((uint64_t)threadIdx.x * per, n_chunks), c1 = min(c0 + per, n_chunks);
+    unsigned long long mine = 0;
+    for (uint64_t j0 = c0; j0 < c1; j0 += 8) {
+        unsigned long long v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = j0 + u < c1 ? __ldcg(&job.chunks[j0 + u]) : 0ull;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) mine += v[u];
+    }
+    unsigned long long total;
+    unsigned long long run = block_exclusive_scan(mine, scan_scratch, &total);
+    if (SCAN) {
+        for (uint64_t j0 = c0; j0 < c1; j0 += 8) {
+            unsigned long long v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = j0 + u < c1 ? __ldcg(&job.chunks[j0 + u]) : 0ull;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (j0 + u < c1) job.chunks[j0 + u] = run;
+                run += v[u];
+            }
+        }
+    }
+    return total;
+}
+
+// Scratch of the block that resolves a job (1024 threads).
+struct ResolveShared {
+    uint32_t hist[kSelDigitBins];
+    unsigned long long scan[33];
+    uint32_t ties[256];
+    uint32_t bin, before, n_ties;
+};
+
+// Finds tau among the job's n candidates, all of which lie in [base, base + 2^width), given
+// that `below` keys are smaller than every candidate; marks the kept candidates; scans the
+// chunk counts into positions.  The offset of tau inside the band is settled from the top
+// in one to three digits of at most 12 bits each.  Whole block, 1024 threads.
+__device__ __forceinline__ void resolve_job(const SelJob& job, ResolveShared& sh, uint32_t n, uint32_t base,
+                                            int width, uint32_t below, uint64_t n_chunks)
+{
     MaskSelect* sel = job.sel;
-    const uint32_t found = job.hist[kSelBins];
-    const uint32_t n = min(found, kSelCandCap);
-    if (found > kSelCandCap && threadIdx.x == 0) atomicOr(status, kStatusScratch);
-    const uint32_t digit = sel->bin_hi;
-    uint32_t below = sel->below_hi;                    // keys below everything fixed so far
-    uint32_t prefix = digit;                           // the bits of tau fixed so far
-    int fixed = 32 - kSelFirstShift;                   // how many they are
-    // the remaining 21 bits in two digits of 11 and 10 bits
-    for (int round = 0; round < 2; ++round) {
-        const int bits = round == 0 ? 11 : 10;
-        const int shift = 32 - fixed - bits;
-        for (int b = threadIdx.x; b < kSelBins; b += blockDim.x) s_hist[b] = 0u;
-        if (threadIdx.x == 0) { s_bin = 0u; s_before = 0u; }
+    const int rounds = (width + 11) / 12;
+    const int per_round = rounds ? (width + rounds - 1) / rounds : 0;
+    uint32_t prefix = 0u;                              // the bits of tau - base fixed so far
+    int fixed = 0;                                     // how many they are
+    while (fixed < width) {
+        const int bits = width - fixed < per_round ? width - fixed : per_round;
+        const int shift = width - fixed - bits;
+        for (int b = threadIdx.x; b < kSelDigitBins; b += blockDim.x) sh.hist[b] = 0u;
+        if (threadIdx.x == 0) { sh.bin = 0u; sh.before = 0u; }
         __syncthreads();
-        for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
-            const uint32_t key = job.cand[c].x;
-            if ((key >> (shift + bits)) == prefix) atomicAdd(&s_hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
-        }
+        for_each_candidate(job, n, [&](uint2 kc) {
+            const uint32_t rel = kc.x - base;
+            if (fixed == 0 || (rel >> (shift + bits)) == prefix)
+                atomicAdd(&sh.hist[(rel >> shift) & ((1u << bits) - 1u)], 1u);
+        });
         __syncthreads();
-        // thread t owns bins 2t and 2t + 1; the rank looked for is k - 1 - below
+        // thread t owns bins 4t .. 4t + 3; the rank looked for is k - 1 - below
         const uint32_t r = (uint32_t)(job.k - 1) - below;
-        const uint32_t v0 = s_hist[2 * threadIdx.x], v1 = s_hist[2 * threadIdx.x + 1];
+        uint32_t v[4], mine = 0u;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { v[i] = sh.hist[4 * threadIdx.x + i]; mine += v[i]; }
         unsigned long long total;
-        const uint32_t before = (uint32_t)block_exclusive_scan((unsigned long long)(v0 + v1), scratch, &total);
-        if (r >= before && r < before + v0 + v1) {     // exactly one thread
-            const bool second = r >= before + v0;
-            s_bin = 2 * threadIdx.x + (second ? 1u : 0u);
-            s_before = before + (second ? v0 : 0u);
+        uint32_t before = (uint32_t)block_exclusive_scan((unsigned long long)mine, sh.scan, &total);
+        if (r >= before && r < before + mine) {        // exactly one thread
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (r >= before && r < before + v[i]) {
+                    sh.bin = 4 * threadIdx.x + i;
+                    sh.before = before;
+                }
+                before += v[i];
+            }
         }
         __syncthreads();
-        prefix = (prefix << bits) | s_bin;
-        below += s_before;
+        prefix = (prefix << bits) | sh.bin;
+        below += sh.before;
         fixed += bits;
         __syncthreads();
     }
-    const uint32_t tau = prefix;
+    const uint32_t tau = base + prefix;
+    const uint32_t rem = (uint32_t)job.k - below;      // ties to keep, >= 1
     if (threadIdx.x == 0) {
         sel->tau = tau;
         sel->below = below;
-        sel->rem = (uint32_t)job.k - below;            // ties to keep, >= 1
+        sel->rem = rem;
+        sh.n_ties = 0u;
     }
+    __syncthreads();
     // the candidates that are kept: below tau, or equal to it with fewer than `rem` equal
     // keys at smaller coordinates.  Equal keys are rare, so their coordinates are gathered
     // in shared memory and ranked there; a list that does not fit is ranked in place.
     constexpr uint32_t kTieCap = 256;
-    __shared__ uint32_t s_ties[kTieCap];
-    __shared__ uint32_t s_nties;
-    const uint32_t rem = (uint32_t)job.k - below;
-    if (threadIdx.x == 0) s_nties = 0u;
-    __syncthreads();
-    for (uint32_t c = threadIdx.x; c < n; c += blockDim.x) {
-        const uint2 kc = job.cand[c];
+    for_each_candidate(job, n, [&](uint2 kc) {
         if (kc.x < tau) {
             atomicOr(&job.keep[kc.y >> 5], 1u << (kc.y & 31u));
             atomicAdd(&job.chunks[kc.y >> 10], 1ull);
         } else if (kc.x == tau) {
-            const uint32_t slot = atomicAdd(&s_nties, 1u);
-            if (slot < kTieCap) s_ties[slot] = kc.y;
+            const uint32_t slot = atomicAdd(&sh.n_ties, 1u);
+            if (slot < kTieCap) sh.ties[slot] = kc.y;
         }
-    }
+    });
     __syncthreads();
-    const uint32_t n_ties = s_nties;
+    const uint32_t n_ties = sh.n_ties;
     if (n_ties <= kTieCap) {
         for (uint32_t i = threadIdx.x; i < n_ties; i += blockDim.x) {
-            const uint32_t coord = s_ties[i];
+            const uint32_t coord = sh.ties[i];
             uint32_t before = 0;
-            for (uint32_t o = 0; o < n_ties; ++o) before += s_ties[o] < coord ? 1u : 0u;
+            for (uint32_t o = 0; o < n_ties; ++o) before += sh.ties[o] < coord ? 1u : 0u;
             if (before < rem) {
                 atomicOr(&job.keep[coord >> 5], 1u << (coord & 31u));
                 atomicAdd(&job.chunks[coord >> 10], 1ull);
@@ -542,17 +620,88 @@ k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status, u
     }
     // every count is final: scan them in place (reads from L2, where the atomics landed)
     __syncthreads();
-    const uint64_t per = (n_chunks + blockDim.x - 1) / blockDim.x;
-    const uint64_t lo = min((uint64_t)threadIdx.x * per, n_chunks), hi = min(lo + per, n_chunks);
-    unsigned long long mine = 0;
-    for (uint64_t j = lo; j < hi; ++j) mine += __ldcg(&job.chunks[j]);
-    unsigned long long total;
-    unsigned long long run = block_exclusive_scan(mine, scratch, &total);
-    for (uint64_t j = lo; j < hi; ++j) {
-        const unsigned long long v = __ldcg(&job.chunks[j]);
-        job.chunks[j] = run;
-        run += v;
+    chunk_counts_sum<true>(job, n_chunks, sh.scan);
+}
+
+// One block of 1024 threads per job, behind k_selc_collect.  PREDICTED: the keys below the
+// band are the sum of the chunk counts; the prediction holds if the list did not overflow
+// and the rank looked for falls among the candidates.  If it does not, the job is flagged
+// for k_selc_redo and its candidate counter is cleared.
+template <bool PREDICTED>
+__global__ void __launch_bounds__(1024)
+k_selc_resolve(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status, uint64_t n_chunks)
+{
+    __shared__ ResolveShared sh;
+    const SelJob job = jobs[blockIdx.x];
+    MaskSelect* sel = job.sel;
+    const uint32_t found = job.hist[kSelBins];
+    if (!PREDICTED) {
+        if (found > kSelCandCap && threadIdx.x == 0) atomicOr(status, kStatusScratch);
+        resolve_job(job, sh, min(found, kSelCandCap), sel->bin_hi << kSelFirstShift, kSelFirstShift, sel->below_hi,
+                    n_chunks);
+        return;
     }
+    const unsigned long long total = chunk_counts_sum<false>(job, n_chunks, sh.scan);
+    const bool holds = found <= kSelCandCap && job.k >= 1 && total <= job.k - 1 && job.k - 1 - total < (uint64_t)found;
+    if (!holds) {
+        if (threadIdx.x == 0) {
+            sel->fallback = 1u;
+            job.hist[kSelBins] = 0u;
+        }
+        return;
+    }
+    resolve_job(job, sh, found, job.lo, 32 - __clz(job.hi - job.lo), (uint32_t)total, n_chunks);
+}
+
+// The jobs whose prediction failed, one block of 1024 threads per job, every step of the
+// histogram form inside the block: first-digit histogram over all keys, the digit that holds
+// rank k - 1, the collecting pass, the candidates.  Every other job returns at once.
+__global__ void __launch_bounds__(1024)
+k_selc_redo(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status, uint64_t n_chunks)
+{
+    __shared__ ResolveShared sh;
+    const SelJob job = jobs[blockIdx.x];
+    MaskSelect* sel = job.sel;
+    if (!sel->fallback) return;
+    static_assert(kSelBins <= kSelDigitBins, "the first-digit histogram uses the resolve scratch");
+    for (int b = threadIdx.x; b < kSelBins; b += blockDim.x) sh.hist[b] = 0u;
+    if (threadIdx.x == 0) { sh.bin = 0u; sh.before = 0u; }
+    __syncthreads();
+    const uint64_t calls = (job.d + 3) / 4;
+    for (uint64_t t = threadIdx.x; t < calls; t += blockDim.x) {
+        const uint4 k4 = mask_keys(job.seed, t);
+        const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (t * 4 + j < job.d) atomicAdd(&sh.hist[keys[j] >> kSelFirstShift], 1u);
+    }
+    __syncthreads();
+    {
+        // thread t owns bins 2t and 2t + 1
+        const uint32_t r = (uint32_t)(job.k - 1);
+        const uint32_t v0 = sh.hist[2 * threadIdx.x], v1 = sh.hist[2 * threadIdx.x + 1];
+        unsigned long long total;
+        const uint32_t before = (uint32_t)block_exclusive_scan((unsigned long long)(v0 + v1), sh.scan, &total);
+        if (r >= before && r < before + v0 + v1) {     // exactly one thread (none if k = 0)
+            const bool second = r >= before + v0;
+            sh.bin = 2 * threadIdx.x + (second ? 1u : 0u);
+            sh.before = before + (second ? v0 : 0u);
+        }
+        __syncthreads();
+    }
+    const uint32_t digit = sh.bin, below = sh.before;
+    if (threadIdx.x == 0) {
+        sel->bin_hi = digit;
+        sel->below_hi = below;
+    }
+    const uint32_t lo = digit << kSelFirstShift, hi = lo | ((1u << kSelFirstShift) - 1u);
+    for (uint64_t chunk = threadIdx.x >> 5; chunk < n_chunks; chunk += blockDim.x >> 5)
+        collect_chunk(job, chunk, lo, hi);
+    __threadfence();
+    __syncthreads();
+    const uint32_t found = __ldcg(&job.hist[kSelBins]);
+    if (found > kSelCandCap && threadIdx.x == 0) atomicOr(status, kStatusScratch);
+    resolve_job(job, sh, min(found, kSelCandCap), lo, kSelFirstShift, below, n_chunks);
 }
 
 // Position, among the kept coordinates of the block's chunk of 1024, of the first kept

@@ -85,7 +85,7 @@ _sig("eden_profile_get", _int, [_vp, _u32, ctypes.POINTER(ctypes.c_char_p), ctyp
                                 ctypes.POINTER(_f64), ctypes.POINTER(_f64)])
 
 STATUS_ZERO_VECTOR, STATUS_NONFINITE, STATUS_NO_DATA, STATUS_TIMEOUT, STATUS_SCRATCH = 1, 2, 4, 8, 16
-OPT_PLAN_VARIANT, OPT_ROW_STAGING, OPT_SEL_ROUNDS, OPT_SLAB_MIB, OPT_SLAB_STREAMS, OPT_SLAB_SIDES = 1, 2, 3, 4, 5, 6
+OPT_PLAN_VARIANT, OPT_ROW_STAGING, OPT_SEL_ROUNDS, OPT_SLAB_MIB, OPT_SLAB_STREAMS, OPT_SLAB_SIDES, OPT_SEL_BAND, OPT_SEL_AHEAD = 1, 2, 3, 4, 5, 6, 7, 8
 PACKET_COORDS = 1024
 UNIFORM_MAX_INDEX = 127
 UNIFORM_MIN_DELTA = 0.0625
@@ -401,7 +401,7 @@ class Context:
         _check(_lib.eden_force_generic_kernels(self._h, 1 if on else 0))
 
     def set_option(self, option: int, value: int):
-        """eden_set_option: OPT_PLAN_VARIANT / OPT_ROW_STAGING / OPT_SEL_ROUNDS."""
+        """eden_set_option: one of the OPT_* switches of this module."""
         _check(_lib.eden_set_option(self._h, int(option), int(value)))
 
     def profile(self, on: bool):

@@ -274,7 +274,22 @@ def test_sub_bit_selection_in_three_histogram_rounds(E, bits, d):
     run_workload(E, work, options=[(E.OPT_SEL_ROUNDS, 3)])
 
 
-@pytest.mark.parametrize("rounds", [2, 3])
+@pytest.mark.parametrize("band", [50, 10, 0])
+@pytest.mark.parametrize("bits,d", [(0.1, 200003), (0.5, 70001), (0.9, 9), (0.25, (1 << 21) + 77), (0.01, 50)])
+def test_sub_bit_selection_with_a_predicted_band(E, bits, d, band):
+    # the default form reads the keys once and keeps those inside a band predicted for the
+    # threshold; a job whose threshold is outside is redone with the histogram round.  Five
+    # standard deviations (the default): the prediction holds; one: it fails for about a third
+    # of the clients, so one call mixes both; empty band: every client is redone.  The masks
+    # and everything that follows from them must equal the oracle's in all three.
+    n = 6
+    rng = np.random.default_rng(d + band)
+    xs = rng.standard_normal((n, d)).astype(np.float32)
+    work = synth.Workload("adhoc", n, d, np.full(n, bits), synth.client_seeds(d + 3 + band, n), 0.0, lambda c: xs[c], d)
+    run_workload(E, work, check_clients=range(n), options=[(E.OPT_SEL_ROUNDS, 1), (E.OPT_SEL_BAND, band)])
+
+
+@pytest.mark.parametrize("rounds", [1, 2, 3])
 @pytest.mark.parametrize("which,extra", [(0, 1), (1, 2), (2, 1)])
 def test_mask_threshold_on_a_pair_of_equal_keys(E, which, extra, rounds):
     # Section 4.1 asks for a sample of exactly d*p coordinates.  With seed 1 and d = 2^17 three
@@ -327,13 +342,31 @@ def test_many_small_clients(E):
     run_workload(E, work)
 
 
-def test_mixed_budgets_in_one_call(E):
-    d, n = 50000, 7
+@pytest.mark.parametrize("ahead", [1, 0])
+@pytest.mark.parametrize("d", [50000, (1 << 20) + 17])
+def test_mixed_budgets_in_one_call(E, d, ahead):
+    # budgets below and above one bit in one call: by default the b < 1 senders' masks are
+    # selected on a side stream while the other senders' passes run (ahead = 1); in line
+    # otherwise.  Two calls in a row on one context, so that the second call's side stream
+    # has to wait for the first call's use of the same scratch.
+    n = 9
     rng = np.random.default_rng(5)
     xs = rng.standard_normal((n, d)).astype(np.float32)
-    bits = np.array([0.3, 1.0, 2.0, 0.1, 4.0, 8.0, 1.5])
+    bits = np.array([0.3, 1.0, 2.0, 0.1, 4.0, 8.0, 1.5, 0.3, 0.75])
     work = synth.Workload("adhoc", n, d, bits, synth.client_seeds(9, n), 0.2, lambda c: xs[c], 9)
-    run_workload(E, work)
+    run_workload(E, work, options=[(E.OPT_SEL_AHEAD, ahead)])
+    ctx = _ctx(E, d, n)
+    ctx.set_option(E.OPT_SEL_AHEAD, ahead)
+    x_gpu = torch.from_numpy(xs).cuda()
+    zeros = lambda: [torch.zeros(E.code_bytes(d, float(b)), dtype=torch.uint8, device="cuda") for b in bits]
+    first = ctx.encode(x_gpu, bits, work.seeds, codes=zeros())
+    again = ctx.encode(x_gpu, bits, work.seeds, codes=zeros())
+    torch.cuda.synchronize()
+    assert ctx.status() == 0
+    for a, b in zip(first[0], again[0]):
+        assert torch.equal(a, b)
+    assert torch.equal(first[1], again[1])
+    ctx.close()
 
 
 def test_generic_kernels_agree_with_the_oracle_on_large_shapes(E):
@@ -422,7 +455,7 @@ def test_all_packets_lost_is_reported_not_fatal(E, d):
 
 def test_options_are_checked(E):
     ctx = _ctx(E, 1024, 1)
-    for opt, bad in ((E.OPT_PLAN_VARIANT, 4), (E.OPT_ROW_STAGING, 2), (E.OPT_SEL_ROUNDS, 1), (E.OPT_SLAB_MIB, -1),
+    for opt, bad in ((E.OPT_PLAN_VARIANT, 4), (E.OPT_ROW_STAGING, 2), (E.OPT_SEL_ROUNDS, 0), (E.OPT_SEL_ROUNDS, 4), (E.OPT_SEL_BAND, 121), (E.OPT_SEL_BAND, -1), (E.OPT_SEL_AHEAD, 2), (E.OPT_SLAB_MIB, -1),
                      (E.OPT_SLAB_STREAMS, 0), (E.OPT_SLAB_SIDES, 4), (99, 0)):
         with pytest.raises(E.EdenError) as e:
             ctx.set_option(opt, bad)
