@@ -1565,7 +1565,8 @@ int encode_common(eden_ctx* ctx, const float* x, uint64_t ld_x, uint64_t d, uint
             if (rc) return rc;
             if (batch.two_pass)
                 LAUNCH(ctx, "sel_compact", 4.0 * gn * (double)d + 4.0 * (double)kept, k_selc_compact,
-                       dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
+                       dim3((batch.grid + kSelThreads / 32 - 1) / (kSelThreads / 32), gn), kSelThreads, 0,
+                       (const SelJob*)batch.d_jobs, (uint64_t)batch.grid);
             else
                 LAUNCH(ctx, "sel_compact", 4.0 * gn * (double)d + 4.0 * (double)kept, k_selb_compact,
                        dim3(batch.grid, gn), kSelThreads, 0, (const SelJob*)batch.d_jobs);
@@ -1825,8 +1826,9 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
         }
         if (g.subbit) {
             if (batch.two_pass)
-                LAUNCH(ctx, "sel_scatter", 8.0 * (double)kept + 4.0 * (double)kept, k_selc_scatter, batch.grid,
-                       kSelThreads, 0, (const SelJob*)batch.d_jobs, gn, d, out);
+                LAUNCH(ctx, "sel_scatter", 8.0 * (double)kept + 4.0 * (double)kept, k_selc_scatter,
+                       (batch.grid + kSelThreads / 32 - 1) / (kSelThreads / 32), kSelThreads, 0,
+                       (const SelJob*)batch.d_jobs, gn, d, out, (uint64_t)batch.grid);
             else
                 LAUNCH(ctx, "sel_scatter", 8.0 * (double)kept + 4.0 * (double)kept, k_selb_scatter, batch.grid,
                        kSelThreads, 0, (const SelJob*)batch.d_jobs, gn, d, out);

@@ -704,69 +704,126 @@ k_selc_redo(const SelJob* __restrict__ jobs, uint32_t* __restrict__ status, uint
     resolve_job(job, sh, min(found, kSelCandCap), lo, kSelFirstShift, below, n_chunks);
 }
 
-// Position, among the kept coordinates of the block's chunk of 1024, of the first kept
-// coordinate of thread t's four (coordinates 4t .. 4t + 3), and the thread's four mask bits.
-// Every warp reads the chunk's 32 bitmap words (lane l word l), scans their population
-// counts with shuffles and hands each thread the count before its word; the bits below the
-// thread's nibble inside the word complete it.  No shared memory, no block barrier.
-__device__ __forceinline__ uint32_t keep_position(const uint32_t* __restrict__ keep, uint32_t& nibble)
+// One warp walks one chunk of 1024 coordinates in eight pieces of 128, lane l taking the
+// four coordinates 128 i + 4 l .. + 3 of piece i, so that the vector accesses of a piece are
+// one contiguous 512 bytes.  Lane l also holds the chunk's bitmap word l; a shuffle scan of
+// the population counts gives the kept coordinates before each word.
+struct ChunkMask {
+    uint32_t word;      // bitmap word `lane` of the chunk
+    uint32_t before;    // kept coordinates of the chunk in the words below it
+};
+
+__device__ __forceinline__ ChunkMask chunk_mask(const uint32_t* __restrict__ keep, uint64_t chunk)
 {
     const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t word = keep[(uint64_t)blockIdx.x * 32u + lane];
-    uint32_t inc = (uint32_t)__popc(word);
+    ChunkMask m;
+    m.word = keep[chunk * 32u + lane];
+    uint32_t inc = (uint32_t)__popc(m.word);
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
         if (lane >= (uint32_t)o) inc += v;
     }
-    const uint32_t w = threadIdx.x >> 3;                          // the thread's word in the chunk
-    const uint32_t mine = __shfl_sync(0xffffffffu, word, w);
-    const uint32_t before = __shfl_sync(0xffffffffu, inc, w) - (uint32_t)__popc(mine);
-    const uint32_t shift = 4u * (threadIdx.x & 7u);
-    nibble = (mine >> shift) & 0xFu;
-    return before + (uint32_t)__popc(mine & ((1u << shift) - 1u));
+    m.before = inc - (uint32_t)__popc(m.word);
+    return m;
+}
+
+// The lane's four mask bits in piece i and the position, among the chunk's kept coordinates,
+// of the first of them that is kept.
+__device__ __forceinline__ uint32_t piece_position(const ChunkMask& m, int i, uint32_t& nibble)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const int w = 4 * i + (int)(lane >> 3);                       // the word that holds the lane's nibble
+    const uint32_t word = __shfl_sync(0xffffffffu, m.word, w);
+    const uint32_t before = __shfl_sync(0xffffffffu, m.before, w);
+    const uint32_t shift = 4u * (lane & 7u);
+    nibble = (word >> shift) & 0xFu;
+    return before + (uint32_t)__popc(word & ((1u << shift) - 1u));
 }
 
 // Sender: y_c[pos] = x_c[i] for the kept coordinates of every job, from the bitmap.
 __global__ void __launch_bounds__(kSelThreads)
-k_selc_compact(const SelJob* __restrict__ jobs)
+k_selc_compact(const SelJob* __restrict__ jobs, uint64_t n_chunks)
 {
     const SelJob job = jobs[blockIdx.y];
-    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    uint32_t nib;
-    uint64_t pos = keep_position(job.keep, nib) + job.chunks[blockIdx.x];
-    if (((uintptr_t)job.in & 15u) == 0 && t * 4 + 3 < job.d) {
-        // one coalesced 16-byte load per thread, whatever the mask keeps
-        const float4 x4 = *reinterpret_cast<const float4*>(job.in + t * 4);
-        const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t chunk = (uint64_t)blockIdx.x * (kSelThreads / 32) + (threadIdx.x >> 5);
+    if (chunk >= n_chunks) return;
+    const uint64_t base = chunk * kSelChunk;
+    const bool vec = ((uintptr_t)job.in & 15u) == 0 && base + kSelChunk <= job.d;
+    // the whole chunk's input first (eight 16-byte loads in flight per lane), whatever the mask keeps
+    float xs[8][4];
+    if (vec) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if ((nib >> j) & 1u) job.out[pos++] = xs[j];
+        for (int i = 0; i < 8; ++i) {
+            const float4 x4 = *reinterpret_cast<const float4*>(job.in + base + 128u * i + 4u * lane);
+            xs[i][0] = x4.x; xs[i][1] = x4.y; xs[i][2] = x4.z; xs[i][3] = x4.w;
+        }
     } else {
 #pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint64_t c = base + 128u * i + 4u * lane + j;
+                xs[i][j] = c < job.d ? job.in[c] : 0.f;
+            }
+    }
+    const ChunkMask m = chunk_mask(job.keep, chunk);
+    float* out = job.out + job.chunks[chunk];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t nib;
+        uint32_t pos = piece_position(m, i, nib);
+#pragma unroll
         for (int j = 0; j < 4; ++j)
-            if ((nib >> j) & 1u) job.out[pos++] = job.in[t * 4 + j];
+            if ((nib >> j) & 1u) out[pos++] = xs[i][j];
     }
 }
 
-// Receiver: out[i] += sum over the jobs of yhat_c[pos_c(i)] for the coordinates job c kept.
+// Receiver: out[i] += sum over the jobs of yhat_c[pos_c(i)] for the coordinates job c kept
+// (Section 4.1: the receiver restores through the same mask).  One pass over out.
 __global__ void __launch_bounds__(kSelThreads)
-k_selc_scatter(const SelJob* __restrict__ jobs, uint32_t n_jobs, uint64_t d, float* __restrict__ out)
+k_selc_scatter(const SelJob* __restrict__ jobs, uint32_t n_jobs, uint64_t d, float* __restrict__ out,
+               uint64_t n_chunks)
 {
-    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    float add[4] = {0.f, 0.f, 0.f, 0.f};
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint64_t chunk = (uint64_t)blockIdx.x * (kSelThreads / 32) + (threadIdx.x >> 5);
+    if (chunk >= n_chunks) return;
+    const uint64_t base = chunk * kSelChunk;
+    float add[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) add[i][j] = 0.f;
     for (uint32_t c = 0; c < n_jobs; ++c) {
         const SelJob job = jobs[c];
-        uint32_t nib;
-        uint64_t pos = keep_position(job.keep, nib) + job.chunks[blockIdx.x];
+        const ChunkMask m = chunk_mask(job.keep, chunk);
+        const float* in = job.in + job.chunks[chunk];
 #pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if ((nib >> j) & 1u) add[j] += job.in[pos++];
+        for (int i = 0; i < 8; ++i) {
+            uint32_t nib;
+            uint32_t pos = piece_position(m, i, nib);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if ((nib >> j) & 1u) add[i][j] += in[pos++];
+        }
     }
+    const bool vec = ((uintptr_t)out & 15u) == 0 && base + kSelChunk <= d;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const uint64_t i = t * 4 + j;
-        if (i < d && add[j] != 0.f) out[i] += add[j];
+    for (int i = 0; i < 8; ++i) {
+        const uint64_t c0 = base + 128u * i + 4u * lane;
+        if (vec) {
+            if (add[i][0] != 0.f || add[i][1] != 0.f || add[i][2] != 0.f || add[i][3] != 0.f) {
+                float4* p = reinterpret_cast<float4*>(out + c0);
+                float4 v = *p;
+                v.x += add[i][0]; v.y += add[i][1]; v.z += add[i][2]; v.w += add[i][3];
+                *p = v;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (c0 + j < d && add[i][j] != 0.f) out[c0 + j] += add[i][j];
+        }
     }
 }
 
