@@ -369,6 +369,14 @@ int eden_force_generic_kernels(eden_ctx* ctx, int on);
                                      one slab's second pass can overlap the next slab's first */
 int eden_set_option(eden_ctx* ctx, int option, int value);
 
+/* Host only, no GPU: the band of 32-bit keys [*lo, *hi] in which form 1 of the mask
+ * selection (EDEN_OPT_SEL_ROUNDS) expects the threshold of a mask that keeps k of d
+ * coordinates (Section 4.1: a sample of exactly d*p coordinates; the keys that rank them
+ * are uniform 32-bit words), `tenths` being EDEN_OPT_SEL_BAND's value.  *lo > *hi: no
+ * prediction (the band would not fit the candidate list, or tenths = 0).  Returns
+ * EDEN_ERR_INVALID_ARG for k = 0, k > d, tenths outside 0..120 or null pointers. */
+int eden_mask_threshold_band(uint64_t d, uint64_t k, int tenths, uint32_t* lo, uint32_t* hi);
+
 /* Optional per-kernel timing for benchmarks: while enabled, every kernel launch is
  * bracketed by CUDA events on the context's stream.  eden_profile_collect synchronises
  * and folds the records since eden_profile_enable(ctx, 1) into one entry per kernel

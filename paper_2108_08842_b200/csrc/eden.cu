@@ -1211,8 +1211,9 @@ int run_selection(eden_ctx* ctx, const FixedLayout& f, uint64_t seed, uint64_t d
 namespace {
 
 // Selection jobs of a group of clients with b < 1.  The scratch sits behind the group's
-// work buffers: n MaskSelect slots, n double histograms (contiguous, cleared by one
-// memset), n chunk arrays, then the job table itself.
+// work buffers, or in the arena of a call that selects ahead (SelectionAhead): n MaskSelect
+// slots, n histogram triples (contiguous with the slots, cleared by one memset), n chunk
+// arrays, the job table itself, then the candidate lists and the mask bitmaps.
 struct SelBatch {
     SelJob* d_jobs;
     uint32_t n;
@@ -1368,6 +1369,13 @@ struct SelectionAhead {
 };
 
 }  // namespace
+
+extern "C" int eden_mask_threshold_band(uint64_t d, uint64_t k, int tenths, uint32_t* lo, uint32_t* hi)
+{
+    if (!lo || !hi || d == 0 || k == 0 || k > d || tenths < 0 || tenths > 120) return EDEN_ERR_INVALID_ARG;
+    predicted_band(d, k, tenths, lo, hi);
+    return EDEN_OK;
+}
 
 // How one client's transform is split into sweeps over HBM (host only).
 extern "C" int eden_pass_plan(uint64_t d, double bits, uint32_t* pass_bits, uint32_t max_passes,

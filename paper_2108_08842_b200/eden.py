@@ -74,6 +74,7 @@ _sig("eden_profile_enable", _int, [_vp, _int])
 _sig("eden_force_generic_kernels", _int, [_vp, _int])
 _sig("eden_set_option", _int, [_vp, _int, _int])
 _sig("eden_self_check", _int, [])
+_sig("eden_mask_threshold_band", _int, [_u64, _u64, _int, _vp, _vp])
 _sig("eden_after_kept_count", _u64, [_u64, _f64])
 _sig("eden_after_code_bytes", _u64, [_u64, _f64])
 _sig("eden_after_workspace_bytes", _u64, [_u64, _u32])
@@ -129,6 +130,13 @@ def recv_mask_words(d: int, bits: float) -> int:
 
 def workspace_bytes(d_max: int, n_batch: int) -> int:
     return int(_lib.eden_workspace_bytes(d_max, n_batch))
+
+
+def mask_threshold_band(d: int, k: int, tenths: int = 40):
+    """eden_mask_threshold_band: (lo, hi) of the band of keys predicted to hold the mask's threshold."""
+    lo, hi = ctypes.c_uint32(), ctypes.c_uint32()
+    _check(_lib.eden_mask_threshold_band(d, k, tenths, ctypes.byref(lo), ctypes.byref(hi)))
+    return int(lo.value), int(hi.value)
 
 
 def after_kept_count(d: int, bits: float) -> int:

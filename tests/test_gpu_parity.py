@@ -531,20 +531,22 @@ def test_host_buffer_entry_points(E, d, n):
     assert np.max(np.abs(out.astype(np.float64) - ref)) <= MEAN_TOL * np.max(np.abs(ref))
 
 
-@pytest.mark.parametrize("d,bits", [(20000, 2.0), ((1 << 21) + 7, 1.0)])
+@pytest.mark.parametrize("d,bits", [(20000, 2.0), ((1 << 21) + 7, 1.0), ((1 << 17) + 5, (2.0, 0.5, 0.25))])
 def test_output_vector_that_is_only_4_byte_aligned(E, d, bits):
     # mean / acc one float past a 16-byte boundary: the receiver must not use its 128-bit
-    # stores on it (it takes the shape-generic kernels) and gives the same mean
+    # accesses on it (the transform takes the shape-generic kernels, the scatter of the b < 1
+    # senders its scalar form) and gives the same mean
     n = 3
+    bits = list(bits) if isinstance(bits, tuple) else [bits] * n
     rng = np.random.default_rng(d)
     xs = rng.standard_normal((n, d)).astype(np.float32)
     seeds = [int(s) for s in synth.client_seeds(d + 3, n)]
-    enc = [O.encode(xs[c], bits, seeds[c]) for c in range(n)]
-    ref, _ = O.mean([e["codes"] for e in enc], [float(np.float32(e["scale"])) for e in enc], [bits] * n, seeds, d)
+    enc = [O.encode(xs[c], bits[c], seeds[c]) for c in range(n)]
+    ref, _ = O.mean([e["codes"] for e in enc], [float(np.float32(e["scale"])) for e in enc], bits, seeds, d)
     ctx = _ctx(E, d, n)
     g_codes = []
-    for e in enc:
-        buf = np.zeros(E.code_bytes(d, bits), dtype=np.uint8)
+    for e, b in zip(enc, bits):
+        buf = np.zeros(E.code_bytes(d, b), dtype=np.uint8)
         buf[: e["codes"].nbytes] = e["codes"].view(np.uint8)
         g_codes.append(torch.from_numpy(buf).cuda())
     g_scales = torch.tensor([np.float32(e["scale"]) for e in enc], dtype=torch.float32, device="cuda")
@@ -552,12 +554,12 @@ def test_output_vector_that_is_only_4_byte_aligned(E, d, bits):
     assert buf.data_ptr() % 16 == 0
     out = buf[1:1 + d]
     launches = ctx.launch_count
-    ctx.mean(g_codes, g_scales, [bits] * n, seeds, d, None, out)
+    ctx.mean(g_codes, g_scales, bits, seeds, d, None, out)
     assert ctx.status() == 0 and ctx.launch_count > launches
     got = buf.cpu().numpy()
     assert got[0] == 0 and np.all(got[1 + d:] == 0)                 # nothing outside the vector
     assert np.max(np.abs(got[1:1 + d].astype(np.float64) - ref)) <= MEAN_TOL * np.max(np.abs(ref))
-    ctx.decode_accumulate(g_codes, g_scales, [bits] * n, seeds, d, out)
+    ctx.decode_accumulate(g_codes, g_scales, bits, seeds, d, out)
     got = buf.cpu().numpy()
     assert got[0] == 0 and np.all(got[1 + d:] == 0)
     assert np.max(np.abs(got[1:1 + d].astype(np.float64) - (1 + n) * ref)) <= MEAN_TOL * (1 + n) * np.max(np.abs(ref))

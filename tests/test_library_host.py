@@ -197,3 +197,40 @@ def test_uniform_family_host_figures_match_the_oracle(lib):
     assert lib.eden_encode_uniform(None, None, 0, 8, 1, None, None, None, None) == -1
     assert lib.eden_mean_uniform(None, None, None, None, None, None, 8, 1, None) == -1
     assert lib.eden_index_histogram(None, None, 8, 1, None) == -1
+
+
+def test_predicted_band_of_the_mask_threshold(lib):
+    # Section 4.1: the mask keeps exactly k of d coordinates, the k smallest 32-bit keys.  The
+    # one-pass selection predicts where the k-th smallest key lies; here the prediction is set
+    # against the oracle's keys: four standard deviations hold it nearly always, one standard
+    # deviation about two times in three (so centre and width are both right), and the band
+    # is empty where it could not fit the candidate list or is switched off
+    band = lib.eden_mask_threshold_band
+    band.restype = ctypes.c_int
+    band.argtypes = [ctypes.c_uint64, ctypes.c_uint64, ctypes.c_int,
+                     ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ctypes.c_uint32)]
+    lo, hi = ctypes.c_uint32(), ctypes.c_uint32()
+    d, trials = 2048, 120
+    for k in (205, 1024, 1900):
+        inside4 = inside1 = 0
+        for seed in range(1, trials + 1):
+            keys = np.sort(np.array([O.mask_key(seed, i) for i in range(d)], dtype=np.uint64))
+            tau = int(keys[k - 1])
+            assert band(d, k, 40, lo, hi) == 0
+            inside4 += lo.value <= tau <= hi.value
+            assert band(d, k, 10, lo, hi) == 0
+            inside1 += lo.value <= tau <= hi.value
+        assert inside4 >= trials - 1, (k, inside4)
+        assert 0.5 * trials <= inside1 <= 0.85 * trials, (k, inside1)
+    # width: 8 standard deviations of the k-th smallest of d uniform keys, sqrt(p(1-p)/d) 2^32 each
+    assert band(1 << 23, 1 << 22, 40, lo, hi) == 0
+    sd = np.sqrt(0.25 / (1 << 23)) * 2.0 ** 32
+    assert abs((hi.value - lo.value) - 8 * sd) < 0.01 * 8 * sd
+    assert abs((hi.value + lo.value) / 2 - 2.0 ** 31) < 4
+    # no room for twelve standard deviations of candidates at 2^27 coordinates: narrowed, not dropped
+    assert band(1 << 27, 1 << 26, 120, lo, hi) == 0 and lo.value < hi.value
+    expected = (1 << 27) * (hi.value - lo.value + 1) / 2.0 ** 32
+    assert 55000 < expected < 61440
+    assert band(1 << 20, 1000, 0, lo, hi) == 0 and lo.value > hi.value      # switched off
+    assert band(1 << 20, 0, 40, lo, hi) == -1 and band(1 << 20, (1 << 20) + 1, 40, lo, hi) == -1
+    assert band(1 << 20, 5, 121, lo, hi) == -1
