@@ -425,23 +425,48 @@ __device__ __forceinline__ void collect_chunk(const SelJob& job, uint64_t chunk,
 {
     const uint32_t lane = threadIdx.x & 31u;
     const bool empty = lo > hi;
+    const uint32_t span = hi - lo;
     uint32_t word = 0u;
     const uint64_t t0 = chunk * (kSelChunk / 4) + lane * 8u;
+    if (t0 * 4 + 32 <= job.d) {
+        // all 32 coordinates exist: no bounds checks, and four Philox calls at a time with
+        // nothing between them, so that their multiply chains interleave
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        const uint64_t t = t0 + c;
-        if (t * 4 >= job.d) break;
-        const uint4 k4 = mask_keys(job.seed, t);
-        const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
+        for (int half = 0; half < 2; ++half) {
+            uint4 k4[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const uint64_t i = t * 4 + j;
-            if (i >= job.d) break;
-            if (keys[j] < lo) {
-                word |= 1u << (4 * c + j);
-            } else if (keys[j] <= hi && !empty) {
-                const uint32_t slot = atomicAdd(&job.hist[kSelBins], 1u);
-                if (slot < kSelCandCap) job.cand[slot] = make_uint2(keys[j], (uint32_t)i);
+            for (int c = 0; c < 4; ++c) k4[c] = mask_keys(job.seed, t0 + 4 * half + c);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t keys[4] = {k4[c].x, k4[c].y, k4[c].z, k4[c].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int bit = 16 * half + 4 * c + j;
+                    word |= (keys[j] < lo ? 1u : 0u) << bit;
+                    if (keys[j] - lo <= span && !empty) {
+                        const uint32_t slot = atomicAdd(&job.hist[kSelBins], 1u);
+                        if (slot < kSelCandCap) job.cand[slot] = make_uint2(keys[j], (uint32_t)(t0 * 4) + bit);
+                    }
+                }
+            }
+        }
+    } else {
+#pragma unroll 1
+        for (int c = 0; c < 8; ++c) {
+            const uint64_t t = t0 + c;
+            if (t * 4 >= job.d) break;
+            const uint4 k4 = mask_keys(job.seed, t);
+            const uint32_t keys[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint64_t i = t * 4 + j;
+                if (i >= job.d) break;
+                if (keys[j] < lo) {
+                    word |= 1u << (4 * c + j);
+                } else if (keys[j] <= hi && !empty) {
+                    const uint32_t slot = atomicAdd(&job.hist[kSelBins], 1u);
+                    if (slot < kSelCandCap) job.cand[slot] = make_uint2(keys[j], (uint32_t)i);
+                }
             }
         }
     }
