@@ -121,10 +121,11 @@ int eden_pass_plan(uint64_t d, double bits, uint32_t* pass_bits, uint32_t max_pa
 int eden_table(uint32_t W, float* centroids, float* boundaries);
 
 /* Host only.  The kernels search the intervals of code widths 2..4 with multiply-adds whose
- * constants are derived from the table above; EDEN_OK if every boundary that search can
- * form is bit-identical to the table's fp32 boundary and no boundary is too small for the
- * kernels' exact comparison (both hold for the tables of Section 3; eden_create refuses
- * to run otherwise). */
+ * constants are derived from the table above, and those of widths 5..8 through a table of
+ * cells of width 2^-(W-2); EDEN_OK if every boundary that search can form is bit-identical
+ * to the table's fp32 boundary, no boundary is too small for the kernels' exact
+ * comparison, and no cell holds two boundaries (all hold for the tables of Section 3;
+ * eden_create refuses to run otherwise). */
 int eden_self_check(void);
 
 /* ---- context ---------------------------------------------------------------------- */

@@ -92,6 +92,9 @@ struct Tables {
     std::vector<float> centroids[9], boundaries[9];
     FmaTree tree[9];
     bool tree_exact;
+    float2 cells[9 - kCellMinWidth][kCellMax];
+    float cell_zmax[9];
+    int cell_count[9];
 };
 
 // fma(a, b, c) rounded towards zero, for a in {0, 1} and operands whose exact sum fits a double
@@ -171,6 +174,38 @@ bool build_fma_tree(int W, const float* pb, const float* pv, FmaTree& tr)
     return false;
 }
 
+// Cell table of the one-step interval search for code width W (see c_cells): false if a
+// cell would hold two boundaries or the table does not fit.
+bool build_cells(int W, const float* pb, float2* cells, float* zmax, int* count)
+{
+    const int n_bound = (1 << (W - 1)) - 1;
+    const double K = (double)(1 << (W - 2));               // cells per unit
+    const int n_cells = (int)std::floor((double)pb[n_bound - 1] * K) + 2;
+    if (n_cells > kCellMax) return false;
+    int j = 0;                                              // boundaries below the current cell
+    for (int c = 0; c < n_cells; ++c) {
+        const double lo = c / K, hi = (c + 1) / K;
+        int inside = 0;
+        float t_in = 0.f;
+        while (j + inside < n_bound && (double)pb[j + inside] < hi) {
+            if ((double)pb[j + inside] < lo) return false;  // not sorted
+            t_in = pb[j + inside];
+            ++inside;
+        }
+        if (inside > 1) return false;
+        uint32_t bits = 4u * (uint32_t)j;
+        float count_as_float;
+        std::memcpy(&count_as_float, &bits, sizeof(float));
+        cells[c].x = inside ? -1073741824.f * t_in : -3.0e38f;
+        cells[c].y = count_as_float;
+        j += inside;
+    }
+    if (j != n_bound) return false;
+    *zmax = (float)((n_cells - 0.5) / K);                   // exact: a small multiple of a power of two
+    *count = n_cells;
+    return true;
+}
+
 const Tables& tables()
 {
     static Tables t;
@@ -205,6 +240,12 @@ const Tables& tables()
                 t.tree_exact = build_fma_tree(4, coarse, t.pos_value + off, t.tree[W]) && t.tree_exact;
             }
         }
+        std::memset(t.cells, 0, sizeof(t.cells));
+        std::memset(t.cell_zmax, 0, sizeof(t.cell_zmax));
+        std::memset(t.cell_count, 0, sizeof(t.cell_count));
+        for (int W = kCellMinWidth; W <= 8; ++W)
+            t.tree_exact = build_cells(W, t.pos_boundary + (1 << (W - 1)) - 1, t.cells[W - kCellMinWidth],
+                                       &t.cell_zmax[W], &t.cell_count[W]) && t.tree_exact;
     });
     return t;
 }
@@ -427,6 +468,9 @@ extern "C" int eden_create(eden_ctx** out, int cuda_device, void* cuda_stream,
         return EDEN_ERR_INVALID_ARG;
     }
     if (cudaMemcpyToSymbol(c_tree, t.tree, sizeof(t.tree)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_cells, t.cells, sizeof(t.cells)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_cell_zmax, t.cell_zmax, sizeof(t.cell_zmax)) != cudaSuccess ||
+        cudaMemcpyToSymbol(c_cell_count, t.cell_count, sizeof(t.cell_count)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_pos_boundary, t.pos_boundary, sizeof(t.pos_boundary)) != cudaSuccess ||
         cudaMemcpyToSymbol(c_pos_value, t.pos_value, sizeof(t.pos_value)) != cudaSuccess ||
         cudaMemsetAsync(ctx->ws, 0, 256, ctx->stream) != cudaSuccess ||

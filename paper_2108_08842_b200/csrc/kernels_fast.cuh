@@ -705,14 +705,39 @@ __device__ __forceinline__ void fma_magnitude_pair(float az0, float az1, const T
     m1 = __float_as_uint(f1);
 }
 
+// The wide tables (W >= kCellMinWidth) in one step per coordinate (see c_cells): clamp, the
+// cell's byte offset straight from the mantissa of |z| 2^(W+1) + 2^23 rounded towards zero
+// (eight bytes per cell, three fraction bits masked off), one 64-bit load, one saturated
+// multiply-add; the pair's indices (times four) by one packed multiply-add.
+template <int W>
+__device__ __forceinline__ void cell_magnitude_pair(float az0, float az1, const float2* cells, float zmax,
+                                                    uint32_t& m0, uint32_t& m1)
+{
+    static_assert(W >= kCellMinWidth && W <= 8, "code widths with a cell table");
+    constexpr float k8 = (float)(8 << (W - 2));
+    static_assert(kCellMax * 8 <= 0x1000, "the offset mask below");
+    const float c0 = fminf(az0, zmax), c1 = fminf(az1, zmax);
+    const uint32_t o0 = __float_as_uint(__fmaf_rz(c0, k8, 8388608.f)) & 0xFF8u;
+    const uint32_t o1 = __float_as_uint(__fmaf_rz(c1, k8, 8388608.f)) & 0xFF8u;
+    const float2 e0 = *reinterpret_cast<const float2*>(reinterpret_cast<const char*>(cells) + o0);
+    const float2 e1 = *reinterpret_cast<const float2*>(reinterpret_cast<const char*>(cells) + o1);
+    const u64 ind = pack2(fma_sat(c0, 1073741824.f, e0.x), fma_sat(c1, 1073741824.f, e1.x));
+    const float four = __uint_as_float(4u);                // subnormal: its bit pattern is the integer
+    float f0, f1;
+    unpack2(fma2(ind, pack2(four, four), pack2(e0.y, e1.y)), f0, f1);
+    m0 = __float_as_uint(f0);
+    m1 = __float_as_uint(f1);
+}
+
 // The thread's 32 consecutive coordinates -> their W words of the code bit stream
 // (coordinate l in bits [l*W, l*W + W) of the 32*W-bit group), and sum |h| Q(|z|)
 // (accumulated as sum |z| Q(|z|) for W > 1, so that |z| = |h| / ||y|| is formed once).
 template <int W>
 __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_norm, bool live,
-                                                 const float* s_tb, const float* s_tv,
+                                                 const float* s_tb, const float* s_tv, const float2* s_cells,
                                                  uint32_t (&words)[W], float& dot)
 {
+    [[maybe_unused]] const float zmax = c_cell_zmax[W];
     constexpr uint32_t half = 1u << (W - 1);
     if constexpr (W == 1) {
         // one bit per coordinate: the code is "not negative" and Q(|z|) is the same value
@@ -755,7 +780,8 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
                 uint32_t m0, m1;
                 float q0, q1;
                 u64 root = 0ull;
-                fma_magnitude_pair<W>(az0, az1, tp, m0, m1, root, s_tb);
+                if constexpr (W >= kCellMinWidth) cell_magnitude_pair<W>(az0, az1, s_cells, zmax, m0, m1);
+                else fma_magnitude_pair<W>(az0, az1, tp, m0, m1, root, s_tb);
                 if constexpr (W == 2) {
                     // two values: the smaller plus the indicator times their distance (the sum may
                     // miss the larger value by one unit in the last place, far inside the scale's tolerance)
@@ -793,8 +819,9 @@ __device__ __forceinline__ void quantise_pack_32(const u64 (&v)[16], float inv_n
         unpack2(v[k], h[0], h[1]);
         const float az2[2] = {fabsf(h[0]) * inv_norm, fabsf(h[1]) * inv_norm};
         uint32_t m2[2];
-        u64 root;
-        fma_magnitude_pair<W>(az2[0], az2[1], tp, m2[0], m2[1], root, s_tb);
+        [[maybe_unused]] u64 root;
+        if constexpr (W >= kCellMinWidth) cell_magnitude_pair<W>(az2[0], az2[1], s_cells, zmax, m2[0], m2[1]);
+        else fma_magnitude_pair<W>(az2[0], az2[1], tp, m2[0], m2[1], root, s_tb);
 #pragma unroll
         for (int e = 1; e >= 0; --e) {
             const int l = 2 * k + e;
@@ -976,6 +1003,8 @@ template <int W, bool FRAC>
 struct EncTables {
     float tb[1 << (W - 1)], tv[1 << (W - 1)];
     float tb0[FRAC && W > 1 ? 1 << (W - 2) : 1], tv0[FRAC && W > 1 ? 1 << (W - 2) : 1];
+    // one-step search of the wide tables (integer budgets): see c_cells
+    float2 cells[!FRAC && W >= kCellMinWidth ? kCellMax : 1];
     // uniform-interval family (W = 8): the 128 values of this client by magnitude index
     __device__ __forceinline__ void fill_uniform(int t, const float* __restrict__ values)
     {
@@ -989,6 +1018,8 @@ struct EncTables {
             tb[j] = -1073741824.f * c_pos_boundary[table_offset(W) + j];
             tv[j] = c_pos_value[table_offset(W) + j];
         }
+        if constexpr (!FRAC && W >= kCellMinWidth)
+            for (int j = t; j < c_cell_count[W]; j += kFastThreads) cells[j] = c_cells[W - kCellMinWidth][j];
         if (FRAC)
             for (int j = t; j < (half >> 1); j += kFastThreads) {
                 tb0[j] = -1073741824.f * c_pos_boundary[table_offset(W > 1 ? W - 1 : 1) + j];
@@ -1055,7 +1086,7 @@ __device__ __forceinline__ float enc_last_tile(u64 (&v)[16], const ClientDesc& c
         const uint32_t coins = group_coins(cd.seed, (base >> 5) + t, cd.coin_thr);
         quantise_pack_frac<W>(v, inv_norm, live, coins, tab.tb, tab.tv, tab.tb0, tab.tv0, words, dot);
     } else {
-        quantise_pack_32<W>(v, inv_norm, live, tab.tb, tab.tv, words, dot);
+        quantise_pack_32<W>(v, inv_norm, live, tab.tb, tab.tv, tab.cells, words, dot);
     }
     __builtin_assume(__isGlobal(cd.codes));
     store_words<W>(cd.codes + ((base >> 5) + t) * W, words);

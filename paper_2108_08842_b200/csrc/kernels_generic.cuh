@@ -95,6 +95,20 @@ struct FmaTree {
 };
 __constant__ FmaTree c_tree[9];  // by code width
 
+// The same search for the wide tables (W >= kCellMinWidth) in one step: the positive axis is
+// cut into cells of width 2^-(W-2), narrower than the smallest gap between two boundaries of
+// the table, so that a cell holds at most one boundary; floor(|z| 2^(W-2)) picks the cell,
+// whose entry gives that boundary (as -2^30 t; a cell without one holds -3e38, which never
+// fires) and the number of boundaries below the cell, and one saturated multiply-add decides
+// the boundary inside.  Entry: x = -2^30 t, y = the float whose bit pattern is four times
+// the count (the byte offset of a value in a table of floats).  The last cell lies wholly
+// above the last boundary, and |z| is clamped to its middle (c_cell_zmax).
+constexpr int kCellMinWidth = 5;
+constexpr int kCellMax = 288;
+__constant__ float2 c_cells[9 - kCellMinWidth][kCellMax];
+__constant__ float c_cell_zmax[9];
+__constant__ int c_cell_count[9];
+
 // Interval rule of Section 2.2.1 on one normalised coordinate: magnitude index m =
 // number of positive boundaries strictly below |z| (an endpoint belongs to the interval
 // nearer zero), by a branch-free binary search over the sorted boundaries in `tb`.
