@@ -234,3 +234,22 @@ def test_predicted_band_of_the_mask_threshold(lib):
     assert band(1 << 20, 1000, 0, lo, hi) == 0 and lo.value > hi.value      # switched off
     assert band(1 << 20, 0, 40, lo, hi) == -1 and band(1 << 20, (1 << 20) + 1, 40, lo, hi) == -1
     assert band(1 << 20, 5, 121, lo, hi) == -1
+
+
+def test_wide_tables_fit_one_boundary_per_cell(lib):
+    # the sender searches the tables of code widths 5..8 through cells of width 2^-(W-2)
+    # (Section 2.2.1's interval rule in one step): that is exact only if no cell
+    # [c 2^-(W-2), (c+1) 2^-(W-2)) holds two of the table's positive fp32 boundaries, and the
+    # table of cells must fit its 288 entries.  Checked here on the library's own tables and
+    # on the oracle's, independently of eden_self_check.
+    for W in range(5, 9):
+        cent = (ctypes.c_float * (1 << W))()
+        bnd = (ctypes.c_float * ((1 << W) - 1))()
+        assert lib.eden_table(W, cent, bnd) == 0
+        for pos in (np.array([b for b in bnd if b > 0], dtype=np.float64),
+                    np.array([b for b in O.table(W)[1] if b > 0], dtype=np.float64)):
+            assert pos.size == (1 << (W - 1)) - 1
+            cells = np.floor(pos * (1 << (W - 2))).astype(np.int64)
+            assert np.unique(cells).size == cells.size, W
+            assert cells.max() + 2 <= 288
+    assert lib.eden_self_check() == 0
