@@ -257,7 +257,18 @@ def run_gpu(args):
     if work.drop_prob > 0:
         masks_np = [work.recv_mask(c, eden.num_packets(d, float(bits[c]))) for c in range(n)]
         masks_gpu = [torch.from_numpy(m.view(np.int32)).to(dev) for m in masks_np]
-    ctx = eden.Context(local_rank, d_max=d, n_batch=n, host_staging=True)
+    after = args.after_bits is not None
+    if after:
+        # Section 4.1's other order: the mask over the rotated coordinates (b < 1, no packet loss)
+        if not 0.0 < args.after_bits < 1.0:
+            raise SystemExit("--after-bits: a budget below one bit")
+        work.bits = np.full(n, float(args.after_bits))
+        work.drop_prob = 0.0
+        bits = work.bits
+        masks_np = masks_gpu = None
+        work.quantiser = "sparsification after the rotation, b=%g" % args.after_bits
+    ctx = eden.Context(local_rank, workspace_bytes_=eden.after_workspace_bytes(d, n) if after else None,
+                       d_max=d, n_batch=n, host_staging=True)
     if args.sel_rounds:
         ctx.set_option(eden.OPT_SEL_ROUNDS, args.sel_rounds)
     if args.sel_inline:
@@ -286,6 +297,14 @@ def run_gpu(args):
 
         def mean_step():
             ctx.mean_uniform(codes, scales, deltas, seeds, d, masks_gpu, mean)
+    elif after:
+        codes = [torch.empty(eden.after_code_bytes(d, float(b)), dtype=torch.uint8, device=dev) for b in bits]
+
+        def encode_step():
+            ctx.encode_sparsify_after(x_gpu, bits, seeds, codes, scales)
+
+        def mean_step():
+            ctx.mean_sparsify_after(codes, scales, bits, seeds, d, mean)
     else:
         codes = ctx.alloc_codes(d, bits)
 
@@ -379,7 +398,7 @@ def run_gpu(args):
                     "peak_source": "of " + peak_kind, "unit": "GB/s", "frac": achieved / peak,
                     "frac_of_nominal_8000": achieved / 8000.0,
                     "traffic": (traffic_table[top_name] * n * float(eden.rot_dim(d, float(bits[0])))
-                                if top_name in traffic_table and len(set(map(float, bits))) == 1 else None),
+                                if top_name in traffic_table and len(set(map(float, bits))) == 1 and not after else None),
                     "traffic_source": "ncu dram__bytes_read+write, one client, scaled by clients per launch "
                                       "(profiles/ncu_dram_traffic.txt; null if the kernels changed since the capture)",
                     "algorithmic_bytes_per_launch": top["bytes"] / top["launches"],
@@ -402,7 +421,7 @@ def run_gpu(args):
     # ---- end to end: same step through the host-buffer entry points (pinned memory),
     #      host->device and device->host copies inside the timed region
     e2e = None
-    if not args.no_e2e and not uniform and not args.sharded:
+    if not args.no_e2e and not uniform and not after and not args.sharded:
         codes_h = [torch.empty(eden.code_bytes(d, float(b)), dtype=torch.uint8, pin_memory=True).numpy()
                    for b in bits]
         scales_h = torch.empty(n, dtype=torch.float32, pin_memory=True).numpy()
@@ -434,7 +453,7 @@ def run_gpu(args):
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not uniform and not args.sharded:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not uniform and not after and not args.sharded:
         # one wave of clients at the workload's own dimension (the same rotation the GPU is timed on)
         threads = min(cores, n, 8)
         sample = synth.make(args.workload, d=d, n=threads, seed=rank)
@@ -562,6 +581,9 @@ def main():
                          "Lloyd-Max tables; device-resident timing only (no end-to-end or CPU leg)")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="experiment: no per-kernel event bracketing in the timed region (no kernel table, no roofline)")
+    ap.add_argument("--after-bits", type=float, default=None,
+                    help="time Section 4.1's other order instead (eden_encode_sparsify_after / eden_mean_sparsify_after "
+                         "at this budget below one bit for every sender, no packet loss); device-resident timing only")
     ap.add_argument("--sel-rounds", type=int, default=0,
                     help="experiment: form of the b < 1 mask selection (EDEN_OPT_SEL_ROUNDS; 0 keeps the default)")
     ap.add_argument("--sel-inline", action="store_true",

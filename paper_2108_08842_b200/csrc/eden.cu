@@ -1682,7 +1682,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
                          const double* bits, const double* delta, const uint64_t* seeds,
                          const uint32_t* const* recv_masks, uint64_t d, uint32_t n,
                          float* out, uint64_t divisor /* 0: accumulate into out; else overwrite out with the sum / divisor */,
-                         uint32_t recv_shift = 10)
+                         uint32_t recv_shift = 10, const uint32_t* recv_ones = nullptr /* per client: set bits of its bitmap, if known */)
 {
     if (!ctx || !codes || !scales || !seeds || !out || ((uintptr_t)out & 3u)) return EDEN_ERR_INVALID_ARG;
     const bool mean = divisor != 0;
@@ -1730,6 +1730,7 @@ static int decode_common(eden_ctx* ctx, const uint8_t* const* codes, const float
             cd.codes = (uint32_t*)codes[p.index];
             cd.recv = recv_masks ? recv_masks[p.index] : nullptr;
             cd.recv_shift = recv_shift;
+            cd.recv_ones = recv_ones ? recv_ones[p.index] : 0u;
             cd.seed = seeds[p.index];
             cd.valid = p.k;
             cd.d = d;
@@ -2076,6 +2077,12 @@ extern "C" int eden_encode_sparsify_after(eden_ctx* ctx, const float* x, uint64_
     if (rc) return rc;
     for (uint32_t c = 0; c < n; ++c)
         if (!codes[c] || ((uintptr_t)codes[c] & 15u)) return EDEN_ERR_INVALID_ARG;
+    std::vector<const void*> in(n);
+    std::vector<void*> out(n);
+    for (uint32_t c = 0; c < n; ++c) {
+        in[c] = ac.full[c];
+        out[c] = codes[c];
+    }
     // the whole vector with one bit per rotated coordinate, exactly as for b = 1
     const std::vector<double> one(n, 1.0);
     const uint64_t saved = ctx->ws_bytes;
@@ -2083,13 +2090,8 @@ extern "C" int eden_encode_sparsify_after(eden_ctx* ctx, const float* x, uint64_
     rc = encode_common(ctx, x, ld_x, d, n, one.data(), nullptr, seeds, ac.full.data(), scales);
     ctx->ws_bytes = saved;
     if (rc) return rc;
-    std::vector<const void*> in(n);
-    std::vector<void*> out(n);
-    for (uint32_t c = 0; c < n; ++c) {
-        in[c] = ac.full[c];
-        out[c] = codes[c];
+    for (uint32_t c = 0; c < n; ++c)
         CUDA_OK(cudaMemsetAsync(codes[c], 0, eden_after_code_bytes(d, bits[c]), ctx->stream));
-    }
     rc = after_select(ctx, ac, n, bits, seeds, in, out);
     if (rc) return rc;
     const uint64_t n_chunks = (ac.D + kSelChunk - 1) / kSelChunk;
@@ -2122,8 +2124,10 @@ static int after_decode(eden_ctx* ctx, const uint8_t* const* codes, const float*
     const std::vector<double> one(n, 1.0);
     const uint64_t saved = ctx->ws_bytes;
     ctx->ws_bytes = ac.head_bytes;
+    std::vector<uint32_t> kept(n);                     // the masks have exactly this many ones (Section 4.1)
+    for (uint32_t c = 0; c < n; ++c) kept[c] = (uint32_t)eden_kept_count(ac.D, bits[c]);
     rc = decode_common(ctx, (const uint8_t* const*)ac.full.data(), scales, one.data(), nullptr, seeds,
-                       ac.batch.keep.data(), d, n, out, divisor, 0);
+                       ac.batch.keep.data(), d, n, out, divisor, 0, kept.data());
     ctx->ws_bytes = saved;
     return rc;
 }

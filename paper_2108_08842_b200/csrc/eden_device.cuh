@@ -23,7 +23,7 @@ struct ClientDesc {
     uint32_t coin_thr;       // non-integer b > 1: coin threshold round(frac * 256); else 0
     float delta;             // uniform-interval family (Section 4.3): interval width; else 0
     uint32_t recv_shift;     // log2 coordinates per bit of `recv`: 10 (packets), or 0 (one bit per coordinate, W = 1 only)
-    uint32_t reserved;
+    uint32_t recv_ones;      // the number of set bits of `recv` where the caller knows it (a mask of exact size), else 0
     double extra_scale;      // encode: d/k for b < 1 (folded into S), else 1
     double mean_scale;       // decode: 1/n for the mean, 1 for accumulate
     const float* utable;     // uniform-interval family: values of magnitude index 0..127; else nullptr

@@ -298,14 +298,30 @@ k_dec_prep(const ClientDesc* __restrict__ descs, ClientState* __restrict__ state
     const uint64_t per_bit = 1ull << cd.recv_shift;                  // coordinates per bit of the bitmap
     const uint64_t packets = (D + per_bit - 1) >> cd.recv_shift;
     double cnt = 0.0;
-    if (cd.recv) {
+    if (cd.recv && cd.recv_ones) {
+        if (threadIdx.x == 0) cnt = (double)cd.recv_ones;            // a mask of known size: nothing to count
+    } else if (cd.recv) {
         const uint64_t words = (packets + 31) >> 5;
-        for (uint64_t w = threadIdx.x; w < words; w += blockDim.x) {
-            uint32_t v = cd.recv[w];
-            const uint64_t left = packets - (w << 5);
-            if (left < 32) v &= (1u << left) - 1u;
-            cnt += (double)__popc(v);
+        // eight loads in flight per thread: a bitmap with one bit per coordinate (the mask of the
+        // other order of Section 4.1) is megabytes long and one block walks it
+        uint32_t ones = 0u;
+        for (uint64_t w0 = threadIdx.x; w0 < words; w0 += 8ull * blockDim.x) {
+            uint32_t v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const uint64_t w = w0 + (uint64_t)u * blockDim.x;
+                v[u] = w < words ? cd.recv[w] : 0u;
+                const uint64_t left = w < words ? packets - (w << 5) : 32;
+                if (left < 32) v[u] &= (1u << left) - 1u;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) ones += (uint32_t)__popc(v[u]);
+            if (ones >= 0x80000000u) {                      // keep the 32-bit partial count from wrapping
+                cnt += (double)ones;
+                ones = 0u;
+            }
         }
+        cnt += (double)ones;
     } else if (threadIdx.x == 0) {
         cnt = (double)packets;
     }

@@ -23,9 +23,11 @@ def _bits(words, k):
     return ((words[:, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(-1)[:k]
 
 
-def run_after(E, xs, bits, seeds, threads=4):
+def run_after(E, xs, bits, seeds, threads=4, options=()):
     n, d = xs.shape
     ctx = E.Context(0, workspace_bytes_=E.after_workspace_bytes(d, n))
+    for opt, val in options:
+        ctx.set_option(opt, val)
     codes, scales = ctx.encode_sparsify_after(torch.from_numpy(xs).cuda(), bits, seeds)
     torch.cuda.synchronize()
     assert ctx.status() == 0
@@ -66,6 +68,18 @@ def run_after(E, xs, bits, seeds, threads=4):
     assert err <= MEAN_TOL * n * np.max(np.abs(ref)) + 1e-6
     ctx.close()
     return mism, ref
+
+
+@pytest.mark.parametrize("options", [[(3, 2)], [(7, 0)]], ids=["histogram_form", "every_job_redone"])
+def test_selection_forms_give_the_same_message(E, options):
+    # the mask's threshold comes from the predicted band (the default, every other test of
+    # this file), from the histogram form, or from the redo path
+    n, d = 3, (1 << 18) + 29
+    rng = np.random.default_rng(18)
+    xs = (rng.standard_normal((n, d)) * 2).astype(np.float32)
+    assert (E.OPT_SEL_ROUNDS, E.OPT_SEL_BAND) == (3, 7)
+    mism, _ = run_after(E, xs, [0.5, 0.1, 0.93], synth.client_seeds(77, n), options=options)
+    assert mism <= 4
 
 
 @pytest.mark.parametrize("d", [1, 33, 1000, 8192, 8193, 40000, (1 << 17) + 3, 1 << 20])
