@@ -1975,6 +1975,22 @@ extern "C" int eden_sparsification_mask(eden_ctx* ctx, uint64_t seed, uint64_t d
     CUDA_OK(cudaSetDevice(ctx->device));
     const FixedLayout f = fixed_layout(d);
     if (f.end > ctx->ws_bytes) return EDEN_ERR_WORKSPACE;
+    // where the workspace has room for it, the batched selection with one job (one pass over
+    // the keys, see start_selection_batch), whose mask bitmap is the answer
+    const uint64_t region = align_up(f.end, 256);
+    if (two_pass_selection(ctx, d) && region + sel_scratch_bytes(ctx, d) <= ctx->ws_bytes) {
+        std::vector<SelJob> jobs(1);
+        std::memset(&jobs[0], 0, sizeof(SelJob));
+        jobs[0].seed = seed;
+        jobs[0].d = d;
+        jobs[0].k = eden_kept_count(d, bits);
+        SelBatch batch;
+        const int rc = start_selection_batch(ctx, ctx->ws + region, d, jobs, batch);
+        if (rc) return rc;
+        CUDA_OK(cudaMemcpyAsync(mask_bits, batch.keep[0], (d + 31) / 32 * sizeof(uint32_t), cudaMemcpyDeviceToDevice,
+                                ctx->stream));
+        return EDEN_OK;
+    }
     const int rc = run_selection(ctx, f, seed, d, eden_kept_count(d, bits));
     if (rc) return rc;
     const unsigned grid = (unsigned)(((d + 3) / 4 + kSelThreads - 1) / kSelThreads);
